@@ -1,0 +1,461 @@
+/*
+ * boa_oracle.c -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+ *
+ * A plain, slow, single-threaded CPU statement of what the batched adaptive
+ * filtered beam search computes.  Only the tests, the smoke check and the
+ * benchmark's cpu_baseline / reference arm may build, load or call it.  It
+ * shares no code, header, table or helper with the CUDA library.
+ *
+ * What each function follows:
+ *   orc_phi            filter distance: number of the query's closed range
+ *                      predicates a point violates (Background, "Graph
+ *                      construction", last paragraph; Eq. 2 gives g = [phi == 0])
+ *   orc_bruteforce     exact range-filtered k-NN (Definition 1, Definition 2, Eq. 1)
+ *   orc_beam_*         filter-aware beam search at one beamwidth (Algorithm 2),
+ *                      with exact L2 distances instead of PQ look-ups
+ *   orc_uncertain      confidence test gamma(D_i) <= eps (Eq. 3)
+ *   orc_boa_search     multi-phase driver (Algorithm 1)
+ *
+ * Readings of points the paper leaves open (each is listed in the design notes):
+ *   - the score dist + lambda*phi is taken in its lambda -> infinity limit: keys
+ *     order by (phi, d2, id) lexicographically; id breaks every tie
+ *   - "visited" means two things in Algorithm 2: a node already scored ("seen",
+ *     the Bloom filter line, here an exact set) and a node already expanded (a
+ *     flag on the worklist entry, the convergence line)
+ *   - distances are squared L2 in fp32; two ways to accumulate them are offered:
+ *     mode 0 sums in double and rounds once, mode 1 uses the 8-way interleaved
+ *     fp32 order described at orc_dist2_lanes
+ *   - a query whose beam holds at most k filter-valid entries is uncertain
+ *   - restart mode runs every phase from the entry point with pool capacity L;
+ *     resume mode keeps pool, flags and seen set, pool capacity Lmax, and only
+ *     lengthens the expandable prefix (reading of "redundancy avoidance")
+ *   - a phase stops after cap_mult*L + cap_add expansions at the latest
+ *
+ * parity pins: tests/test_oracle_pins.py (brute force vs. an independent sort,
+ * g == 1 vs. a library k-NN, the ring-graph hand trace, full-graph search ==
+ * brute force, restart/resume relations, eps special cases, L_avg vs. the
+ * paper's Table III).  Unpinned by the paper itself: the exact trajectories on
+ * large inputs, the constants alpha, tau, lambda.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORC_SENTINEL 0xFFFFFFFFu
+#define ORC_F32 0
+#define ORC_U8 1
+#define ORC_ATTR_I32 0
+#define ORC_ATTR_F32 1
+
+typedef struct {
+    int64_t N;
+    int D, m, R, vec_dtype;
+    const void *vectors;      /* [N][D] float or uint8_t       */
+    const int32_t *attrs;     /* [N][m] 4-byte cells           */
+    const int32_t *attr_types; /* [m]                          */
+    const uint32_t *graph;    /* [N][R], ORC_SENTINEL = no edge */
+    int64_t entry;
+} orc_index;
+
+/* ------------------------------------------------------------------ */
+/* element access                                                      */
+/* ------------------------------------------------------------------ */
+static float orc_elem(const orc_index *ix, int64_t p, int i)
+{
+    if (ix->vec_dtype == ORC_U8)
+        return (float)((const uint8_t *)ix->vectors)[p * ix->D + i];
+    return ((const float *)ix->vectors)[p * ix->D + i];
+}
+
+/* squared L2 distance, summed in double in index order (mode 0 rounds this to float) */
+double orc_dist2_f64(const orc_index *ix, const float *q, int64_t p)
+{
+    double s = 0.0;
+    for (int i = 0; i < ix->D; ++i) {
+        double d = (double)orc_elem(ix, p, i) - (double)q[i];
+        s += d * d;
+    }
+    return s;
+}
+
+/*
+ * Squared L2 distance in fp32, in a fixed order so that a second fp32
+ * implementation can reproduce it bit for bit.  The row is cut into chunks of
+ * 16 bytes (4 floats or 16 bytes of uint8).  Chunk c belongs to partial sum
+ * c mod 8.  Each partial sum runs over its chunks in ascending order and over
+ * the elements of a chunk in ascending order with
+ *     acc = fmaf(x - q, x - q, acc)        (x - q rounded to fp32 first).
+ * The eight partial sums are then added pairwise:
+ *     ((p0+p4) + (p2+p6)) + ((p1+p5) + (p3+p7)).
+ */
+float orc_dist2_lanes(const orc_index *ix, const float *q, int64_t p)
+{
+    const int per = (ix->vec_dtype == ORC_U8) ? 16 : 4;
+    const int nchunks = (ix->D + per - 1) / per;
+    float part[8];
+    for (int g = 0; g < 8; ++g) {
+        float acc = 0.0f;
+        for (int c = g; c < nchunks; c += 8) {
+            for (int j = 0; j < per; ++j) {
+                int i = c * per + j;
+                if (i >= ix->D) break;
+                float diff = orc_elem(ix, p, i) - q[i];
+                acc = fmaf(diff, diff, acc);
+            }
+        }
+        part[g] = acc;
+    }
+    float a04 = part[0] + part[4], a15 = part[1] + part[5];
+    float a26 = part[2] + part[6], a37 = part[3] + part[7];
+    float e = a04 + a26, o = a15 + a37;
+    return e + o;
+}
+
+static float orc_dist2(const orc_index *ix, const float *q, int64_t p, int dist_mode)
+{
+    if (dist_mode == 1) return orc_dist2_lanes(ix, q, p);
+    return (float)orc_dist2_f64(ix, q, p);
+}
+
+/* number of violated closed range predicates; bounds use the column's own type */
+int orc_phi(const orc_index *ix, const int32_t *lo, const int32_t *hi, int64_t p)
+{
+    int v = 0;
+    for (int j = 0; j < ix->m; ++j) {
+        int32_t cell = ix->attrs[p * ix->m + j];
+        if (ix->attr_types[j] == ORC_ATTR_F32) {
+            float a, l, h;
+            memcpy(&a, &cell, 4);
+            memcpy(&l, &lo[j], 4);
+            memcpy(&h, &hi[j], 4);
+            if (!(a >= l && a <= h)) v++;      /* NaN violates */
+        } else {
+            if (cell < lo[j] || cell > hi[j]) v++;
+        }
+    }
+    return v;
+}
+
+/* ------------------------------------------------------------------ */
+/* index                                                               */
+/* ------------------------------------------------------------------ */
+/* point nearest (squared L2 in double, lower id wins ties) to the coordinate mean */
+int64_t orc_medoid(const orc_index *ix)
+{
+    double *mean = (double *)calloc((size_t)ix->D, sizeof(double));
+    for (int64_t p = 0; p < ix->N; ++p)
+        for (int i = 0; i < ix->D; ++i) mean[i] += (double)orc_elem(ix, p, i);
+    for (int i = 0; i < ix->D; ++i) mean[i] /= (double)ix->N;
+    int64_t best = 0;
+    double bestd = INFINITY;
+    for (int64_t p = 0; p < ix->N; ++p) {
+        double s = 0.0;
+        for (int i = 0; i < ix->D; ++i) {
+            double d = (double)orc_elem(ix, p, i) - mean[i];
+            s += d * d;
+        }
+        if (s < bestd) { bestd = s; best = p; }
+    }
+    free(mean);
+    return best;
+}
+
+orc_index *orc_create(const void *vectors, int vec_dtype, int64_t N, int D,
+                      const int32_t *attrs, const int32_t *attr_types, int m,
+                      const uint32_t *graph, int R, int64_t entry)
+{
+    orc_index *ix = (orc_index *)calloc(1, sizeof(orc_index));
+    ix->N = N; ix->D = D; ix->m = m; ix->R = R; ix->vec_dtype = vec_dtype;
+    ix->vectors = vectors; ix->attrs = attrs; ix->attr_types = attr_types; ix->graph = graph;
+    ix->entry = entry;
+    if (entry < 0) ix->entry = orc_medoid(ix);
+    return ix;
+}
+void orc_destroy(orc_index *ix) { free(ix); }
+int64_t orc_entry(const orc_index *ix) { return ix->entry; }
+
+/* ------------------------------------------------------------------ */
+/* exact filtered top-k (Definitions 1 and 2)                          */
+/* ------------------------------------------------------------------ */
+/* Returns |D_f|.  out_ids/out_d2 receive the min(k,|D_f|) valid points of
+   smallest distance, ascending by (d2, id); the rest is padded. */
+int64_t orc_bruteforce(const orc_index *ix, const float *q, const int32_t *lo, const int32_t *hi,
+                       int k, uint32_t *out_ids, double *out_d2)
+{
+    int have = 0;
+    int64_t nvalid = 0;
+    for (int i = 0; i < k; ++i) { out_ids[i] = ORC_SENTINEL; out_d2[i] = INFINITY; }
+    for (int64_t p = 0; p < ix->N; ++p) {
+        if (orc_phi(ix, lo, hi, p) != 0) continue;
+        nvalid++;
+        double d = orc_dist2_f64(ix, q, p);
+        /* ids ascend, so a strict < keeps the lower id ahead on equal distance */
+        int pos = have;
+        while (pos > 0 && d < out_d2[pos - 1]) pos--;
+        if (pos >= k) continue;
+        int last = (have < k) ? have : k - 1;
+        for (int t = last; t > pos; --t) { out_d2[t] = out_d2[t - 1]; out_ids[t] = out_ids[t - 1]; }
+        out_d2[pos] = d; out_ids[pos] = (uint32_t)p;
+        if (have < k) have++;
+    }
+    return nvalid;
+}
+
+/* ------------------------------------------------------------------ */
+/* filter-aware beam search (Algorithm 2)                              */
+/* ------------------------------------------------------------------ */
+typedef struct {
+    int phi;
+    float d2;
+    uint32_t id;
+    int expanded;
+} orc_entry_t;
+
+typedef struct {
+    const orc_index *ix;
+    int C;               /* pool capacity */
+    int size;
+    orc_entry_t *pool;   /* C + R slots, ascending by (phi, d2, id) */
+    uint8_t *seen;       /* [N] */
+    uint32_t *touched;   /* ids set in seen, for a cheap reset */
+    int64_t ntouched, touched_cap;
+    int64_t n_expand, n_scored;
+    int hit_cap;
+} orc_state;
+
+static int orc_less(const orc_entry_t *a, const orc_entry_t *b)
+{
+    if (a->phi != b->phi) return a->phi < b->phi;
+    if (a->d2 != b->d2) return a->d2 < b->d2;
+    return a->id < b->id;
+}
+
+orc_state *orc_state_new(const orc_index *ix, int C)
+{
+    orc_state *st = (orc_state *)calloc(1, sizeof(orc_state));
+    st->ix = ix; st->C = C;
+    st->pool = (orc_entry_t *)calloc((size_t)(C + ix->R + 1), sizeof(orc_entry_t));
+    st->seen = (uint8_t *)calloc((size_t)ix->N, 1);
+    st->touched_cap = 1024;
+    st->touched = (uint32_t *)malloc((size_t)st->touched_cap * sizeof(uint32_t));
+    return st;
+}
+void orc_state_free(orc_state *st)
+{
+    free(st->pool); free(st->seen); free(st->touched); free(st);
+}
+
+static void orc_mark_seen(orc_state *st, uint32_t id)
+{
+    st->seen[id] = 1;
+    if (st->ntouched == st->touched_cap) {
+        st->touched_cap *= 2;
+        st->touched = (uint32_t *)realloc(st->touched, (size_t)st->touched_cap * sizeof(uint32_t));
+    }
+    st->touched[st->ntouched++] = id;
+}
+
+static void orc_pool_insert(orc_state *st, orc_entry_t e)
+{
+    int pos = st->size;
+    while (pos > 0 && orc_less(&e, &st->pool[pos - 1])) { st->pool[pos] = st->pool[pos - 1]; pos--; }
+    st->pool[pos] = e;
+    st->size++;
+}
+
+/* L_i <- {s}: empty seen set, pool holding only the entry point */
+void orc_beam_init(orc_state *st, int C, const float *q, const int32_t *lo, const int32_t *hi, int dist_mode)
+{
+    const orc_index *ix = st->ix;
+    for (int64_t t = 0; t < st->ntouched; ++t) st->seen[st->touched[t]] = 0;
+    st->ntouched = 0; st->size = 0; st->C = C;
+    st->n_expand = 0; st->n_scored = 0; st->hit_cap = 0;
+    orc_entry_t e;
+    e.id = (uint32_t)ix->entry; e.expanded = 0;
+    e.phi = orc_phi(ix, lo, hi, ix->entry);
+    e.d2 = orc_dist2(ix, q, ix->entry, dist_mode);
+    orc_mark_seen(st, e.id);
+    orc_pool_insert(st, e);
+}
+
+/* run the loop of Algorithm 2 at beamwidth L until every one of the first L
+   pool entries is expanded; gives up (hit_cap) when an unexpanded entry is left
+   after max_expand expansions of this call */
+void orc_beam_run(orc_state *st, int L, const float *q, const int32_t *lo, const int32_t *hi,
+                  int dist_mode, int64_t max_expand)
+{
+    const orc_index *ix = st->ix;
+    int64_t done = 0;
+    st->hit_cap = 0;
+    for (;;) {
+        int lim = st->size < L ? st->size : L;
+        int u = -1;
+        for (int t = 0; t < lim; ++t)
+            if (!st->pool[t].expanded) { u = t; break; }
+        if (u < 0) break;                               /* converged */
+        if (done >= max_expand) { st->hit_cap = 1; break; }
+        st->pool[u].expanded = 1;
+        st->n_expand++; done++;
+        uint32_t uid = st->pool[u].id;
+        for (int j = 0; j < ix->R; ++j) {
+            uint32_t n = ix->graph[(int64_t)uid * ix->R + j];
+            if (n == ORC_SENTINEL || st->seen[n]) continue;
+            orc_mark_seen(st, n);
+            st->n_scored++;
+            orc_entry_t e;
+            e.id = n; e.expanded = 0;
+            e.phi = orc_phi(ix, lo, hi, n);
+            e.d2 = orc_dist2(ix, q, n, dist_mode);
+            orc_pool_insert(st, e);
+        }
+        if (st->size > st->C) st->size = st->C;          /* keep the C best */
+    }
+}
+
+/* K_i <- the k nearest filter-valid pool entries; returns how many there are */
+int orc_beam_result(const orc_state *st, int k, uint32_t *out_ids, float *out_d2)
+{
+    int have = 0;
+    for (int t = 0; t < st->size && have < k; ++t)
+        if (st->pool[t].phi == 0) { out_ids[have] = st->pool[t].id; out_d2[have] = st->pool[t].d2; have++; }
+    for (int t = have; t < k; ++t) { out_ids[t] = ORC_SENTINEL; out_d2[t] = INFINITY; }
+    return have;
+}
+
+int orc_state_size(const orc_state *st) { return st->size; }
+int64_t orc_state_expanded(const orc_state *st) { return st->n_expand; }
+int64_t orc_state_scored(const orc_state *st) { return st->n_scored; }
+int orc_state_hit_cap(const orc_state *st) { return st->hit_cap; }
+void orc_state_pool(const orc_state *st, uint32_t *ids, float *d2, int32_t *phi, int32_t *expanded)
+{
+    for (int t = 0; t < st->size; ++t) {
+        ids[t] = st->pool[t].id; d2[t] = st->pool[t].d2;
+        phi[t] = st->pool[t].phi; expanded[t] = st->pool[t].expanded;
+    }
+}
+
+/*
+ * Confidence test (Eq. 3).  V = filter-valid entries among the first L pool
+ * entries.  gamma = (d_max - d_k)/d_max on Euclidean norms; gamma <= eps is
+ * evaluated without square roots as d2_k >= (1-eps)^2 * d2_max, in fp32, the
+ * constant rounded once to float.  Returns 1 when the query must escalate.
+ */
+int orc_uncertain(const orc_state *st, int L, int k, double eps)
+{
+    int lim = st->size < L ? st->size : L;
+    int nv = 0;
+    float d2k = 0.0f, d2max = 0.0f;
+    for (int t = 0; t < lim; ++t) {
+        if (st->pool[t].phi != 0) continue;
+        nv++;
+        if (nv == k) d2k = st->pool[t].d2;
+        d2max = st->pool[t].d2;                           /* entries ascend */
+    }
+    if (nv <= k) return 1;
+    if (eps < 0.0) return 1;
+    if (eps >= 1.0) return 0;
+    float c = (float)((1.0 - eps) * (1.0 - eps));
+    float rhs = c * d2max;
+    return !(d2k >= rhs);
+}
+
+/* ------------------------------------------------------------------ */
+/* multi-phase driver (Algorithm 1)                                    */
+/* ------------------------------------------------------------------ */
+/* what resume mode carries from one phase of a query to the next: the pool
+   with its expanded flags, and the ids of the seen set */
+typedef struct {
+    int size;
+    orc_entry_t *pool;
+    int64_t ntouched;
+    uint32_t *touched;
+} orc_saved;
+
+static orc_saved *orc_save(const orc_state *st)
+{
+    orc_saved *sv = (orc_saved *)calloc(1, sizeof(orc_saved));
+    sv->size = st->size;
+    sv->pool = (orc_entry_t *)malloc((size_t)(st->size + 1) * sizeof(orc_entry_t));
+    memcpy(sv->pool, st->pool, (size_t)st->size * sizeof(orc_entry_t));
+    sv->ntouched = st->ntouched;
+    sv->touched = (uint32_t *)malloc((size_t)(st->ntouched + 1) * sizeof(uint32_t));
+    memcpy(sv->touched, st->touched, (size_t)st->ntouched * sizeof(uint32_t));
+    return sv;
+}
+static void orc_saved_free(orc_saved *sv)
+{
+    if (!sv) return;
+    free(sv->pool); free(sv->touched); free(sv);
+}
+/* put a saved search back into the working state */
+static void orc_restore(orc_state *st, const orc_saved *sv, int C)
+{
+    for (int64_t t = 0; t < st->ntouched; ++t) st->seen[st->touched[t]] = 0;
+    st->ntouched = 0; st->C = C;
+    st->n_expand = 0; st->n_scored = 0; st->hit_cap = 0;
+    for (int64_t t = 0; t < sv->ntouched; ++t) orc_mark_seen(st, sv->touched[t]);
+    st->size = sv->size;
+    memcpy(st->pool, sv->pool, (size_t)sv->size * sizeof(orc_entry_t));
+}
+
+/*
+ * widths[0..n_widths): beamwidth of each phase.  mode 0 = restart, 1 = resume.
+ * Outputs are indexed by the original query index whatever phase wrote them.
+ * phase_active[p] receives |A| at the start of phase p.  n_expand / n_scored
+ * add up over the phases a query ran; flags bit 0 = some phase hit its
+ * expansion cap.
+ */
+void orc_boa_search(const orc_index *ix, const float *queries, int64_t Q,
+                    const int32_t *lo, const int32_t *hi, int k,
+                    const int32_t *widths, int n_widths, double eps, double tau,
+                    int mode, int dist_mode, int cap_mult, int cap_add,
+                    uint32_t *out_ids, float *out_d2,
+                    int32_t *final_L, int32_t *n_expand, int32_t *n_scored, int32_t *flags,
+                    int64_t *phase_active)
+{
+    int Cmax = 0;
+    for (int p = 0; p < n_widths; ++p) if (widths[p] > Cmax) Cmax = widths[p];
+    orc_state *st = orc_state_new(ix, Cmax);
+    for (int p = 0; p < n_widths; ++p) phase_active[p] = 0;
+
+    uint8_t *active = (uint8_t *)malloc((size_t)Q + 1);             /* the set A */
+    orc_saved **saved = (orc_saved **)calloc((size_t)Q + 1, sizeof(orc_saved *));
+    for (int64_t i = 0; i < Q; ++i) {
+        active[i] = 1; final_L[i] = 0; n_expand[i] = 0; n_scored[i] = 0; flags[i] = 0;
+        for (int t = 0; t < k; ++t) { out_ids[i * k + t] = ORC_SENTINEL; out_d2[i * k + t] = INFINITY; }
+    }
+    int64_t n_active = Q;
+    for (int p = 0; p < n_widths; ++p) {                            /* one phase per turn */
+        if (!((double)n_active > tau * (double)Q)) break;           /* while |A| > tau*rho */
+        phase_active[p] = n_active;
+        const int L = widths[p];
+        const int64_t cap = (int64_t)cap_mult * L + cap_add;
+        for (int64_t i = 0; i < Q; ++i) {
+            if (!active[i]) continue;
+            const float *q = queries + i * ix->D;
+            const int32_t *l = lo + i * ix->m, *h = hi + i * ix->m;
+            if (mode == 1 && saved[i]) {
+                orc_restore(st, saved[i], Cmax);
+                orc_saved_free(saved[i]); saved[i] = NULL;
+            } else {
+                orc_beam_init(st, mode == 1 ? Cmax : L, q, l, h, dist_mode);
+            }
+            orc_beam_run(st, L, q, l, h, dist_mode, cap);
+            orc_beam_result(st, k, out_ids + i * k, out_d2 + i * k);    /* scatter */
+            final_L[i] = L;
+            n_expand[i] += (int32_t)st->n_expand;
+            n_scored[i] += (int32_t)st->n_scored;
+            if (st->hit_cap) flags[i] |= 1;
+            if (!orc_uncertain(st, L, k, eps)) {                    /* F: confident */
+                active[i] = 0; n_active--;
+            } else if (mode == 1 && p + 1 < n_widths) {
+                saved[i] = orc_save(st);
+            }
+        }
+    }
+    for (int64_t i = 0; i < Q; ++i) orc_saved_free(saved[i]);
+    free(saved);
+    free(active);
+    orc_state_free(st);
+}
