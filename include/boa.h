@@ -1,0 +1,150 @@
+/*
+ * boa.h -- C interface of the B200 (sm_100a) library for batched, beamwidth-adaptive,
+ * range-filtered graph beam search (BOA / BOA+).
+ *
+ * All functions are extern "C", take plain pointers and sizes, return an int
+ * status (BOA_OK == 0, negative == error), never throw, abort or print.  Unless a
+ * parameter says "host", a pointer is a DEVICE pointer on the current CUDA
+ * device and must be 16-byte aligned.  The caller owns every buffer it passes.
+ * `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ */
+#ifndef BOA_H
+#define BOA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct boa_index boa_index; /* opaque */
+
+enum { BOA_F32 = 0, BOA_U8 = 1 };            /* element type of the stored vectors      */
+enum { BOA_ATTR_I32 = 0, BOA_ATTR_F32 = 1 }; /* cell type of one attribute column       */
+
+enum {
+    BOA_OK = 0,
+    BOA_EINVAL = -1, /* bad argument (null, range, alignment, unsupported shape) */
+    BOA_ENOMEM = -2, /* device or host allocation failed                         */
+    BOA_ECUDA = -3,  /* a CUDA call failed; boa_last_cuda_error() has its code   */
+    BOA_EGRAPH = -4  /* the graph names a node id >= N                           */
+};
+
+#define BOA_NO_ID 0xFFFFFFFFu /* "no edge" in graph rows, "no result" in out_ids */
+#define BOA_MAX_ATTRS 8
+#define BOA_MAX_DEGREE 64
+#define BOA_MAX_WIDTH 1024 /* largest beamwidth / pool capacity */
+#define BOA_MAX_PHASES 8
+#define BOA_MAX_POINTS ((int64_t)1 << 28)
+
+/* Keys of boa_set_param. */
+enum {
+    BOA_PARAM_EPS = 0,      /* confidence threshold eps of Eq. 3; default 0.05               */
+    BOA_PARAM_GROWTH = 1,   /* alpha of Algorithm 1: width of phase p+1 = min(Lmax, alpha*w_p); default 4 */
+    BOA_PARAM_TAU = 2,      /* residual fraction tau of Algorithm 1; default 0                */
+    BOA_PARAM_MODE = 3,     /* 0 = restart every phase from the entry point (Algorithm 1 as
+                               printed), 1 = resume: later phases continue from the pool the
+                               earlier ones built (the "redundancy avoidance" paragraph)      */
+    BOA_PARAM_PLUS_K = 4,   /* 0 or 1 = BOA; K >= 2 = BOA+: the first phase is issued as K
+                               sub-batches and wider phases overlap them ("Pipelining
+                               Multiple Batches")                                            */
+    BOA_PARAM_CAP_MULT = 5, /* a phase at width L gives up after CAP_MULT*L + CAP_ADD        */
+    BOA_PARAM_CAP_ADD = 6,  /*   expansions; defaults 8 and 64                               */
+    BOA_PARAM_HASH_LOG2 = 7 /* 0 = choose per phase; else log2 of the per-query table of
+                               recently scored ids (10..14).  Never changes results.         */
+};
+
+/*
+ * Build a search index (problem statement of the paper's Background section: points
+ * p = (x_p, a_p) with m numeric attributes, and a proximity graph of out-degree <= R).
+ *
+ *   vectors     [N][D] row-major, float (BOA_F32) or uint8_t (BOA_U8); D % 4 == 0 for
+ *               floats, D % 16 == 0 for bytes; values must be finite
+ *   attrs       [N][m] row-major 4-byte cells; column j is int32 or float per attr_types[j]
+ *   attr_types  HOST array [m]
+ *   graph       [N][R] node ids, BOA_NO_ID pads short rows; self references and
+ *               repeated ids inside a row are tolerated (ignored by the search)
+ *   entry       start node s of every search (Algorithm 2, "entry medoid s"); -1 = the
+ *               point nearest to the coordinate-wise mean, lower id on ties
+ *
+ * The index copies and re-lays-out everything into device memory it owns, so the
+ * inputs may be freed when the call returns.  The call synchronises `stream`.
+ * Errors: BOA_EINVAL (nulls, N < 1, N > BOA_MAX_POINTS, m outside 1..8, R outside 1..64,
+ * bad D, misaligned pointers, entry >= N), BOA_EGRAPH, BOA_ENOMEM, BOA_ECUDA.
+ */
+int boa_index_create(boa_index** out, const void* vectors, int vec_dtype, int64_t N, int D,
+                     const void* attrs, const int* attr_types, int m, const uint32_t* graph, int R,
+                     int64_t entry, void* stream);
+
+/* Free the index and everything it owns.  NULL is accepted. */
+int boa_index_destroy(boa_index* index);
+
+/* The start node the index uses (host value). */
+int64_t boa_index_entry(const boa_index* index);
+
+/*
+ * Algorithm 1 (BOA) over one batch: every query is searched with Algorithm 2
+ * (filter-aware beam search) at beamwidth L0; queries that fail the confidence test of
+ * Eq. 3 are compacted and searched again at wider beamwidths up to Lmax.  L0 == Lmax is
+ * the fixed-beamwidth baseline.
+ *
+ *   queries   [Q][D] float
+ *   lo, hi    [Q][m] closed bounds, cell types as the index's columns; lo > hi is legal
+ *             (empty valid set); an unconstrained attribute gets the type's full range
+ *   out_ids   [Q][k]  ids of the filter-valid nearest points found, ascending by
+ *             (squared distance, id), duplicate-free; BOA_NO_ID fills unused slots
+ *   out_dists [Q][k]  squared L2 distances in fp32; +inf in unused slots
+ *
+ * Asynchronous on `stream`: no host synchronisation; outputs are valid once the stream
+ * has run the enqueued work.  Scratch memory is owned by the index and grows (a device
+ * allocation) only when Q or Lmax exceed every earlier call's; two searches on one
+ * index must not overlap in time.  With BOA+ a second stream owned by the index is
+ * used and joined back into `stream` before the call's work ends.
+ * Errors (before any launch): BOA_EINVAL for nulls, Q < 0, k < 1, k > L0, L0 > Lmax,
+ * Lmax > BOA_MAX_WIDTH, misaligned pointers.  Q == 0 is a no-op.
+ */
+int boa_search(boa_index* index, const float* queries, int64_t Q, const void* lo, const void* hi,
+               int k, int L0, int Lmax, uint32_t* out_ids, float* out_dists, void* stream);
+
+/* Set one parameter (keys above).  BOA_EINVAL for an unknown key or a value out of range. */
+int boa_set_param(boa_index* index, int key, double value);
+
+/* Explicit phase widths (HOST array, strictly increasing, 1..BOA_MAX_PHASES entries)
+   replacing the geometric schedule of Algorithm 1; n == 0 restores it.  With an
+   explicit schedule boa_search requires L0 == widths[0] and Lmax == widths[n-1]. */
+int boa_set_schedule(boa_index* index, const int* widths, int n);
+
+/*
+ * Per-query statistics of the last boa_search on this index, copied on `stream` into
+ * caller DEVICE buffers of Q int32 each (any may be NULL):
+ *   final_L   width of the last phase the query ran (its mean is the paper's L_avg)
+ *   n_expand  nodes expanded, summed over the phases the query ran
+ *   n_scored  neighbour distances computed (a node forgotten by the bounded table of
+ *             scored ids and met again is counted again)
+ *   flags     bit 0: a phase stopped at its expansion cap
+ */
+int boa_get_stats(boa_index* index, int32_t* final_L, int32_t* n_expand, int32_t* n_scored,
+                  int32_t* flags, void* stream);
+
+/* Number of queries that entered each phase of the last search: writes up to n values
+   into the HOST array `active` and returns the number of phases in *n_phases.
+   Synchronises `stream`. */
+int boa_get_phase_counts(boa_index* index, int64_t* active, int n, int* n_phases, void* stream);
+
+/* Bytes of index-owned scratch a search of Q queries up to width Lmax needs. */
+int boa_workspace_bytes(const boa_index* index, int64_t Q, int Lmax, size_t* bytes);
+
+/* Number of kernel launches the last boa_search enqueued. */
+int boa_last_launch_count(const boa_index* index);
+
+/* cudaError_t of the most recent failing CUDA call made by this library (0 if none). */
+int boa_last_cuda_error(void);
+
+/* Static text for a status code. */
+const char* boa_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BOA_H */

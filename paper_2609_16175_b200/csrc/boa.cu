@@ -1,0 +1,662 @@
+// C interface of the library: index construction, the phase driver of Algorithm 1
+// (BOA) and the overlapped schedule of BOA+, statistics.  sm_100a only.
+#include "../../include/boa.h"
+
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "boa_search.cuh"
+
+namespace {
+
+thread_local int g_last_cuda = 0;
+
+#define BOA_CUDA(expr)                                   \
+    do {                                                 \
+        cudaError_t e__ = (expr);                        \
+        if (e__ != cudaSuccess) {                        \
+            g_last_cuda = (int)e__;                      \
+            return e__ == cudaErrorMemoryAllocation ? BOA_ENOMEM : BOA_ECUDA; \
+        }                                                \
+    } while (0)
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ------------------------------------------------------------------ index build kernels
+// Record i = [vector bytes | m attribute cells | zero padding], rec_stride bytes.
+__global__ void build_records_kernel(const uint8_t* __restrict__ vec, const int32_t* __restrict__ attrs,
+                                     uint8_t* __restrict__ rec, int64_t N, int vec_bytes, int m,
+                                     int stride)
+{
+    const int cps = stride / 16;
+    const int64_t total = N * cps;
+    for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total;
+         idx += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = idx / cps;
+        const int off = (int)(idx % cps) * 16;
+        uint4 v;
+        if (off + 16 <= vec_bytes) {
+            v = *reinterpret_cast<const uint4*>(vec + row * vec_bytes + off);
+        } else {
+            uint32_t w[4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int a = (off + 4 * t - vec_bytes) / 4;
+                w[t] = (a >= 0 && a < m) ? (uint32_t)attrs[row * m + a] : 0u;
+            }
+            v = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        *reinterpret_cast<uint4*>(rec + row * stride + off) = v;
+    }
+}
+
+// Copy the graph; self references and repeats inside a row become BOA_NO_ID, so the
+// search never meets one id twice in a row.  Flags ids >= N.
+__global__ void clean_graph_kernel(const uint32_t* __restrict__ in, uint32_t* __restrict__ out,
+                                   int64_t N, int R, int* __restrict__ bad)
+{
+    for (int64_t row = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; row < N;
+         row += (int64_t)gridDim.x * blockDim.x) {
+        const uint32_t* src = in + row * R;
+        uint32_t* dst = out + row * R;
+        for (int j = 0; j < R; ++j) {
+            uint32_t id = src[j];
+            if (id != BOA_NO_ID) {
+                if ((int64_t)id >= N) { atomicOr(bad, 1); id = BOA_NO_ID; }
+                else if ((int64_t)id == row) id = BOA_NO_ID;
+                else {
+                    for (int t = 0; t < j; ++t)
+                        if (src[t] == id) { id = BOA_NO_ID; break; }
+                }
+            }
+            dst[j] = id;
+        }
+    }
+}
+
+__device__ __forceinline__ double elem_at(const void* vec, int dtype, int64_t i)
+{
+    return dtype == BOA_U8 ? (double)reinterpret_cast<const uint8_t*>(vec)[i]
+                           : (double)reinterpret_cast<const float*>(vec)[i];
+}
+
+// partial[b][d] = sum over rows b, b+nb, b+2nb, ... of x[row][d]   (fixed order)
+__global__ void column_partial_kernel(const void* vec, int dtype, int64_t N, int D, double* partial)
+{
+    const int nb = gridDim.x;
+    for (int d = threadIdx.x; d < D; d += blockDim.x) {
+        double s = 0.0;
+        for (int64_t r = blockIdx.x; r < N; r += nb) s += elem_at(vec, dtype, r * D + d);
+        partial[(size_t)blockIdx.x * D + d] = s;
+    }
+}
+__global__ void column_mean_kernel(const double* partial, int nb, int64_t N, int D, double* mean)
+{
+    const int d = blockIdx.x * blockDim.x + threadIdx.x;
+    if (d >= D) return;
+    double s = 0.0;
+    for (int b = 0; b < nb; ++b) s += partial[(size_t)b * D + d];
+    mean[d] = s / (double)N;
+}
+// One warp per point: squared distance to the mean in double; per-block argmin.
+__global__ void medoid_block_kernel(const void* vec, int dtype, int64_t N, int D, const double* mean,
+                                    double* best_d, int64_t* best_i)
+{
+    __shared__ double sd[8];
+    __shared__ int64_t si[8];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    double bd = INFINITY;
+    int64_t bi = INT64_MAX;
+    for (int64_t r = blockIdx.x * 8 + warp; r < N; r += (int64_t)gridDim.x * 8) {
+        double s = 0.0;
+        for (int d = lane; d < D; d += 32) {
+            const double x = elem_at(vec, dtype, r * D + d) - mean[d];
+            s += x * x;
+        }
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (s < bd || (s == bd && r < bi)) { bd = s; bi = r; }
+    }
+    if (lane == 0) { sd[warp] = bd; si[warp] = bi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w)
+            if (sd[w] < bd || (sd[w] == bd && si[w] < bi)) { bd = sd[w]; bi = si[w]; }
+        best_d[blockIdx.x] = bd;
+        best_i[blockIdx.x] = bi;
+    }
+}
+
+__global__ void fill_outputs_kernel(uint32_t* ids, float* d2, int64_t n, int32_t* final_L,
+                                    int32_t* n_expand, int32_t* n_scored, int32_t* flags, int64_t Q)
+{
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        ids[i] = BOA_NO_ID;
+        d2[i] = __int_as_float(0x7f800000);
+        if (i < Q) { final_L[i] = 0; n_expand[i] = 0; n_scored[i] = 0; flags[i] = 0; }
+    }
+}
+
+// dst[0] = src[0]: freezes a survivor count at a point of a stream's order.
+__global__ void copy_word_kernel(uint32_t* dst, const uint32_t* src) { *dst = *src; }
+
+}  // namespace
+
+// ------------------------------------------------------------------ the index
+struct boa_index {
+    int64_t N = 0;
+    int D = 0, m = 0, R = 0, vec_dtype = 0;
+    int rec_stride = 0, nchunks = 0, attr_off = 0;
+    uint32_t attr_float_mask = 0;
+    int64_t entry = 0;
+    uint8_t* rec = nullptr;
+    uint32_t* graph = nullptr;
+    int device = 0, num_sms = 0;
+    // parameters
+    double eps = 0.05, growth = 4.0, tau = 0.0;
+    int mode = 0, plus_k = 0, cap_mult = 8, cap_add = 64, hash_log2 = 0;
+    int n_sched = 0;
+    int sched[BOA_MAX_PHASES] = {0};
+    // scratch
+    int64_t ws_Q = 0;
+    int ws_spill = 0;
+    uint32_t* lists = nullptr;     // [BOA_MAX_PHASES][ws_Q]
+    uint32_t* counters = nullptr;  // see enum below
+    int32_t* stats = nullptr;      // [4][ws_Q]
+    uint64_t* spill = nullptr;     // [ws_Q][ws_spill]
+    int32_t* spill_size = nullptr; // [ws_Q]
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    // last search
+    int64_t last_Q = 0;
+    int last_phases = 0;
+    int last_launches = 0;
+    int last_widths[BOA_MAX_PHASES] = {0};
+};
+
+namespace {
+// layout of boa_index::counters (uint32 words)
+constexpr int kCntCount = 0;                          // [P+1] survivors entering phase p (p>=1)
+constexpr int kCntConsumed = 16;                      // [P+1] list positions already searched
+constexpr int kCntSnap = 32;                          // [pool] frozen end of phase 1's list
+constexpr int kCntTicket = 48;                        // one per launch
+constexpr int kMaxLaunches = 128;
+constexpr int kCntWords = kCntTicket + kMaxLaunches;
+
+typedef void (*SearchKernel)(const boa::SearchParams);
+
+struct KernelChoice {
+    SearchKernel fn;
+    int rs;
+};
+
+template <int VT, int CPL, int U>
+KernelChoice pick_rs(int R)
+{
+    if (R <= 32) return {boa::boa_search_kernel<VT, CPL, 1, U>, 1};
+    return {boa::boa_search_kernel<VT, CPL, 2, U>, 2};
+}
+
+KernelChoice pick_kernel(const boa_index* ix)
+{
+    const int cpl = (ix->nchunks + 7) / 8;
+    if (ix->vec_dtype == BOA_F32) {
+        switch (cpl) {
+            case 1: return pick_rs<0, 1, 8>(ix->R);
+            case 2: return pick_rs<0, 2, 4>(ix->R);
+            case 3: return pick_rs<0, 3, 2>(ix->R);
+            case 4: return pick_rs<0, 4, 2>(ix->R);
+            default: return pick_rs<0, 0, 1>(ix->R);
+        }
+    }
+    switch (cpl) {
+        case 1: return pick_rs<1, 1, 8>(ix->R);
+        case 2: return pick_rs<1, 2, 4>(ix->R);
+        default: return pick_rs<1, 0, 1>(ix->R);
+    }
+}
+
+int choose_hash_log2(const boa_index* ix, int L)
+{
+    if (ix->hash_log2) return ix->hash_log2;
+    int want = 16 * L;              // about the ids one search at width L scores
+    int lg = 10;
+    while ((1 << lg) < want && lg < 13) ++lg;
+    return lg;
+}
+
+int phase_widths(const boa_index* ix, int L0, int Lmax, int* w)
+{
+    if (ix->n_sched > 0) {
+        for (int i = 0; i < ix->n_sched; ++i) w[i] = ix->sched[i];
+        return ix->n_sched;
+    }
+    int n = 0;
+    double cur = L0;
+    w[n++] = L0;
+    while (w[n - 1] < Lmax && n < BOA_MAX_PHASES) {
+        cur = cur * ix->growth;
+        int next = cur >= (double)Lmax ? Lmax : (int)cur;
+        if (next <= w[n - 1]) next = w[n - 1] + 1;
+        if (next > Lmax || n == BOA_MAX_PHASES - 1) next = Lmax;
+        w[n++] = next;
+    }
+    return n;
+}
+
+int ensure_workspace(boa_index* ix, int64_t Q, int Lmax)
+{
+    const int need_spill = ix->mode == 1 ? ((Lmax + 1) & ~1) : 0;
+    if (ix->counters == nullptr) {
+        BOA_CUDA(cudaMalloc(&ix->counters, kCntWords * sizeof(uint32_t)));
+    }
+    if (Q > ix->ws_Q || need_spill > ix->ws_spill) {
+        const int64_t nq = Q > ix->ws_Q ? Q : ix->ws_Q;
+        const int ns = need_spill > ix->ws_spill ? need_spill : ix->ws_spill;
+        cudaFree(ix->lists); cudaFree(ix->stats); cudaFree(ix->spill); cudaFree(ix->spill_size);
+        ix->lists = nullptr; ix->stats = nullptr; ix->spill = nullptr; ix->spill_size = nullptr;
+        ix->ws_Q = 0; ix->ws_spill = 0;
+        BOA_CUDA(cudaMalloc(&ix->lists, (size_t)BOA_MAX_PHASES * nq * sizeof(uint32_t)));
+        BOA_CUDA(cudaMalloc(&ix->stats, (size_t)4 * nq * sizeof(int32_t)));
+        BOA_CUDA(cudaMalloc(&ix->spill_size, (size_t)nq * sizeof(int32_t)));
+        if (ns > 0) BOA_CUDA(cudaMalloc(&ix->spill, (size_t)nq * ns * sizeof(uint64_t)));
+        ix->ws_Q = nq;
+        ix->ws_spill = ns;
+    }
+    return BOA_OK;
+}
+
+struct LaunchPlan {
+    boa_index* ix;
+    KernelChoice kc;
+    boa::SearchParams base;
+    int n_phases;
+    int widths[BOA_MAX_PHASES];
+    int launches;
+};
+
+// One launch of Algorithm 2 over positions [begin, end) of phase p's work list.
+int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_ptr,
+                 const uint32_t* end_ptr, uint32_t begin, uint32_t end, uint32_t expected_items)
+{
+    boa_index* ix = lp.ix;
+    if (lp.launches >= kMaxLaunches) return BOA_EINVAL;
+    boa::SearchParams sp = lp.base;
+    const int L = lp.widths[p];
+    const int Lmax = lp.widths[lp.n_phases - 1];
+    sp.L = L;
+    sp.C = ix->mode == 1 ? Lmax : L;
+    sp.hash_log2 = choose_hash_log2(ix, L);
+    sp.max_expand = ix->cap_mult * L + ix->cap_add;
+    sp.first_phase = p == 0;
+    sp.resume_in = (ix->mode == 1 && p > 0);
+    sp.last_phase = p == lp.n_phases - 1;
+    sp.spill_out = (ix->mode == 1 && !sp.last_phase);
+    sp.in_list = p == 0 ? nullptr : ix->lists + (size_t)p * ix->ws_Q;
+    sp.in_begin_ptr = begin_ptr;
+    sp.in_end_ptr = end_ptr;
+    sp.in_begin = begin;
+    sp.in_end = end;
+    sp.active_count = p == 0 ? nullptr : ix->counters + kCntCount + p;
+    sp.ticket = ix->counters + kCntTicket + lp.launches;
+    sp.out_list = ix->lists + (size_t)(p + 1 < BOA_MAX_PHASES ? p + 1 : p) * ix->ws_Q;
+    sp.out_count = ix->counters + kCntCount + p + 1;
+
+    const boa::WarpSmem lay = boa::warp_smem_layout(sp.C, sp.hash_log2, ix->D, lp.kc.rs);
+    const size_t smem = (size_t)lay.total * boa::kWarpsPerCta;
+    if (smem > 48 * 1024) {
+        BOA_CUDA(cudaFuncSetAttribute((const void*)lp.kc.fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)smem));
+    }
+    int per_sm = 0;
+    BOA_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, (const void*)lp.kc.fn,
+                                                           boa::kThreads, smem));
+    if (per_sm < 1) return BOA_EINVAL;
+    int64_t grid = (int64_t)per_sm * ix->num_sms;
+    const int64_t need = ((int64_t)expected_items + boa::kWarpsPerCta - 1) / boa::kWarpsPerCta;
+    if (need < grid) grid = need < 1 ? 1 : need;
+    lp.kc.fn<<<(unsigned)grid, boa::kThreads, smem, st>>>(sp);
+    BOA_CUDA(cudaGetLastError());
+    lp.launches++;
+    return BOA_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ C interface
+extern "C" {
+
+int boa_last_cuda_error(void) { return g_last_cuda; }
+
+const char* boa_strerror(int status)
+{
+    switch (status) {
+        case BOA_OK: return "ok";
+        case BOA_EINVAL: return "invalid argument";
+        case BOA_ENOMEM: return "out of memory";
+        case BOA_ECUDA: return "CUDA call failed";
+        case BOA_EGRAPH: return "graph names a node id outside the index";
+        default: return "unknown status";
+    }
+}
+
+int boa_index_create(boa_index** out, const void* vectors, int vec_dtype, int64_t N, int D,
+                     const void* attrs, const int* attr_types, int m, const uint32_t* graph, int R,
+                     int64_t entry, void* stream)
+{
+    if (!out) return BOA_EINVAL;
+    *out = nullptr;
+    if (!vectors || !attrs || !attr_types || !graph) return BOA_EINVAL;
+    if (N < 1 || N > BOA_MAX_POINTS) return BOA_EINVAL;
+    if (m < 1 || m > BOA_MAX_ATTRS || R < 1 || R > BOA_MAX_DEGREE) return BOA_EINVAL;
+    if (vec_dtype != BOA_F32 && vec_dtype != BOA_U8) return BOA_EINVAL;
+    if (D < 1 || (vec_dtype == BOA_F32 && D % 4 != 0) || (vec_dtype == BOA_U8 && D % 16 != 0))
+        return BOA_EINVAL;
+    if (D > 16384) return BOA_EINVAL;
+    if (!aligned16(vectors) || !aligned16(attrs) || !aligned16(graph)) return BOA_EINVAL;
+    if (entry >= N || entry < -1) return BOA_EINVAL;
+    for (int j = 0; j < m; ++j)
+        if (attr_types[j] != BOA_ATTR_I32 && attr_types[j] != BOA_ATTR_F32) return BOA_EINVAL;
+
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    boa_index* ix = new (std::nothrow) boa_index();
+    if (!ix) return BOA_ENOMEM;
+    auto fail = [&](int code) { boa_index_destroy(ix); return code; };
+#define BOA_TRY(expr)                                                      \
+    do {                                                                   \
+        cudaError_t e__ = (expr);                                          \
+        if (e__ != cudaSuccess) {                                          \
+            g_last_cuda = (int)e__;                                        \
+            return fail(e__ == cudaErrorMemoryAllocation ? BOA_ENOMEM : BOA_ECUDA); \
+        }                                                                  \
+    } while (0)
+
+    ix->N = N; ix->D = D; ix->m = m; ix->R = R; ix->vec_dtype = vec_dtype;
+    const int vec_bytes = vec_dtype == BOA_U8 ? D : 4 * D;
+    ix->nchunks = vec_bytes / 16;
+    ix->attr_off = vec_bytes;
+    ix->rec_stride = (vec_bytes + 4 * m + 31) & ~31;
+    for (int j = 0; j < m; ++j)
+        if (attr_types[j] == BOA_ATTR_F32) ix->attr_float_mask |= 1u << j;
+    BOA_TRY(cudaGetDevice(&ix->device));
+    BOA_TRY(cudaDeviceGetAttribute(&ix->num_sms, cudaDevAttrMultiProcessorCount, ix->device));
+    BOA_TRY(cudaMalloc(&ix->rec, (size_t)N * ix->rec_stride));
+    BOA_TRY(cudaMalloc(&ix->graph, (size_t)N * R * sizeof(uint32_t)));
+    BOA_TRY(cudaStreamCreateWithFlags(&ix->side, cudaStreamNonBlocking));
+    BOA_TRY(cudaEventCreateWithFlags(&ix->ev_fork, cudaEventDisableTiming));
+    BOA_TRY(cudaEventCreateWithFlags(&ix->ev_join, cudaEventDisableTiming));
+
+    const int blocks = ix->num_sms * 8;
+    build_records_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const uint8_t*>(vectors),
+                                                 reinterpret_cast<const int32_t*>(attrs), ix->rec, N,
+                                                 vec_bytes, m, ix->rec_stride);
+    BOA_TRY(cudaGetLastError());
+    int* d_bad = nullptr;
+    BOA_TRY(cudaMalloc(&d_bad, sizeof(int)));
+    cudaError_t e = cudaMemsetAsync(d_bad, 0, sizeof(int), st);
+    if (e == cudaSuccess) {
+        clean_graph_kernel<<<blocks, 128, 0, st>>>(graph, ix->graph, N, R, d_bad);
+        e = cudaGetLastError();
+    }
+    int h_bad = 0;
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&h_bad, d_bad, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    cudaFree(d_bad);
+    BOA_TRY(e);
+    if (h_bad) return fail(BOA_EGRAPH);
+
+    if (entry >= 0) {
+        ix->entry = entry;
+    } else {
+        // medoid: the point nearest to the coordinate-wise mean, lower id on ties
+        const int nb = (int)(N < 1024 ? N : 1024);
+        const int mb = (int)((N + 7) / 8 < 2048 ? (N + 7) / 8 : 2048);
+        double *partial = nullptr, *mean = nullptr, *bd = nullptr;
+        int64_t* bi = nullptr;
+        e = cudaMalloc(&partial, (size_t)nb * D * sizeof(double));
+        if (e == cudaSuccess) e = cudaMalloc(&mean, (size_t)D * sizeof(double));
+        if (e == cudaSuccess) e = cudaMalloc(&bd, (size_t)mb * sizeof(double));
+        if (e == cudaSuccess) e = cudaMalloc(&bi, (size_t)mb * sizeof(int64_t));
+        double* h_bd = (double*)malloc((size_t)mb * sizeof(double));
+        int64_t* h_bi = (int64_t*)malloc((size_t)mb * sizeof(int64_t));
+        if (e == cudaSuccess && h_bd && h_bi) {
+            column_partial_kernel<<<nb, 128, 0, st>>>(vectors, vec_dtype, N, D, partial);
+            column_mean_kernel<<<(D + 127) / 128, 128, 0, st>>>(partial, nb, N, D, mean);
+            medoid_block_kernel<<<mb, 256, 0, st>>>(vectors, vec_dtype, N, D, mean, bd, bi);
+            e = cudaGetLastError();
+            if (e == cudaSuccess)
+                e = cudaMemcpyAsync(h_bd, bd, (size_t)mb * sizeof(double), cudaMemcpyDeviceToHost, st);
+            if (e == cudaSuccess)
+                e = cudaMemcpyAsync(h_bi, bi, (size_t)mb * sizeof(int64_t), cudaMemcpyDeviceToHost, st);
+            if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+            if (e == cudaSuccess) {
+                double best = INFINITY;
+                int64_t besti = INT64_MAX;
+                for (int b = 0; b < mb; ++b)
+                    if (h_bd[b] < best || (h_bd[b] == best && h_bi[b] < besti)) {
+                        best = h_bd[b]; besti = h_bi[b];
+                    }
+                ix->entry = besti;
+            }
+        }
+        const bool host_oom = !h_bd || !h_bi;
+        free(h_bd); free(h_bi);
+        cudaFree(partial); cudaFree(mean); cudaFree(bd); cudaFree(bi);
+        if (host_oom) return fail(BOA_ENOMEM);
+        BOA_TRY(e);
+    }
+#undef BOA_TRY
+    *out = ix;
+    return BOA_OK;
+}
+
+int boa_index_destroy(boa_index* ix)
+{
+    if (!ix) return BOA_OK;
+    cudaFree(ix->rec); cudaFree(ix->graph); cudaFree(ix->lists); cudaFree(ix->counters);
+    cudaFree(ix->stats); cudaFree(ix->spill); cudaFree(ix->spill_size);
+    if (ix->side) cudaStreamDestroy(ix->side);
+    if (ix->ev_fork) cudaEventDestroy(ix->ev_fork);
+    if (ix->ev_join) cudaEventDestroy(ix->ev_join);
+    delete ix;
+    return BOA_OK;
+}
+
+int64_t boa_index_entry(const boa_index* ix) { return ix ? ix->entry : -1; }
+
+int boa_set_param(boa_index* ix, int key, double v)
+{
+    if (!ix || v != v) return BOA_EINVAL;
+    switch (key) {
+        case BOA_PARAM_EPS: ix->eps = v; return BOA_OK;
+        case BOA_PARAM_GROWTH: if (!(v > 1.0)) return BOA_EINVAL; ix->growth = v; return BOA_OK;
+        case BOA_PARAM_TAU: if (v < 0.0) return BOA_EINVAL; ix->tau = v; return BOA_OK;
+        case BOA_PARAM_MODE: if (v != 0.0 && v != 1.0) return BOA_EINVAL; ix->mode = (int)v; return BOA_OK;
+        case BOA_PARAM_PLUS_K:
+            if (v < 0.0 || v > 64.0 || v != floor(v)) return BOA_EINVAL;
+            ix->plus_k = (int)v; return BOA_OK;
+        case BOA_PARAM_CAP_MULT:
+            if (v < 0.0 || v > 1024.0 || v != floor(v)) return BOA_EINVAL;
+            ix->cap_mult = (int)v; return BOA_OK;
+        case BOA_PARAM_CAP_ADD:
+            if (v < 0.0 || v > 1e6 || v != floor(v)) return BOA_EINVAL;
+            ix->cap_add = (int)v; return BOA_OK;
+        case BOA_PARAM_HASH_LOG2:
+            if (v != 0.0 && (v < 10.0 || v > 14.0 || v != floor(v))) return BOA_EINVAL;
+            ix->hash_log2 = (int)v; return BOA_OK;
+        default: return BOA_EINVAL;
+    }
+}
+
+int boa_set_schedule(boa_index* ix, const int* widths, int n)
+{
+    if (!ix || n < 0 || n > BOA_MAX_PHASES || (n > 0 && !widths)) return BOA_EINVAL;
+    for (int i = 0; i < n; ++i) {
+        if (widths[i] < 1 || widths[i] > BOA_MAX_WIDTH) return BOA_EINVAL;
+        if (i > 0 && widths[i] <= widths[i - 1]) return BOA_EINVAL;
+    }
+    ix->n_sched = n;
+    for (int i = 0; i < n; ++i) ix->sched[i] = widths[i];
+    return BOA_OK;
+}
+
+int boa_workspace_bytes(const boa_index* ix, int64_t Q, int Lmax, size_t* bytes)
+{
+    if (!ix || !bytes || Q < 0 || Lmax < 1 || Lmax > BOA_MAX_WIDTH) return BOA_EINVAL;
+    size_t b = kCntWords * sizeof(uint32_t);
+    b += (size_t)BOA_MAX_PHASES * Q * sizeof(uint32_t) + (size_t)5 * Q * sizeof(int32_t);
+    if (ix->mode == 1) b += (size_t)Q * ((Lmax + 1) & ~1) * sizeof(uint64_t);
+    *bytes = b;
+    return BOA_OK;
+}
+
+int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, const void* hi, int k,
+               int L0, int Lmax, uint32_t* out_ids, float* out_dists, void* stream)
+{
+    if (!ix) return BOA_EINVAL;
+    if (Q < 0 || Q > (int64_t)0x7FFFFFFF) return BOA_EINVAL;
+    if (k < 1 || k > L0 || L0 > Lmax || Lmax > BOA_MAX_WIDTH) return BOA_EINVAL;
+    if (ix->n_sched > 0 && (L0 != ix->sched[0] || Lmax != ix->sched[ix->n_sched - 1])) return BOA_EINVAL;
+    if (Q == 0) { ix->last_Q = 0; ix->last_phases = 0; ix->last_launches = 0; return BOA_OK; }
+    if (!queries || !lo || !hi || !out_ids || !out_dists) return BOA_EINVAL;
+    if (!aligned16(queries) || !aligned16(lo) || !aligned16(hi) || !aligned16(out_ids) ||
+        !aligned16(out_dists))
+        return BOA_EINVAL;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+
+    int rc = ensure_workspace(ix, Q, Lmax);
+    if (rc != BOA_OK) return rc;
+
+    LaunchPlan lp;
+    lp.ix = ix;
+    lp.kc = pick_kernel(ix);
+    lp.n_phases = phase_widths(ix, L0, Lmax, lp.widths);
+    lp.launches = 0;
+    boa::SearchParams& b = lp.base;
+    memset(&b, 0, sizeof(b));
+    b.rec = ix->rec; b.graph = ix->graph; b.N = ix->N; b.D = ix->D; b.m = ix->m; b.R = ix->R;
+    b.rec_stride = ix->rec_stride; b.nchunks = ix->nchunks; b.attr_off = ix->attr_off;
+    b.attr_float_mask = ix->attr_float_mask; b.entry = (uint32_t)ix->entry;
+    b.queries = queries;
+    b.lo = reinterpret_cast<const int32_t*>(lo);
+    b.hi = reinterpret_cast<const int32_t*>(hi);
+    b.out_ids = out_ids; b.out_d2 = out_dists; b.Q = Q; b.k = k;
+    b.tau_q = ix->tau * (double)Q;
+    if (ix->eps < 0.0) b.eps_mode = -1;
+    else if (ix->eps >= 1.0) b.eps_mode = 1;
+    else { b.eps_mode = 0; b.c_eps = (float)((1.0 - ix->eps) * (1.0 - ix->eps)); }
+    b.final_L = ix->stats; b.n_expand = ix->stats + ix->ws_Q; b.n_scored = ix->stats + 2 * ix->ws_Q;
+    b.flags = ix->stats + 3 * ix->ws_Q;
+    b.spill = ix->spill; b.spill_size = ix->spill_size; b.spill_stride = ix->ws_spill;
+
+    ix->last_Q = Q;
+    ix->last_phases = lp.n_phases;
+    for (int p = 0; p < lp.n_phases; ++p) ix->last_widths[p] = lp.widths[p];
+
+    BOA_CUDA(cudaMemsetAsync(ix->counters, 0, kCntWords * sizeof(uint32_t), st));
+    lp.launches = 0;
+    int extra_launches = 0;
+
+    if (!((double)Q > b.tau_q)) {
+        // Algorithm 1's loop body never runs: every query returns "nothing found"
+        const int64_t n = Q * k > Q ? Q * k : Q;
+        fill_outputs_kernel<<<ix->num_sms * 4, 256, 0, st>>>(out_ids, out_dists, Q * k, b.final_L,
+                                                            b.n_expand, b.n_scored, b.flags, Q);
+        (void)n;
+        BOA_CUDA(cudaGetLastError());
+        ix->last_launches = 1;
+        ix->last_phases = 0;
+        return BOA_OK;
+    }
+
+    const int K = (ix->plus_k >= 2 && lp.n_phases > 1 && ix->tau == 0.0) ? ix->plus_k : 1;
+    uint32_t* cnt = ix->counters + kCntCount;
+    uint32_t* consumed = ix->counters + kCntConsumed;
+    uint32_t* snap = ix->counters + kCntSnap;
+    int n_pools = 0;
+    if (K == 1) {
+        // BOA: one launch per phase, each over the survivors of the one before
+        rc = launch_phase(lp, 0, st, nullptr, nullptr, 0u, (uint32_t)Q, (uint32_t)Q);
+        if (rc != BOA_OK) return rc;
+        for (int p = 1; p < lp.n_phases; ++p) {
+            rc = launch_phase(lp, p, st, nullptr, cnt + p, 0u, 0u, (uint32_t)Q);
+            if (rc != BOA_OK) return rc;
+        }
+    } else {
+        // BOA+: the first phase goes out as K sub-batches on the caller's stream.  After
+        // the sub-batch in the middle and after the last one the survivors gathered so
+        // far are escalated together through all wider phases on the side stream, so
+        // the wide searches of the first pool overlap the remaining narrow sub-batches.
+        const int mid = (K + 1) / 2;
+        for (int j = 0; j < K; ++j) {
+            const uint32_t b0 = (uint32_t)((Q * j) / K), b1 = (uint32_t)((Q * (j + 1)) / K);
+            if (b1 > b0) {
+                rc = launch_phase(lp, 0, st, nullptr, nullptr, b0, b1, b1 - b0);
+                if (rc != BOA_OK) return rc;
+            }
+            if (j + 1 == mid || j + 1 == K) {
+                uint32_t* my_snap = snap + n_pools++;     // one word per pooled escalation
+                copy_word_kernel<<<1, 1, 0, st>>>(my_snap, cnt + 1);
+                extra_launches++;
+                BOA_CUDA(cudaGetLastError());
+                BOA_CUDA(cudaEventRecord(ix->ev_fork, st));
+                BOA_CUDA(cudaStreamWaitEvent(ix->side, ix->ev_fork, 0));
+                for (int p = 1; p < lp.n_phases; ++p) {
+                    const uint32_t* endp = (p == 1) ? my_snap : cnt + p;
+                    rc = launch_phase(lp, p, ix->side, consumed + p, endp, 0u, 0u, (uint32_t)Q);
+                    if (rc != BOA_OK) return rc;
+                    copy_word_kernel<<<1, 1, 0, ix->side>>>(consumed + p, endp);
+                    extra_launches++;
+                    BOA_CUDA(cudaGetLastError());
+                }
+            }
+        }
+        BOA_CUDA(cudaEventRecord(ix->ev_join, ix->side));
+        BOA_CUDA(cudaStreamWaitEvent(st, ix->ev_join, 0));
+    }
+    ix->last_launches = lp.launches + extra_launches;
+    return BOA_OK;
+}
+
+int boa_get_stats(boa_index* ix, int32_t* final_L, int32_t* n_expand, int32_t* n_scored, int32_t* flags,
+                  void* stream)
+{
+    if (!ix) return BOA_EINVAL;
+    if (ix->last_Q == 0) return BOA_OK;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    int32_t* dst[4] = {final_L, n_expand, n_scored, flags};
+    for (int i = 0; i < 4; ++i) {
+        if (!dst[i]) continue;
+        BOA_CUDA(cudaMemcpyAsync(dst[i], ix->stats + (size_t)i * ix->ws_Q,
+                                 (size_t)ix->last_Q * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+    }
+    return BOA_OK;
+}
+
+int boa_get_phase_counts(boa_index* ix, int64_t* active, int n, int* n_phases, void* stream)
+{
+    if (!ix || !active || n < 0) return BOA_EINVAL;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (n_phases) *n_phases = ix->last_phases;
+    if (ix->last_Q == 0 || ix->last_phases == 0) return BOA_OK;
+    uint32_t h[BOA_MAX_PHASES + 1] = {0};
+    BOA_CUDA(cudaMemcpyAsync(h, ix->counters + kCntCount, sizeof(h), cudaMemcpyDeviceToHost, st));
+    BOA_CUDA(cudaStreamSynchronize(st));
+    const double tau_q = ix->tau * (double)ix->last_Q;
+    bool stopped = false;
+    for (int p = 0; p < n && p < ix->last_phases; ++p) {
+        const int64_t a = p == 0 ? ix->last_Q : (int64_t)h[p];
+        if (!((double)a > tau_q)) stopped = true;
+        active[p] = stopped ? 0 : a;
+    }
+    return BOA_OK;
+}
+
+int boa_last_launch_count(const boa_index* ix) { return ix ? ix->last_launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,216 @@
+"""CUDA library against the CPU oracle, element by element, through the C interface."""
+import numpy as np
+import pytest
+import torch
+
+from boa_synth import C1, C2, C3, C4, C5, SENTINEL, clean_rows, exact_knn_graph, make_workload
+from oracle.boa_oracle import OracleIndex, default_widths
+from tests.helpers import assert_bit_parity, gpu_search, make_pair
+
+pytestmark = pytest.mark.gpu
+
+
+def _workload(name):
+    if name == "c1":
+        return C1, make_workload(C1, seed=0)
+    if name == "c2":
+        w = C2.scaled(40_000, 300, name="c2_40k")
+    elif name == "c3":
+        w = C3.scaled(30_000, 200, name="c3_30k")
+    elif name == "c4":
+        w = C4.scaled(50_000, 200, name="c4_50k")
+    elif name == "c5":
+        w = C5.scaled(8_000, 100, name="c5_8k")
+    return w, make_workload(w, seed=1)
+
+
+_cache = {}
+
+
+def _get(name):
+    if name not in _cache:
+        w, d = _workload(name)
+        _cache[name] = (w, d) + make_pair(d)
+    return _cache[name]
+
+
+@pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4", "c5"])
+@pytest.mark.parametrize("mode", ["restart", "resume"])
+def test_boa_matches_oracle_bit_for_bit(name, mode):
+    w, d, orc, gpu, g = _get(name)
+    assert orc.entry == gpu.entry
+    widths = default_widths(w.L0, min(w.Lmax, 256))
+    o = orc.search(d["queries"], d["lo"], d["hi"], w.k, widths, mode=mode, dist_mode=1)
+    r = gpu_search(gpu, g, w.k, widths, mode=mode)
+    assert_bit_parity(o, r, f"{name}/{mode}")
+    assert len(set(o["final_L"].tolist())) > 1 or name == "c1"
+
+
+@pytest.mark.parametrize("name", ["c2", "c4"])
+def test_integer_data_matches_double_accumulation_too(name):
+    """Every partial sum of integer-valued rows is below 2^24, so the fp32 order cannot
+    matter: the GPU must also equal the oracle's double-precision distance mode."""
+    w, d, orc, gpu, g = _get(name)
+    widths = default_widths(w.L0, 128)
+    o = orc.search(d["queries"], d["lo"], d["hi"], w.k, widths, mode="resume", dist_mode=0)
+    r = gpu_search(gpu, g, w.k, widths, mode="resume")
+    assert_bit_parity(o, r, name)
+
+
+@pytest.mark.parametrize("name", ["c3", "c5"])
+def test_float_data_within_tolerance_of_double_accumulation(name):
+    """Against distances summed in double: ids identical except at near-ties (gap below
+    1e-5 relative), distances within 1e-5 relative."""
+    w, d, orc, gpu, g = _get(name)
+    widths = [64]
+    o = orc.search(d["queries"], d["lo"], d["hi"], w.k, widths, dist_mode=0)
+    r = gpu_search(gpu, g, w.k, widths)
+    for i in range(w.Q):
+        oi, ri = o["ids"][i], r["ids"][i]
+        n = int((oi != SENTINEL).sum())
+        assert int((ri != SENTINEL).sum()) == n
+        np.testing.assert_allclose(r["d2"][i][:n], o["d2"][i][:n], rtol=1e-5)
+        for t in np.nonzero(oi[:n] != ri[:n])[0]:
+            near = np.abs(o["d2"][i][:n] - o["d2"][i][t]) <= 1e-5 * o["d2"][i][t]
+            assert near.sum() > 1 or ri[t] in oi[:n], (i, t)
+
+
+@pytest.mark.parametrize("name", ["c2", "c3"])
+@pytest.mark.parametrize("plus_k", [2, 5, 10])
+def test_boa_plus_equals_boa(name, plus_k):
+    w, d, orc, gpu, g = _get(name)
+    widths = default_widths(w.L0, 256)
+    for mode in ("restart", "resume"):
+        a = gpu_search(gpu, g, w.k, widths, mode=mode, plus_k=0)
+        b = gpu_search(gpu, g, w.k, widths, mode=mode, plus_k=plus_k)
+        assert (a["ids"] == b["ids"]).all() and (a["d2"].view(np.uint32) == b["d2"].view(np.uint32)).all()
+        assert (a["final_L"] == b["final_L"]).all() and (a["n_expand"] == b["n_expand"]).all()
+        assert (a["phase_active"] == b["phase_active"]).all()
+
+
+def test_fixed_width_500_not_a_power_of_two():
+    w, d, orc, gpu, g = _get("c2")
+    o = orc.search(d["queries"][:80], d["lo"][:80], d["hi"][:80], w.k, [500], dist_mode=1)
+    r = gpu_search(gpu, g, w.k, [500], sel=slice(0, 80))
+    assert_bit_parity(o, r, "fixed500")
+
+
+def test_eps_and_tau_special_cases():
+    w, d, orc, gpu, g = _get("c2")
+    widths = default_widths(16, 128)
+    for eps in (-1.0, 1.0, 0.0, 0.3):
+        o = orc.search(d["queries"], d["lo"], d["hi"], w.k, widths, eps=eps, dist_mode=1)
+        r = gpu_search(gpu, g, w.k, widths, eps=eps)
+        assert_bit_parity(o, r, f"eps={eps}")
+    o0 = orc.search(d["queries"], d["lo"], d["hi"], w.k, widths, dist_mode=1)
+    for tau in ((o0["phase_active"][1] + 0.5) / w.Q, (o0["phase_active"][1] - 0.5) / w.Q, 1.0, 2.0):
+        o = orc.search(d["queries"], d["lo"], d["hi"], w.k, widths, tau=tau, dist_mode=1)
+        r = gpu_search(gpu, g, w.k, widths, tau=tau)
+        assert_bit_parity(o, r, f"tau={tau}")
+
+
+def test_expansion_cap():
+    w, d, orc, gpu, g = _get("c2")
+    o = orc.search(d["queries"], d["lo"], d["hi"], w.k, [16, 64], cap=(1, 3), dist_mode=1)
+    r = gpu_search(gpu, g, w.k, [16, 64], cap=(1, 3))
+    assert (o["flags"] & 1).any()
+    assert_bit_parity(o, r, "cap")
+
+
+def test_ring_hand_trace_on_gpu():
+    x = np.zeros((8, 4), dtype=np.float32)
+    x[:, 0] = np.arange(8)
+    d = dict(vectors=x, attrs=(np.arange(8) % 2).astype(np.int32)[:, None],
+             attr_types=np.zeros(1, np.int32),
+             graph=np.stack([(np.arange(8) - 1) % 8, (np.arange(8) + 1) % 8], 1).astype(np.uint32),
+             queries=np.array([[5.2, 0, 0, 0]], dtype=np.float32),
+             lo=np.array([[1]], np.int32), hi=np.array([[1]], np.int32))
+    orc, gpu, g = make_pair(d, entry=0)
+    r = gpu_search(gpu, g, 2, [3])
+    assert r["ids"][0].tolist() == [5, 7]
+    np.testing.assert_allclose(r["d2"][0], [0.04, 3.24], rtol=1e-5)
+    assert r["n_expand"][0] == 5 and r["n_scored"][0] == 6
+
+
+def test_full_width_search_equals_bruteforce_on_gpu():
+    rng = np.random.default_rng(7)
+    N, D, R, k = 300, 8, 6, 10
+    x = rng.integers(0, 32, size=(N, D)).astype(np.float32)
+    g5 = exact_knn_graph(x, R - 1, device="cpu")
+    ring = ((np.arange(N) + 1) % N).astype(np.uint32)[:, None]
+    d = dict(vectors=x, attrs=rng.integers(0, 100, size=(N, 2)).astype(np.int32),
+             attr_types=np.zeros(2, np.int32), graph=clean_rows(np.concatenate([g5, ring], 1)),
+             queries=rng.integers(0, 32, size=(25, D)).astype(np.float32))
+    d["lo"] = rng.integers(0, 50, size=(25, 2)).astype(np.int32)
+    d["hi"] = (d["lo"] + rng.integers(20, 60, size=(25, 2))).astype(np.int32)
+    orc, gpu, g = make_pair(d)
+    gt_ids, gt_d2, nvalid = orc.bruteforce(d["queries"], d["lo"], d["hi"], k)
+    r = gpu_search(gpu, g, k, [N], cap=(8, 64))
+    assert (r["ids"] == gt_ids).all()
+    assert (r["n_expand"] == N).all()
+    fin = gt_ids != SENTINEL
+    assert (r["d2"][fin].astype(np.float64) == gt_d2[fin]).all()
+
+
+def test_dirty_graph_rows_empty_ranges_and_short_answers():
+    w = C2.scaled(5000, 64, name="c2_dirty")
+    d = make_workload(w, seed=9)
+    rng = np.random.default_rng(0)
+    gph = d["graph"].copy()
+    rows = rng.integers(0, w.N, size=800)
+    gph[rows, 3] = rows.astype(np.uint32)                   # self references
+    gph[rows, 7] = gph[rows, 1]                             # repeats
+    gph[rng.integers(0, w.N, size=500), rng.integers(0, w.R, size=500)] = SENTINEL
+    d["graph"] = gph
+    d["lo"][0], d["hi"][0] = d["hi"][0].copy(), d["lo"][0].copy() - 1      # lo > hi: empty
+    d["hi"][1] = d["lo"][1]                                  # very few valid points
+    d["lo"][2] = np.iinfo(np.int32).min
+    d["hi"][2] = np.iinfo(np.int32).max                      # unconstrained
+    orc, gpu, g = make_pair(d)
+    widths = [16, 64, 128]
+    for mode in ("restart", "resume"):
+        o = orc.search(d["queries"], d["lo"], d["hi"], w.k, widths, mode=mode, dist_mode=1)
+        r = gpu_search(gpu, g, w.k, widths, mode=mode)
+        assert_bit_parity(o, r, f"dirty/{mode}")
+    assert (r["ids"][0] == SENTINEL).all() and np.isinf(r["d2"][0]).all()
+    assert r["final_L"][0] == 128
+
+
+def test_k_equals_L0_and_k_one():
+    w, d, orc, gpu, g = _get("c2")
+    for k, widths in ((16, [16, 64]), (1, [16, 64])):
+        o = orc.search(d["queries"], d["lo"], d["hi"], k, widths, dist_mode=1)
+        r = gpu_search(gpu, g, k, widths)
+        assert_bit_parity(o, r, f"k={k}")
+
+
+def test_empty_batch_and_argument_errors():
+    from paper_2609_16175_b200 import BoaError
+    w, d, orc, gpu, g = _get("c2")
+    gpu.set_schedule([])
+    q0 = g["queries"][:0]
+    ids, d2 = gpu.search(q0, g["lo"][:0], g["hi"][:0], 10, 16, 64)
+    assert ids.shape == (0, 10)
+    for k, L0, Lmax in ((0, 16, 64), (17, 16, 64), (10, 64, 16), (10, 16, 4096)):
+        with pytest.raises(BoaError):
+            gpu.search(g["queries"], g["lo"], g["hi"], k, L0, Lmax)
+    bad = g["graph"].clone()
+    bad[5, 2] = w.N + 3
+    from paper_2609_16175_b200 import BoaIndex
+    with pytest.raises(BoaError) as e:
+        BoaIndex(g["vectors"], g["attrs"], d["attr_types"].tolist(), bad)
+    assert e.value.status == -4
+
+
+def test_explicit_entry_and_growth_schedule():
+    w, d, _, _, _ = _get("c2")
+    orc, gpu, g = make_pair(d, entry=123)
+    assert gpu.entry == 123
+    gpu.set_schedule([])
+    gpu.set_param("growth", 4)
+    gpu.set_param("mode", 0)
+    ids, d2 = gpu.search(g["queries"], g["lo"], g["hi"], 10, 16, 100)     # 16, 64, 100
+    torch.cuda.synchronize()
+    o = orc.search(d["queries"], d["lo"], d["hi"], 10, [16, 64, 100], dist_mode=1)
+    assert (ids.cpu().numpy().view(np.uint32) == o["ids"]).all()
+    assert gpu.phase_counts() == o["phase_active"].tolist()
