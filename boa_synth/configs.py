@@ -35,15 +35,19 @@ class Workload:
     L0: int
     Lmax: int
     # generator knobs (latent geometry; see generate.py)
-    dz: int = 12           # latent dimension of the cluster mixture
+    dz: int = 6            # latent dimension of the cluster mixture
     spread: float = 1.0    # std of cluster centres in latent space
-    sigma_l: float = 0.35  # within-cluster std in latent space
+    sigma_l: float = 0.6   # within-cluster std in latent space (clusters overlap)
     sigma_n: float = 0.04  # isotropic ambient noise, relative to the latent scale
     # graph knobs for graph == "mixed"
     r_long: int = 6        # multi-scale long edges per node
-    r_attr: int = 0        # attribute-cell neighbours per node
-    attr_frac: float = 0.02  # fraction of the data one attribute cell holds
-    t_near: int = 8        # neighbouring clusters searched for kNN candidates
+    long_attr_aware: bool = True  # long edges land on attribute-near points of the far cell
+    r_rev: int = 4         # reverse copies of nearest-neighbour edges per node
+    r_attr: int = 16       # attribute-window neighbours per node
+    attr_fracs: Tuple[float, ...] = (0.1, 0.01)  # fraction of the data inside one attribute window
+    t_near: int = 16       # neighbouring cells searched for kNN candidates
+    k_cand: int = 64       # nearest candidates the occlusion pruning starts from
+    prune_alpha: float = 1.2  # occlusion factor (0 = plain nearest neighbours)
 
     def scaled(self, N: int, Q: int | None = None, name: str | None = None) -> "Workload":
         """Same recipe at another size; points per cluster kept where possible."""
@@ -74,7 +78,7 @@ C3 = Workload(name="c3_unit96", N=1_000_000, D=96, vec_dtype="f32", vec_kind="un
 C4 = Workload(name="c4_u8_10m", N=10_000_000, D=128, vec_dtype="u8", vec_kind="int_latent",
               n_clusters=4096, attrs=("uniform_int", "uniform_int"), R=64, graph="mixed",
               Q=10_000, sel_kind="loguniform", sel_lo=0.005, sel_hi=0.50, k=10, L0=32, Lmax=512,
-              r_long=8)
+              r_long=8, r_attr=32, r_rev=8)
 
 C5 = Workload(name="c5_f960", N=1_000_000, D=960, vec_dtype="f32", vec_kind="float_latent",
               n_clusters=512, attrs=("uniform_int", "uniform_float", "zipf_cat", "zipf_cat"),

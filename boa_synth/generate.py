@@ -181,88 +181,185 @@ def exact_knn_graph(vectors: np.ndarray, R: int, device: str | None = None) -> n
     return out
 
 
-def _attr_cells(attrs: np.ndarray, types: np.ndarray, frac: float) -> np.ndarray:
-    """Cell id of every point on a rank-quantile grid holding ~frac of the data per cell."""
+def _rank_columns(attrs: np.ndarray, types: np.ndarray) -> np.ndarray:
+    """Rank of every point in every attribute column, scaled to [0, 1)."""
     n, m = attrs.shape
-    g = max(1, int(round(frac ** (-1.0 / m))))
-    cell = np.zeros(n, dtype=np.int64)
+    out = np.empty((n, m), dtype=np.float32)
     for j in range(m):
         vals = _column_values(attrs[:, j], types[j])
         order = np.argsort(vals, kind="stable")
         rank = np.empty(n, dtype=np.int64)
         rank[order] = np.arange(n)
-        cell = cell * g + np.minimum(rank * g // n, g - 1)
-    return cell
+        out[:, j] = rank / float(n)
+    return out
+
+
+def _zorder(ranks01: np.ndarray, bits: int = 7) -> np.ndarray:
+    """Morton code of the attribute rank vector (bits per attribute, interleaved)."""
+    n, m = ranks01.shape
+    q = np.minimum((ranks01 * (1 << bits)).astype(np.int64), (1 << bits) - 1)
+    code = np.zeros(n, dtype=np.int64)
+    for b in range(bits - 1, -1, -1):
+        for j in range(m):
+            code = (code << 1) | ((q[:, j] >> b) & 1)
+    return code
+
+
+def _diversify(x: torch.Tensor, y_all: torch.Tensor, cand_idx: torch.Tensor, cand_d: torch.Tensor,
+               keep: int, alpha: float) -> torch.Tensor:
+    """Occlusion pruning of sorted candidate lists: walking a list from near to far, a
+    candidate survives unless an already kept one is alpha times closer to it than the
+    node itself is.  Returns, per node, candidate slots reordered so that survivors come
+    first (in distance order) followed by the pruned ones (in distance order)."""
+    B, K = cand_idx.shape
+    yc = y_all[cand_idx]                                   # B x K x D
+    yn = (yc * yc).sum(-1)
+    pd = yn[:, :, None] + yn[:, None, :] - 2.0 * torch.bmm(yc, yc.transpose(1, 2))
+    alive = torch.ones((B, K), dtype=torch.bool, device=x.device)
+    chosen = torch.zeros((B, K), dtype=torch.bool, device=x.device)
+    count = torch.zeros(B, dtype=torch.int64, device=x.device)
+    for t in range(K):
+        take = alive[:, t] & (count < keep)
+        chosen[:, t] = take
+        count += take.to(torch.int64)
+        occl = (alpha * pd[:, t, :] <= cand_d) & take[:, None]
+        occl[:, :t + 1] = False
+        alive &= ~occl
+    # stable partition: chosen first
+    key = (~chosen).to(torch.int64) * K + torch.arange(K, device=x.device)[None, :]
+    return torch.argsort(key, dim=1)
+
+
+def _cells(vectors: np.ndarray, cl: np.ndarray, nc: int, dev: torch.device):
+    """Voronoi cells of the label means in data space: returns (cell of every point,
+    cell means).  A point sits in the cell of its nearest mean, whatever its label."""
+    x = torch.from_numpy(np.ascontiguousarray(vectors)).to(dev)
+    means = torch.zeros((nc, vectors.shape[1]), dtype=torch.float64, device=dev)
+    lab = torch.from_numpy(cl.astype(np.int64)).to(dev)
+    cnt = torch.bincount(lab, minlength=nc).clamp_(min=1).to(torch.float64)
+    step = 1 << 18
+    for s in range(0, x.shape[0], step):
+        means.index_add_(0, lab[s:s + step], x[s:s + step].to(torch.float64))
+    means = (means / cnt[:, None]).to(torch.float32)
+    mn = (means * means).sum(1)
+    cell = torch.empty(x.shape[0], dtype=torch.int64, device=dev)
+    for s in range(0, x.shape[0], step):
+        xb = x[s:s + step].to(torch.float32)
+        cell[s:s + step] = _sq_dists(xb, (xb * xb).sum(1), means, mn).argmin(1)
+    return cell.cpu().numpy(), means.cpu().numpy()
 
 
 def mixed_graph(w: Workload, vectors: np.ndarray, attrs: np.ndarray, types: np.ndarray,
                 cl: np.ndarray, centres: np.ndarray, ss_graph, device: str | None = None) -> np.ndarray:
-    """Degree-R fixture: approximate kNN (exact among the points of the t_near
-    nearest clusters), optional attribute-cell neighbours, and multi-scale long
-    edges to random points of clusters at log-uniformly drawn centre ranks."""
+    """Degree-R fixture built from four kinds of edges:
+      * r_knn  approximate nearest neighbours (exact among the points of the t_near nearest
+               cells), thinned by occlusion pruning so that they spread in direction;
+      * r_rev  reverse copies of those edges, so that no node is left without a way in;
+      * r_attr nearest neighbours among the points whose attribute ranks all lie within a
+               window around the node's own, at one or more window sizes -- the role the
+               threshold passes of the paper's graph construction play;
+      * r_long long edges to random points of cells at log-uniformly drawn centre ranks."""
     dev = _prep_device(device)
     rng = np.random.default_rng(ss_graph)
     n, R, nc = w.N, w.R, w.n_clusters
     r_long = min(w.r_long, R - 1)
     r_attr = min(w.r_attr, R - r_long - 1)
-    r_knn = R - r_long - r_attr
-    order = np.argsort(cl, kind="stable")
-    starts = np.searchsorted(cl[order], np.arange(nc + 1))
-    cdist = ((centres[:, None, :] - centres[None, :, :]) ** 2).sum(-1) if nc <= 4096 else None
-    if cdist is None:
-        raise ValueError("too many clusters")
+    r_rev = min(w.r_rev, R - r_long - r_attr - 1)
+    r_knn = R - r_long - r_attr - r_rev
+    cell, means = _cells(vectors, cl, nc, dev)
+    order = np.argsort(cell, kind="stable")
+    starts = np.searchsorted(cell[order], np.arange(nc + 1))
+    cdist = ((means[:, None, :].astype(np.float64) - means[None, :, :]) ** 2).sum(-1)
     crank = np.argsort(cdist, axis=1, kind="stable")        # crank[c][0] == c
     t_near = min(w.t_near, nc)
-    cells = _attr_cells(attrs, types, w.attr_frac) if r_attr > 0 else None
+    fracs = [f for f in w.attr_fracs if f > 0] if r_attr > 0 else []
+    ranks = torch.from_numpy(_rank_columns(attrs, types)[order]).to(dev) if fracs else None
 
     graph = np.full((n, R), SENTINEL, dtype=np.uint32)
-    xs = torch.from_numpy(np.ascontiguousarray(vectors[order].astype(np.float32)))
+    xs = torch.from_numpy(np.ascontiguousarray(vectors[order].astype(np.float32))).to(dev)
+    order_t = torch.from_numpy(order).to(dev)
     big = 3.0e38
+    k_cand = max(r_knn, min(w.k_cand, 8 * r_knn))
+    blk = 2048
     for c in range(nc):
-        a, b = starts[c], starts[c + 1]
+        a, b = int(starts[c]), int(starts[c + 1])
         if a == b:
             continue
-        cand_parts = [np.arange(starts[t], starts[t + 1]) for t in crank[c, :t_near]]
-        cand = np.concatenate(cand_parts)
-        x = xs[a:b].to(dev)
-        y = xs[torch.from_numpy(cand)].to(dev)
-        d = _sq_dists(x, (x * x).sum(1), y, (y * y).sum(1))
-        # candidates begin with this cluster's own rows, so self sits on the diagonal
-        d[torch.arange(b - a, device=dev), torch.arange(b - a, device=dev)] = big
-        kk = min(r_knn + r_attr, cand.shape[0] - 1)
-        near = torch.topk(d, kk, dim=1, largest=False, sorted=True)
-        near_idx = near.indices.cpu().numpy()
-        rows = order[a:b]
-        take = min(r_knn, kk)
-        graph[rows, :take] = order[cand[near_idx[:, :take]]].astype(np.uint32)
-        if r_attr > 0:
-            cx = torch.from_numpy(cells[order[a:b]]).to(dev)
-            cy = torch.from_numpy(cells[order[cand]]).to(dev)
-            d.scatter_(1, near.indices[:, :take], big)
-            d.masked_fill_(cx[:, None] != cy[None, :], big)
-            ka = min(r_attr, cand.shape[0] - 1)
-            an = torch.topk(d, ka, dim=1, largest=False, sorted=True)
-            a_idx = an.indices.cpu().numpy()
-            a_ok = (an.values < 1.0e38).cpu().numpy()
-            picked = order[cand[a_idx]].astype(np.uint32)
-            # where the cell ran out of points fall back to the next plain neighbours
-            spare = order[cand[near_idx[:, take:take + ka]]].astype(np.uint32) if kk > take else None
-            for t in range(ka):
-                col = picked[:, t].copy()
-                if spare is not None and t < spare.shape[1]:
-                    col = np.where(a_ok[:, t], col, spare[:, t])
-                else:
-                    col = np.where(a_ok[:, t], col, SENTINEL)
-                graph[rows, r_knn + t] = col
-    # long edges: cluster rank drawn log-uniformly in [1, nc), random point inside it
+        cand = torch.from_numpy(np.concatenate(
+            [np.arange(starts[t], starts[t + 1]) for t in crank[c, :t_near]])).to(dev)
+        y = xs[cand]
+        yn = (y * y).sum(1)
+        for s0 in range(a, b, blk):
+            s1 = min(b, s0 + blk)
+            x = xs[s0:s1]
+            d = _sq_dists(x, (x * x).sum(1), y, yn)
+            # candidates begin with this cell's own rows: self is at column (row - a)
+            rows_local = torch.arange(s0 - a, s1 - a, device=dev)
+            d[torch.arange(s1 - s0, device=dev), rows_local] = big
+            kk = min(k_cand, cand.shape[0] - 1)
+            near = torch.topk(d, kk, dim=1, largest=False, sorted=True)
+            if w.prune_alpha > 0 and kk > r_knn:
+                perm = _diversify(x, y, near.indices, near.values, r_knn, w.prune_alpha)
+                sel = torch.gather(near.indices, 1, perm[:, :r_knn])
+            else:
+                sel = near.indices[:, :r_knn]
+            take = sel.shape[1]
+            out_rows = order[s0:s1]
+            graph[out_rows, :take] = order_t[cand[sel]].cpu().numpy().astype(np.uint32)
+            if fracs:
+                d.scatter_(1, sel, big)
+                per = r_attr // len(fracs)
+                col0 = r_knn + r_rev
+                for fi, f in enumerate(fracs):
+                    cnt = per if fi + 1 < len(fracs) else r_attr - per * (len(fracs) - 1)
+                    half = 0.5 * f ** (1.0 / w.m)
+                    dm = d.clone()
+                    for j in range(w.m):
+                        diff = (ranks[s0:s1, j][:, None] - ranks[cand, j][None, :]).abs_()
+                        dm.masked_fill_(diff > half, big)
+                    an = torch.topk(dm, cnt, dim=1, largest=False, sorted=True)
+                    picked = order_t[cand[an.indices]]
+                    picked = torch.where(an.values < 1.0e38, picked, torch.full_like(picked, -1))
+                    pk = picked.cpu().numpy()
+                    graph[out_rows, col0:col0 + cnt] = np.where(pk >= 0, pk, 0xFFFFFFFF).astype(np.uint32)
+                    d.scatter_(1, an.indices, big)
+                    col0 += cnt
+    # reverse edges: v gets up to r_rev of the nodes that point at it, in a seeded random order
+    if r_rev > 0:
+        src = np.repeat(np.arange(n, dtype=np.int64), r_knn)
+        dst = graph[:, :r_knn].reshape(-1).astype(np.int64)
+        ok = dst != int(SENTINEL)
+        src, dst = src[ok], dst[ok]
+        shuffle = rng.permutation(src.shape[0])
+        src, dst = src[shuffle], dst[shuffle]
+        o = np.argsort(dst, kind="stable")
+        src, dst = src[o], dst[o]
+        first = np.searchsorted(dst, np.arange(n))
+        pos = np.arange(dst.shape[0]) - first[dst]
+        keep = pos < r_rev
+        graph[dst[keep], r_knn + pos[keep]] = src[keep].astype(np.uint32)
+    # long edges: cell rank drawn log-uniformly in [1, nc); inside that cell the point whose
+    # attributes are nearest to the node's own along a Z-order curve over the attribute
+    # ranks (plus a small random offset), so that long hops tend to stay inside a range
     if r_long > 0 and nc > 1:
         u = rng.random((n, r_long))
         rank = np.minimum(np.floor(np.exp(u * math.log(nc))).astype(np.int64), nc - 1)
         rank = np.maximum(rank, 1)
-        tgt_cluster = crank[cl[:, None], rank]
-        size = (starts[1:] - starts[:-1])[tgt_cluster]
-        off = np.minimum((rng.random((n, r_long)) * size).astype(np.int64), np.maximum(size - 1, 0))
-        tgt = order[np.minimum(starts[tgt_cluster] + off, n - 1)].astype(np.uint32)
+        tgt_cell = crank[cell[:, None], rank]
+        size = (starts[1:] - starts[:-1])[tgt_cell]
+        if w.long_attr_aware:
+            zc = _zorder(_rank_columns(attrs, types))
+            key = cell.astype(np.int64) * (1 << 32) + zc
+            korder = np.argsort(key, kind="stable")         # grouped by cell, Z-ordered inside
+            ksorted = key[korder]
+            want = tgt_cell.astype(np.int64) * (1 << 32) + zc[:, None]
+            pos = np.searchsorted(ksorted, want.reshape(-1)).reshape(n, r_long)
+            pos = pos + rng.integers(-2, 3, size=(n, r_long))
+            pos = np.clip(pos, starts[tgt_cell], np.maximum(starts[tgt_cell + 1] - 1, starts[tgt_cell]))
+            tgt = korder[np.minimum(pos, n - 1)].astype(np.uint32)
+        else:
+            off = np.minimum((rng.random((n, r_long)) * size).astype(np.int64), np.maximum(size - 1, 0))
+            tgt = order[np.minimum(starts[tgt_cell] + off, n - 1)].astype(np.uint32)
         tgt = np.where(size > 0, tgt, SENTINEL)
         graph[:, R - r_long:] = tgt
     return clean_rows(graph)
