@@ -52,6 +52,8 @@ def parse_args():
     ap.add_argument("--schedule", default="16,512")
     ap.add_argument("--plus-k", type=int, default=0)
     ap.add_argument("--hash-log2", type=int, default=0)
+    ap.add_argument("--stage-rows", type=int, default=0)
+    ap.add_argument("--no-extras", action="store_true", help="debug: skip recall/e2e/cpu legs")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--seed", type=int, default=0)
     return ap.parse_args()
@@ -257,6 +259,7 @@ def main():
     ix.set_param("eps", args.eps)
     ix.set_param("plus_k", args.plus_k)
     ix.set_param("hash_log2", args.hash_log2)
+    ix.set_param("stage_rows", args.stage_rows)
     ix.set_schedule(widths)
     Q, k = w.Q, w.k
     out_ids = torch.empty((Q, k), dtype=torch.int32, device=dev)
@@ -301,6 +304,14 @@ def main():
     phase_counts = ix.phase_counts()
     ids_np = out_ids.cpu().numpy().view(np.uint32)
     d2_np = out_d2.cpu().numpy()
+
+    if args.no_extras:
+        if rank == 0:
+            print(json.dumps({"ms_per_step": ms_per_step, "value": value, "hash_log2": args.hash_log2,
+                              "stage_rows": args.stage_rows, "schedule": widths, "mode": args.mode,
+                              "plus_k": args.plus_k, "mean_scored": float(st["n_scored"].mean()),
+                              "status": ix.device_status()}))
+        return
 
     # ---- end to end through the public call: pinned host inputs in, results out, every step
     hq = torch.from_numpy(d["queries"]).pin_memory()

@@ -51,8 +51,10 @@ enum {
                                Multiple Batches")                                            */
     BOA_PARAM_CAP_MULT = 5, /* a phase at width L gives up after CAP_MULT*L + CAP_ADD        */
     BOA_PARAM_CAP_ADD = 6,  /*   expansions; defaults 8 and 64                               */
-    BOA_PARAM_HASH_LOG2 = 7 /* 0 = choose per phase; else log2 of the per-query table of
-                               recently scored ids (10..14).  Never changes results.         */
+    BOA_PARAM_HASH_LOG2 = 7, /* 0 = choose per phase; else log2 of the per-query table of
+                               recently scored ids (8..14).  Never changes results.          */
+    BOA_PARAM_STAGE_ROWS = 8 /* 0 = choose; else neighbour records one query keeps in flight
+                               in shared memory (2..64).  Never changes results.             */
 };
 
 /*
@@ -137,6 +139,11 @@ int boa_workspace_bytes(const boa_index* index, int64_t Q, int Lmax, size_t* byt
 
 /* Number of kernel launches the last boa_search enqueued. */
 int boa_last_launch_count(const boa_index* index);
+
+/* Device-side status of the last search on this index (HOST int, synchronises
+   `stream`): 0 = fine; bit 0 = an asynchronous copy did not complete within its bounded
+   wait, the affected launches stopped early and their outputs are incomplete. */
+int boa_device_status(boa_index* index, int* status, void* stream);
 
 /* cudaError_t of the most recent failing CUDA call made by this library (0 if none). */
 int boa_last_cuda_error(void);

@@ -15,7 +15,8 @@ import torch
 HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = None
 
-PARAM = dict(eps=0, growth=1, tau=2, mode=3, plus_k=4, cap_mult=5, cap_add=6, hash_log2=7)
+PARAM = dict(eps=0, growth=1, tau=2, mode=3, plus_k=4, cap_mult=5, cap_add=6, hash_log2=7,
+             stage_rows=8)
 F32, U8 = 0, 1
 NO_ID = 0xFFFFFFFF
 
@@ -66,6 +67,8 @@ def load_library():
     L.boa_workspace_bytes.argtypes = [vp, i64, i32, C.POINTER(C.c_size_t)]
     L.boa_last_launch_count.restype = i32
     L.boa_last_launch_count.argtypes = [vp]
+    L.boa_device_status.restype = i32
+    L.boa_device_status.argtypes = [vp, C.POINTER(i32), vp]
     L.boa_last_cuda_error.restype = i32
     L.boa_strerror.restype = C.c_char_p
     L.boa_strerror.argtypes = [i32]
@@ -178,6 +181,11 @@ class BoaIndex:
         b = C.c_size_t(0)
         _check(self._lib.boa_workspace_bytes(self._h, Q, Lmax, C.byref(b)), "boa_workspace_bytes")
         return int(b.value)
+
+    def device_status(self, stream: Optional[torch.cuda.Stream] = None) -> int:
+        v = C.c_int(0)
+        _check(self._lib.boa_device_status(self._h, C.byref(v), _stream_ptr(stream)), "boa_device_status")
+        return int(v.value)
 
     @property
     def last_launch_count(self) -> int:

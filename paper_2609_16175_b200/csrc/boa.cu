@@ -151,7 +151,7 @@ __global__ void copy_word_kernel(uint32_t* dst, const uint32_t* src) { *dst = *s
 struct boa_index {
     int64_t N = 0;
     int D = 0, m = 0, R = 0, vec_dtype = 0;
-    int rec_stride = 0, nchunks = 0, attr_off = 0;
+    int rec_stride = 0, rec_bytes = 0, nchunks = 0, attr_off = 0;
     uint32_t attr_float_mask = 0;
     int64_t entry = 0;
     uint8_t* rec = nullptr;
@@ -159,7 +159,7 @@ struct boa_index {
     int device = 0, num_sms = 0;
     // parameters
     double eps = 0.05, growth = 4.0, tau = 0.0;
-    int mode = 0, plus_k = 0, cap_mult = 8, cap_add = 64, hash_log2 = 0;
+    int mode = 0, plus_k = 0, cap_mult = 8, cap_add = 64, hash_log2 = 0, stage_rows = 0;
     int n_sched = 0;
     int sched[BOA_MAX_PHASES] = {0};
     // scratch
@@ -184,6 +184,7 @@ namespace {
 constexpr int kCntCount = 0;                          // [P+1] survivors entering phase p (p>=1)
 constexpr int kCntConsumed = 16;                      // [P+1] list positions already searched
 constexpr int kCntSnap = 32;                          // [pool] frozen end of phase 1's list
+constexpr int kCntStatus = 47;                        // device status bits
 constexpr int kCntTicket = 48;                        // one per launch
 constexpr int kMaxLaunches = 128;
 constexpr int kCntWords = kCntTicket + kMaxLaunches;
@@ -195,39 +196,30 @@ struct KernelChoice {
     int rs;
 };
 
-template <int VT, int CPL, int U>
-KernelChoice pick_rs(int R)
-{
-    if (R <= 32) return {boa::boa_search_kernel<VT, CPL, 1, U>, 1};
-    return {boa::boa_search_kernel<VT, CPL, 2, U>, 2};
-}
-
 KernelChoice pick_kernel(const boa_index* ix)
 {
-    const int cpl = (ix->nchunks + 7) / 8;
     if (ix->vec_dtype == BOA_F32) {
-        switch (cpl) {
-            case 1: return pick_rs<0, 1, 8>(ix->R);
-            case 2: return pick_rs<0, 2, 4>(ix->R);
-            case 3: return pick_rs<0, 3, 2>(ix->R);
-            case 4: return pick_rs<0, 4, 2>(ix->R);
-            default: return pick_rs<0, 0, 1>(ix->R);
-        }
+        if (ix->R <= 32) return {boa::boa_search_kernel<0, 1>, 1};
+        return {boa::boa_search_kernel<0, 2>, 2};
     }
-    switch (cpl) {
-        case 1: return pick_rs<1, 1, 8>(ix->R);
-        case 2: return pick_rs<1, 2, 4>(ix->R);
-        default: return pick_rs<1, 0, 1>(ix->R);
-    }
+    if (ix->R <= 32) return {boa::boa_search_kernel<1, 1>, 1};
+    return {boa::boa_search_kernel<1, 2>, 2};
 }
 
 int choose_hash_log2(const boa_index* ix, int L)
 {
     if (ix->hash_log2) return ix->hash_log2;
-    int want = 16 * L;              // about the ids one search at width L scores
-    int lg = 10;
-    while ((1 << lg) < want && lg < 13) ++lg;
-    return lg;
+    if (L <= 32) return 10;
+    if (L <= 128) return 11;
+    return 12;
+}
+
+int choose_stage_rows(const boa_index* ix, int rs)
+{
+    int rows = ix->stage_rows ? ix->stage_rows : 8192 / ix->rec_bytes;
+    if (rows < 2) rows = 2;
+    if (rows > 32 * rs) rows = 32 * rs;
+    return rows;
 }
 
 int phase_widths(const boa_index* ix, int L0, int Lmax, int* w)
@@ -292,6 +284,7 @@ int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_p
     sp.L = L;
     sp.C = ix->mode == 1 ? Lmax : L;
     sp.hash_log2 = choose_hash_log2(ix, L);
+    sp.stage_rows = choose_stage_rows(ix, lp.kc.rs);
     sp.max_expand = ix->cap_mult * L + ix->cap_add;
     sp.first_phase = p == 0;
     sp.resume_in = (ix->mode == 1 && p > 0);
@@ -307,8 +300,9 @@ int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_p
     sp.out_list = ix->lists + (size_t)(p + 1 < BOA_MAX_PHASES ? p + 1 : p) * ix->ws_Q;
     sp.out_count = ix->counters + kCntCount + p + 1;
 
-    const boa::WarpSmem lay = boa::warp_smem_layout(sp.C, sp.hash_log2, ix->D, lp.kc.rs);
-    const size_t smem = (size_t)lay.total * boa::kWarpsPerCta;
+    const boa::WarpSmem lay = boa::warp_smem_layout(sp.C, sp.hash_log2, ix->D, lp.kc.rs, sp.stage_rows,
+                                                    ix->rec_bytes);
+    const size_t smem = (size_t)lay.total;
     if (smem > 48 * 1024) {
         BOA_CUDA(cudaFuncSetAttribute((const void*)lp.kc.fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)smem));
@@ -318,7 +312,7 @@ int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_p
                                                            boa::kThreads, smem));
     if (per_sm < 1) return BOA_EINVAL;
     int64_t grid = (int64_t)per_sm * ix->num_sms;
-    const int64_t need = ((int64_t)expected_items + boa::kWarpsPerCta - 1) / boa::kWarpsPerCta;
+    const int64_t need = (int64_t)expected_items;
     if (need < grid) grid = need < 1 ? 1 : need;
     lp.kc.fn<<<(unsigned)grid, boa::kThreads, smem, st>>>(sp);
     BOA_CUDA(cudaGetLastError());
@@ -381,6 +375,7 @@ int boa_index_create(boa_index** out, const void* vectors, int vec_dtype, int64_
     ix->nchunks = vec_bytes / 16;
     ix->attr_off = vec_bytes;
     ix->rec_stride = (vec_bytes + 4 * m + 31) & ~31;
+    ix->rec_bytes = (vec_bytes + 4 * m + 15) & ~15;
     for (int j = 0; j < m; ++j)
         if (attr_types[j] == BOA_ATTR_F32) ix->attr_float_mask |= 1u << j;
     BOA_TRY(cudaGetDevice(&ix->device));
@@ -487,8 +482,11 @@ int boa_set_param(boa_index* ix, int key, double v)
             if (v < 0.0 || v > 1e6 || v != floor(v)) return BOA_EINVAL;
             ix->cap_add = (int)v; return BOA_OK;
         case BOA_PARAM_HASH_LOG2:
-            if (v != 0.0 && (v < 10.0 || v > 14.0 || v != floor(v))) return BOA_EINVAL;
+            if (v != 0.0 && (v < 8.0 || v > 14.0 || v != floor(v))) return BOA_EINVAL;
             ix->hash_log2 = (int)v; return BOA_OK;
+        case BOA_PARAM_STAGE_ROWS:
+            if (v < 0.0 || v > 64.0 || v != floor(v)) return BOA_EINVAL;
+            ix->stage_rows = (int)v; return BOA_OK;
         default: return BOA_EINVAL;
     }
 }
@@ -540,7 +538,8 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
     boa::SearchParams& b = lp.base;
     memset(&b, 0, sizeof(b));
     b.rec = ix->rec; b.graph = ix->graph; b.N = ix->N; b.D = ix->D; b.m = ix->m; b.R = ix->R;
-    b.rec_stride = ix->rec_stride; b.nchunks = ix->nchunks; b.attr_off = ix->attr_off;
+    b.rec_stride = ix->rec_stride; b.rec_bytes = ix->rec_bytes; b.nchunks = ix->nchunks;
+    b.attr_off = ix->attr_off; b.status = ix->counters + kCntStatus;
     b.attr_float_mask = ix->attr_float_mask; b.entry = (uint32_t)ix->entry;
     b.queries = queries;
     b.lo = reinterpret_cast<const int32_t*>(lo);
@@ -658,5 +657,18 @@ int boa_get_phase_counts(boa_index* ix, int64_t* active, int n, int* n_phases, v
 }
 
 int boa_last_launch_count(const boa_index* ix) { return ix ? ix->last_launches : 0; }
+
+int boa_device_status(boa_index* ix, int* status, void* stream)
+{
+    if (!ix || !status) return BOA_EINVAL;
+    *status = 0;
+    if (!ix->counters) return BOA_OK;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    uint32_t h = 0;
+    BOA_CUDA(cudaMemcpyAsync(&h, ix->counters + kCntStatus, sizeof(h), cudaMemcpyDeviceToHost, st));
+    BOA_CUDA(cudaStreamSynchronize(st));
+    *status = (int)h;
+    return BOA_OK;
+}
 
 }  // extern "C"

@@ -2,12 +2,18 @@
 // (Eq. 3) and survivor compaction (Algorithm 1, "compact active queries") fused
 // into its epilogue.  sm_100a only.
 //
-// One warp owns one query from start to convergence.  Its candidate pool, the
-// table of recently scored ids and the query vector live in shared memory.  A
-// pool entry is one 64-bit key
+// One warp (one CTA of 32 threads) owns one query from start to convergence.  Its
+// candidate pool, the table of recently scored ids, the query vector and a staging
+// area for neighbour records live in shared memory.  A pool entry is one 64-bit key
 //     [63:60] phi (violated predicates)  [59:29] fp32 bits of d^2  [28:1] id  [0] expanded
 // so that integer order of keys is the lexicographic order (phi, d^2, id): the
 // lambda -> infinity reading of the paper's score dist + lambda*phi.
+//
+// Neighbour records (vector + attribute cells, one contiguous 32-byte-aligned row
+// each) are fetched with one bulk asynchronous copy (cp.async.bulk, the TMA engine)
+// per row into the staging area; a transaction barrier tells the warp when the bytes
+// have landed.  No register holds data in flight, so one warp keeps up to
+// `stage_rows` whole rows in flight at once.
 //
 // Distances are accumulated in a fixed order: a row is cut into 16-byte chunks,
 // chunk c belongs to lane (c mod 8) of an 8-lane group, each lane runs
@@ -21,9 +27,11 @@
 namespace boa {
 
 constexpr uint32_t kNoId = 0xFFFFFFFFu;
-constexpr int kWarpsPerCta = 4;
-constexpr int kThreads = kWarpsPerCta * 32;
+constexpr int kThreads = 32;           // one warp per CTA
 constexpr uint64_t kKeyMax = ~0ull;
+constexpr uint32_t kWaitLimit = 1u << 22;   // bounded wait on the transaction barrier
+
+enum : uint32_t { kStatusCopyTimeout = 1u };
 
 struct SearchParams {
     // index
@@ -32,6 +40,7 @@ struct SearchParams {
     int64_t N;
     int D, m, R;
     int rec_stride;           // bytes, multiple of 32
+    int rec_bytes;            // bytes of a record that are copied (vector + cells, 16-byte multiple)
     int nchunks;              // 16-byte chunks of one vector
     int attr_off;             // byte offset of the attribute cells inside a record
     uint32_t attr_float_mask; // bit j set: column j is float
@@ -48,6 +57,7 @@ struct SearchParams {
     int L;                    // beamwidth: expandable prefix of the pool
     int C;                    // pool capacity (L in restart mode, Lmax in resume mode)
     int hash_log2;            // size of the table of recently scored ids
+    int stage_rows;           // records the staging area holds
     int max_expand;           // expansions after which a phase gives up
     int first_phase;          // statistics start from zero
     int resume_in;            // load the pool a narrower phase spilled
@@ -65,6 +75,7 @@ struct SearchParams {
     uint32_t* ticket;              // work counter of this launch, zero at start
     uint32_t* out_list;            // survivors of this phase
     uint32_t* out_count;
+    uint32_t* status;              // device status word (kStatus* bits)
     // per-query state
     int32_t* final_L;
     int32_t* n_expand;
@@ -88,28 +99,54 @@ __device__ __forceinline__ float key_d2(uint64_t k)
 }
 __device__ __forceinline__ uint32_t key_phi(uint64_t k) { return (uint32_t)(k >> 60); }
 
-__device__ __forceinline__ uint4 ldg_stream128(const void* p)
+__device__ __forceinline__ uint32_t smem_u32(const void* p)
 {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
+    return (uint32_t)__cvta_generic_to_shared(p);
 }
-__device__ __forceinline__ uint32_t ldg_stream32(const void* p)
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count)
 {
-    uint32_t v;
-    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
-    return v;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
+                 "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// One row, global -> shared, completion counted in bytes on `bar`.  No multicast.
+__device__ __forceinline__ void bulk_load_row(void* dst, const void* src, uint32_t bytes, uint64_t* bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+            smem_u32(dst)),
+        "l"(src), "r"(bytes), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ void fence_async_proxy()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-__device__ __forceinline__ float sq_acc4(float acc, uint4 x, float4 q)
+__device__ __forceinline__ float sq_acc4(float acc, float4 x, float4 q)
 {
     float d;
-    d = __uint_as_float(x.x) - q.x; acc = fmaf(d, d, acc);
-    d = __uint_as_float(x.y) - q.y; acc = fmaf(d, d, acc);
-    d = __uint_as_float(x.z) - q.z; acc = fmaf(d, d, acc);
-    d = __uint_as_float(x.w) - q.w; acc = fmaf(d, d, acc);
+    d = x.x - q.x; acc = fmaf(d, d, acc);
+    d = x.y - q.y; acc = fmaf(d, d, acc);
+    d = x.z - q.z; acc = fmaf(d, d, acc);
+    d = x.w - q.w; acc = fmaf(d, d, acc);
     return acc;
 }
 __device__ __forceinline__ float sq_acc_bytes(float acc, uint32_t w, float4 q)
@@ -120,21 +157,6 @@ __device__ __forceinline__ float sq_acc_bytes(float acc, uint32_t w, float4 q)
     d = (float)((w >> 16) & 0xFFu) - q.z; acc = fmaf(d, d, acc);
     d = (float)(w >> 24) - q.w;           acc = fmaf(d, d, acc);
     return acc;
-}
-
-// One 16-byte chunk of a stored vector against the matching slice of the query.
-template <int VT>
-__device__ __forceinline__ float chunk_acc(float acc, uint4 x, const float4* __restrict__ qs, int c)
-{
-    if (VT == 0) {
-        return sq_acc4(acc, x, qs[c]);
-    } else {
-        acc = sq_acc_bytes(acc, x.x, qs[4 * c + 0]);
-        acc = sq_acc_bytes(acc, x.y, qs[4 * c + 1]);
-        acc = sq_acc_bytes(acc, x.z, qs[4 * c + 2]);
-        acc = sq_acc_bytes(acc, x.w, qs[4 * c + 3]);
-        return acc;
-    }
 }
 
 // Bitonic sort of 32*RS keys held one per (lane, slot); element index = lane + 32*slot.
@@ -169,58 +191,65 @@ __device__ __forceinline__ void sort_keys(uint64_t (&x)[RS], int lane)
 
 // Per-warp shared memory carve-up (bytes), shared by host and device.
 struct WarpSmem {
-    int pool_off, nk_off, nr_off, cand_off, hash_off, q_off, total;
+    int pool_off, nk_off, nr_off, cand_off, hash_off, q_off, stage_off, bar_off, total;
 };
-__host__ __device__ inline WarpSmem warp_smem_layout(int C, int hash_log2, int D, int RS)
+__host__ __device__ inline WarpSmem warp_smem_layout(int C, int hash_log2, int D, int RS,
+                                                     int stage_rows, int rec_bytes)
 {
     WarpSmem s;
     int off = 0;
-    s.pool_off = off; off += ((C + 1) & ~1) * 8;
-    s.nk_off = off;   off += 32 * RS * 8;
-    s.q_off = off;    off += ((D * 4 + 15) & ~15);
-    s.hash_off = off; off += (1 << hash_log2) * 4;
-    s.cand_off = off; off += 32 * RS * 4;
-    s.nr_off = off;   off += 32 * RS * 4;
-    s.total = (off + 15) & ~15;
+    s.stage_off = off; off += stage_rows * rec_bytes;          // 16-byte multiple
+    s.pool_off = off;  off += ((C + 1) & ~1) * 8;
+    s.nk_off = off;    off += 32 * RS * 8;
+    s.q_off = off;     off += ((D * 4 + 15) & ~15);
+    s.hash_off = off;  off += (1 << hash_log2) * 4;
+    s.cand_off = off;  off += 32 * RS * 4;
+    s.nr_off = off;    off += 32 * RS * 4;
+    s.bar_off = off;   off += 16;
+    s.total = (off + 127) & ~127;
     return s;
 }
 
 // ---------------------------------------------------------------- the kernel
-// VT: 0 = float vectors, 1 = uint8 vectors.  CPL: 16-byte chunks each lane of an
-// 8-lane group reads per neighbour (0 = run-time loop for long rows).  RS: adjacency
-// slots per lane (1: R <= 32, 2: R <= 64).  U: neighbour rounds kept in flight.
-template <int VT, int CPL, int RS, int U>
+// VT: 0 = float vectors, 1 = uint8 vectors.  RS: adjacency slots per lane (1: R <= 32,
+// 2: R <= 64).
+template <int VT, int RS>
 __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams p)
 {
-    extern __shared__ __align__(16) uint8_t smem_raw[];
-    const int lane = threadIdx.x & 31;
-    const int warp = threadIdx.x >> 5;
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    const int lane = threadIdx.x;
     const int g = lane & 7;        // lane inside its 8-lane group
     const int gi = lane >> 3;      // group index 0..3
     const unsigned lt_mask = (1u << lane) - 1u;
 
-    const WarpSmem lay = warp_smem_layout(p.C, p.hash_log2, p.D, RS);
-    uint8_t* base = smem_raw + (size_t)warp * lay.total;
-    uint64_t* pool = reinterpret_cast<uint64_t*>(base + lay.pool_off);
-    uint64_t* nk = reinterpret_cast<uint64_t*>(base + lay.nk_off);
-    uint32_t* nr = reinterpret_cast<uint32_t*>(base + lay.nr_off);
-    uint32_t* cand = reinterpret_cast<uint32_t*>(base + lay.cand_off);
-    uint32_t* hash = reinterpret_cast<uint32_t*>(base + lay.hash_off);
-    float4* qs = reinterpret_cast<float4*>(base + lay.q_off);
+    const WarpSmem lay = warp_smem_layout(p.C, p.hash_log2, p.D, RS, p.stage_rows, p.rec_bytes);
+    uint8_t* stage = smem_raw + lay.stage_off;
+    uint64_t* pool = reinterpret_cast<uint64_t*>(smem_raw + lay.pool_off);
+    uint64_t* nk = reinterpret_cast<uint64_t*>(smem_raw + lay.nk_off);
+    uint32_t* nr = reinterpret_cast<uint32_t*>(smem_raw + lay.nr_off);
+    uint32_t* cand = reinterpret_cast<uint32_t*>(smem_raw + lay.cand_off);
+    uint32_t* hash = reinterpret_cast<uint32_t*>(smem_raw + lay.hash_off);
+    float4* qs = reinterpret_cast<float4*>(smem_raw + lay.q_off);
+    uint64_t* bar = reinterpret_cast<uint64_t*>(smem_raw + lay.bar_off);
 
     const uint32_t hmask = (1u << p.hash_log2) - 1u;
     const int hshift = 32 - p.hash_log2;
 
     // work range of this launch
-    uint32_t w_begin = p.in_begin_ptr ? *p.in_begin_ptr : p.in_begin;
-    uint32_t w_end = p.in_end_ptr ? *p.in_end_ptr : p.in_end;
+    const uint32_t w_begin = p.in_begin_ptr ? *p.in_begin_ptr : p.in_begin;
+    const uint32_t w_end = p.in_end_ptr ? *p.in_end_ptr : p.in_end;
     if (p.active_count) {
         // Algorithm 1: "while |A| > tau * rho"
         if (!((double)(*p.active_count) > p.tau_q)) return;
     }
     const uint32_t n_work = w_end > w_begin ? w_end - w_begin : 0u;
 
-    for (;;) {
+    if (lane == 0) mbar_init(bar, 1u);
+    __syncwarp();
+    uint32_t bar_parity = 0;
+    bool dead = false;             // a copy never completed: stop taking work
+
+    while (!dead) {
         uint32_t t = 0;
         if (lane == 0) t = atomicAdd(p.ticket, 1u);
         t = __shfl_sync(0xffffffffu, t, 0);
@@ -243,87 +272,74 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
         const bool my_float = (p.attr_float_mask >> g) & 1u;
         __syncwarp();
 
-        // Scores cand[0..cnt) (distance + violated predicates) into nk[0..cnt).
+        // Scores cand[0..cnt): fetch the records, distance + violated predicates -> nk[0..cnt).
         auto score = [&](int cnt) {
-            constexpr int UU = (CPL == 0) ? 1 : U;
-            constexpr int NC = (CPL == 0) ? 8 : CPL;
-            for (int r0 = 0; r0 < cnt; r0 += 4 * UU) {
-                uint4 v[UU][NC];
-                uint32_t av[UU];
-                float acc[UU];
-                const uint8_t* row[UU];
-                bool act[UU];
-#pragma unroll
-                for (int u = 0; u < UU; ++u) {
-                    const int j = r0 + 4 * u + gi;
-                    act[u] = j < cnt;
-                    const uint32_t n = act[u] ? cand[j] : 0u;
-                    row[u] = p.rec + (size_t)n * p.rec_stride;
-                    av[u] = 0u;
-                    acc[u] = 0.0f;
-                    if (act[u]) {
-#pragma unroll
-                        for (int i = 0; i < NC; ++i) {
-                            const int c = g + 8 * i;
-                            if (c < p.nchunks) v[u][i] = ldg_stream128(row[u] + 16 * c);
-                        }
-                        if (g < p.m) av[u] = ldg_stream32(row[u] + p.attr_off + 4 * g);
-                    }
+            for (int b0 = 0; b0 < cnt && !dead; b0 += p.stage_rows) {
+                const int nb = (cnt - b0 < p.stage_rows) ? cnt - b0 : p.stage_rows;
+                fence_async_proxy();
+                if (lane == 0) mbar_expect_tx(bar, (uint32_t)(nb * p.rec_bytes));
+                __syncwarp();
+                for (int j = lane; j < nb; j += 32) {
+                    const uint32_t n = cand[b0 + j];
+                    bulk_load_row(stage + (size_t)j * p.rec_bytes, p.rec + (size_t)n * p.rec_stride,
+                                  (uint32_t)p.rec_bytes, bar);
                 }
-#pragma unroll
-                for (int u = 0; u < UU; ++u) {
-                    if (act[u]) {
-#pragma unroll
-                        for (int i = 0; i < NC; ++i) {
-                            const int c = g + 8 * i;
-                            if (c < p.nchunks) acc[u] = chunk_acc<VT>(acc[u], v[u][i], qs, c);
-                        }
-                        if (CPL == 0) {
-                            // long rows: keep going in blocks of 8 chunks per lane
-                            for (int c0 = 64; c0 < p.nchunks; c0 += 64) {
-                                uint4 w[8];
-#pragma unroll
-                                for (int i = 0; i < 8; ++i) {
-                                    const int c = c0 + g + 8 * i;
-                                    if (c < p.nchunks) w[i] = ldg_stream128(row[u] + 16 * c);
-                                }
-#pragma unroll
-                                for (int i = 0; i < 8; ++i) {
-                                    const int c = c0 + g + 8 * i;
-                                    if (c < p.nchunks) acc[u] = chunk_acc<VT>(acc[u], w[i], qs, c);
-                                }
+                uint32_t spins = 0;
+                while (!mbar_try_wait(bar, bar_parity)) {
+                    if (++spins > kWaitLimit) { dead = true; break; }
+                }
+                dead = __any_sync(0xffffffffu, dead);
+                bar_parity ^= 1u;
+                if (dead) {
+                    if (lane == 0) atomicOr(p.status, kStatusCopyTimeout);
+                    break;
+                }
+                for (int r0 = 0; r0 < nb; r0 += 4) {
+                    const int j = r0 + gi;
+                    const bool act = j < nb;
+                    const uint8_t* row = stage + (size_t)(act ? j : 0) * p.rec_bytes;
+                    float acc = 0.0f;
+                    if (act) {
+                        if (VT == 0) {
+                            const float4* r4 = reinterpret_cast<const float4*>(row);
+#pragma unroll 4
+                            for (int c = g; c < p.nchunks; c += 8) acc = sq_acc4(acc, r4[c], qs[c]);
+                        } else {
+                            const uint4* r4 = reinterpret_cast<const uint4*>(row);
+                            for (int c = g; c < p.nchunks; c += 8) {
+                                const uint4 x = r4[c];
+                                acc = sq_acc_bytes(acc, x.x, qs[4 * c + 0]);
+                                acc = sq_acc_bytes(acc, x.y, qs[4 * c + 1]);
+                                acc = sq_acc_bytes(acc, x.z, qs[4 * c + 2]);
+                                acc = sq_acc_bytes(acc, x.w, qs[4 * c + 3]);
                             }
                         }
                     }
-                    float a = acc[u];
-                    a += __shfl_xor_sync(0xffffffffu, a, 4);
-                    a += __shfl_xor_sync(0xffffffffu, a, 2);
-                    a += __shfl_xor_sync(0xffffffffu, a, 1);
+                    acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+                    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+                    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
                     bool viol = false;
-                    if (act[u] && g < p.m) {
+                    if (act && g < p.m) {
+                        const uint32_t av = *reinterpret_cast<const uint32_t*>(row + p.attr_off + 4 * g);
                         if (my_float) {
-                            const float x = __uint_as_float(av[u]);
+                            const float x = __uint_as_float(av);
                             viol = !(x >= __int_as_float(my_lo) && x <= __int_as_float(my_hi));
                         } else {
-                            const int32_t x = (int32_t)av[u];
+                            const int32_t x = (int32_t)av;
                             viol = x < my_lo || x > my_hi;
                         }
                     }
-                    const unsigned b = __ballot_sync(0xffffffffu, viol);
-                    const uint32_t phi = __popc((b >> (8 * gi)) & 0xFFu);
-                    if (act[u] && g == 0) {
-                        const int j = r0 + 4 * u + gi;
-                        nk[j] = pack_key(phi, a, cand[j]);
-                    }
+                    const unsigned bal = __ballot_sync(0xffffffffu, viol);
+                    const uint32_t phi = __popc((bal >> (8 * gi)) & 0xFFu);
+                    if (act && g == 0) nk[b0 + j] = pack_key(phi, acc, cand[b0 + j]);
                 }
+                __syncwarp();
             }
-            __syncwarp();
         };
 
-        auto hash_slot = [&](uint32_t id) -> uint32_t { return (id * 0x9E3779B1u) >> hshift; };
         // Returns true when id was not in the table; records it either way.
         auto hash_test_and_set = [&](uint32_t id) -> bool {
-            const uint32_t h = hash_slot(id);
+            const uint32_t h = (id * 0x9E3779B1u) >> hshift;
             int empty = -1;
 #pragma unroll
             for (int pr = 0; pr < 4; ++pr) {
@@ -363,7 +379,7 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
         }
 
         // ---- Algorithm 2 main loop
-        for (;;) {
+        while (!dead) {
             // nearest unexpanded entry among the first L
             const int lim = n < p.L ? n : p.L;
             int pos = -1;
@@ -383,7 +399,6 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
 
             // adjacency row, drop ids scored before, compact the rest
             uint32_t nb[RS];
-            bool fresh[RS];
             const uint32_t* grow = p.graph + (size_t)u_id * p.R;
 #pragma unroll
             for (int s = 0; s < RS; ++s) {
@@ -393,9 +408,9 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
             int cnt = 0;
 #pragma unroll
             for (int s = 0; s < RS; ++s) {
-                fresh[s] = (nb[s] != kNoId) && hash_test_and_set(nb[s]);
-                const unsigned bal = __ballot_sync(0xffffffffu, fresh[s]);
-                if (fresh[s]) cand[cnt + __popc(bal & lt_mask)] = nb[s];
+                const bool fresh = (nb[s] != kNoId) && hash_test_and_set(nb[s]);
+                const unsigned bal = __ballot_sync(0xffffffffu, fresh);
+                if (fresh) cand[cnt + __popc(bal & lt_mask)] = nb[s];
                 cnt += __popc(bal);
             }
             __syncwarp();
@@ -404,43 +419,48 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
 
             // gather + distance + range check (fused)
             score(cnt);
+            if (dead) break;
 
-            // sort the new keys
+            // new keys that cannot enter a full pool are dropped right away; sort the rest
+            const uint64_t worst = (n == p.C) ? (pool[n - 1] >> 1) : (kKeyMax >> 1);
             uint64_t x[RS];
+            int live = 0;
 #pragma unroll
             for (int s = 0; s < RS; ++s) {
                 const int j = lane + 32 * s;
                 x[s] = (j < cnt) ? nk[j] : kKeyMax;
+                if (x[s] != kKeyMax && (x[s] >> 1) >= worst) x[s] = kKeyMax;
+                live += __popc(__ballot_sync(0xffffffffu, x[s] != kKeyMax));
             }
-            if (cnt > 1) sort_keys<RS>(x, lane);
+            if (live == 0) continue;
+            if (live > 1) sort_keys<RS>(x, lane);
             __syncwarp();
 
             // rank of every new key in the pool; drop keys the pool already holds
             int steps = 0;
             while ((1 << steps) <= n) ++steps;
-            int rnk[RS];
             bool keep[RS];
             int kept = 0;
             int pos_new[RS];
 #pragma unroll
             for (int s = 0; s < RS; ++s) {
                 const uint64_t xs = x[s] >> 1;
-                int lo_i = 0, hi_i = n;
-                for (int it = 0; it < steps; ++it) {
-                    const int mid = (lo_i + hi_i) >> 1;
-                    const bool go = (lo_i < hi_i) && ((pool[mid] >> 1) < xs);
-                    if (lo_i < hi_i) { if (go) lo_i = mid + 1; else hi_i = mid; }
-                }
-                rnk[s] = lo_i;
                 const bool valid = x[s] != kKeyMax;
+                int lo_i = 0, hi_i = valid ? n : 0;
+                for (int it = 0; it < steps; ++it) {
+                    if (lo_i < hi_i) {
+                        const int mid = (lo_i + hi_i) >> 1;
+                        if ((pool[mid] >> 1) < xs) lo_i = mid + 1; else hi_i = mid;
+                    }
+                }
                 const bool dup = valid && (lo_i < n) && ((pool[lo_i] >> 1) == xs);
                 const bool nd = valid && !dup;
                 const unsigned bal = __ballot_sync(0xffffffffu, nd);
                 const int pidx = kept + __popc(bal & lt_mask);
-                pos_new[s] = rnk[s] + pidx;
+                pos_new[s] = lo_i + pidx;
                 keep[s] = nd && (pos_new[s] < p.C);
                 const unsigned kb = __ballot_sync(0xffffffffu, keep[s]);
-                if (keep[s]) nr[pidx] = (uint32_t)rnk[s];
+                if (keep[s]) nr[pidx] = (uint32_t)lo_i;
                 kept += __popc(kb);
             }
             __syncwarp();
@@ -454,12 +474,16 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
                 int sh = 0;
                 if (i < n && i >= rmin) {
                     e = pool[i];
-                    int a = 0, b = kept;             // upper_bound(nr, i)
-                    while (a < b) {
-                        const int mid = (a + b) >> 1;
-                        if ((int)nr[mid] <= i) a = mid + 1; else b = mid;
+                    if (kept <= 8) {
+                        for (int j = 0; j < kept; ++j) sh += ((int)nr[j] <= i) ? 1 : 0;
+                    } else {
+                        int a = 0, b = kept;             // upper_bound(nr, i)
+                        while (a < b) {
+                            const int mid = (a + b) >> 1;
+                            if ((int)nr[mid] <= i) a = mid + 1; else b = mid;
+                        }
+                        sh = a;
                     }
-                    sh = a;
                 }
                 __syncwarp();
                 if (sh > 0 && i + sh < p.C) pool[i + sh] = e;
@@ -472,6 +496,7 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
             if (rmin < cur) cur = rmin;
             __syncwarp();
         }
+        if (dead) break;
 
         // ---- result: the k nearest filter-valid entries (valid ones sort first)
         const int lim = n < p.L ? n : p.L;

@@ -40,8 +40,9 @@ def test_boa_matches_oracle_bit_for_bit(name, mode):
     w, d, orc, gpu, g = _get(name)
     assert orc.entry == gpu.entry
     widths = default_widths(w.L0, min(w.Lmax, 256))
-    o = orc.search(d["queries"], d["lo"], d["hi"], w.k, widths, mode=mode, dist_mode=1)
-    r = gpu_search(gpu, g, w.k, widths, mode=mode)
+    eps = {"c4": 0.2}.get(name, 0.05)      # chosen so that some queries stop early, some escalate
+    o = orc.search(d["queries"], d["lo"], d["hi"], w.k, widths, eps=eps, mode=mode, dist_mode=1)
+    r = gpu_search(gpu, g, w.k, widths, eps=eps, mode=mode)
     assert_bit_parity(o, r, f"{name}/{mode}")
     assert len(set(o["final_L"].tolist())) > 1 or name == "c1"
 
