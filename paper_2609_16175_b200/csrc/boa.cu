@@ -187,7 +187,7 @@ constexpr int kCntSnap = 32;                          // [pool] frozen end of ph
 constexpr int kCntStatus = 47;                        // device status bits
 constexpr int kCntTicket = 48;                        // one per launch
 constexpr int kMaxLaunches = 128;
-constexpr int kCntWords = kCntTicket + kMaxLaunches;
+constexpr int kCntWords = kCntTicket + kMaxLaunches;   // 176: the 64-bit words after it stay aligned
 
 typedef void (*SearchKernel)(const boa::SearchParams);
 
@@ -196,29 +196,48 @@ struct KernelChoice {
     int rs;
 };
 
+template <int VT, int CPL>
+KernelChoice pick_rs(int R)
+{
+    if (R <= 32) return {boa::boa_search_kernel<VT, 1, CPL>, 1};
+    return {boa::boa_search_kernel<VT, 2, CPL>, 2};
+}
+
 KernelChoice pick_kernel(const boa_index* ix)
 {
+    const int cpl = (ix->nchunks + 7) / 8;      // 16-byte chunks per lane of an 8-lane group
     if (ix->vec_dtype == BOA_F32) {
-        if (ix->R <= 32) return {boa::boa_search_kernel<0, 1>, 1};
-        return {boa::boa_search_kernel<0, 2>, 2};
+        switch (cpl) {
+            case 1: return pick_rs<0, 1>(ix->R);
+            case 2: return pick_rs<0, 2>(ix->R);
+            case 3: return pick_rs<0, 3>(ix->R);
+            case 4: return pick_rs<0, 4>(ix->R);
+            default: return pick_rs<0, 0>(ix->R);
+        }
     }
-    if (ix->R <= 32) return {boa::boa_search_kernel<1, 1>, 1};
-    return {boa::boa_search_kernel<1, 2>, 2};
+    switch (cpl) {
+        case 1: return pick_rs<1, 1>(ix->R);
+        case 2: return pick_rs<1, 2>(ix->R);
+        default: return pick_rs<1, 0>(ix->R);
+    }
 }
 
 int choose_hash_log2(const boa_index* ix, int L)
 {
     if (ix->hash_log2) return ix->hash_log2;
-    if (L <= 32) return 10;
-    if (L <= 128) return 11;
-    return 12;
+    int lg = (L <= 32) ? 11 : 12;     // 16-bit entries: 4 KB / 8 KB per query
+    int id_bits = 1;
+    while (((int64_t)1 << id_bits) < ix->N) ++id_bits;
+    if (id_bits - (lg - 2) > 16) lg = id_bits - 14;     // tags must fit 16 bits
+    return lg;
 }
 
 int choose_stage_rows(const boa_index* ix, int rs)
 {
     int rows = ix->stage_rows ? ix->stage_rows : 8192 / ix->rec_bytes;
-    if (rows < 2) rows = 2;
     if (rows > 32 * rs) rows = 32 * rs;
+    if (rows >= 16) rows &= ~1;       // two ring slots of equal size
+    if (rows < 1) rows = 1;
     return rows;
 }
 
@@ -245,7 +264,9 @@ int ensure_workspace(boa_index* ix, int64_t Q, int Lmax)
 {
     const int need_spill = ix->mode == 1 ? ((Lmax + 1) & ~1) : 0;
     if (ix->counters == nullptr) {
-        BOA_CUDA(cudaMalloc(&ix->counters, kCntWords * sizeof(uint32_t)));
+        // 12 trailing 64-bit words: section timers of debug builds
+        BOA_CUDA(cudaMalloc(&ix->counters, kCntWords * sizeof(uint32_t) + 12 * sizeof(unsigned long long)));
+        BOA_CUDA(cudaMemset(ix->counters, 0, kCntWords * sizeof(uint32_t) + 12 * sizeof(unsigned long long)));
     }
     if (Q > ix->ws_Q || need_spill > ix->ws_spill) {
         const int64_t nq = Q > ix->ws_Q ? Q : ix->ws_Q;
@@ -284,6 +305,15 @@ int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_p
     sp.L = L;
     sp.C = ix->mode == 1 ? Lmax : L;
     sp.hash_log2 = choose_hash_log2(ix, L);
+    {
+        int id_bits = 1;
+        while (((int64_t)1 << id_bits) < ix->N) ++id_bits;
+        if (id_bits - (sp.hash_log2 - 2) > 16) sp.hash_log2 = id_bits - 14;
+        int bucket_bits = sp.hash_log2 - 2;
+        if (bucket_bits > id_bits) bucket_bits = id_bits;
+        sp.id_bits = id_bits;
+        sp.tag_bits = id_bits - bucket_bits;
+    }
     sp.stage_rows = choose_stage_rows(ix, lp.kc.rs);
     sp.max_expand = ix->cap_mult * L + ix->cap_add;
     sp.first_phase = p == 0;
@@ -482,7 +512,7 @@ int boa_set_param(boa_index* ix, int key, double v)
             if (v < 0.0 || v > 1e6 || v != floor(v)) return BOA_EINVAL;
             ix->cap_add = (int)v; return BOA_OK;
         case BOA_PARAM_HASH_LOG2:
-            if (v != 0.0 && (v < 8.0 || v > 14.0 || v != floor(v))) return BOA_EINVAL;
+            if (v != 0.0 && (v < 8.0 || v > 15.0 || v != floor(v))) return BOA_EINVAL;
             ix->hash_log2 = (int)v; return BOA_OK;
         case BOA_PARAM_STAGE_ROWS:
             if (v < 0.0 || v > 64.0 || v != floor(v)) return BOA_EINVAL;
@@ -540,6 +570,7 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
     b.rec = ix->rec; b.graph = ix->graph; b.N = ix->N; b.D = ix->D; b.m = ix->m; b.R = ix->R;
     b.rec_stride = ix->rec_stride; b.rec_bytes = ix->rec_bytes; b.nchunks = ix->nchunks;
     b.attr_off = ix->attr_off; b.status = ix->counters + kCntStatus;
+    b.timers = reinterpret_cast<unsigned long long*>(ix->counters + kCntWords);
     b.attr_float_mask = ix->attr_float_mask; b.entry = (uint32_t)ix->entry;
     b.queries = queries;
     b.lo = reinterpret_cast<const int32_t*>(lo);
@@ -657,6 +688,19 @@ int boa_get_phase_counts(boa_index* ix, int64_t* active, int n, int* n_phases, v
 }
 
 int boa_last_launch_count(const boa_index* ix) { return ix ? ix->last_launches : 0; }
+
+#ifdef BOA_SECTION_TIMERS
+// Debug builds only: cycles per kernel section, summed over warps (12 values, HOST array).
+int boa_debug_timers(boa_index* ix, unsigned long long* out, int reset)
+{
+    if (!ix || !out || !ix->counters) return BOA_EINVAL;
+    unsigned long long* d = reinterpret_cast<unsigned long long*>(ix->counters + kCntWords);
+    BOA_CUDA(cudaDeviceSynchronize());
+    BOA_CUDA(cudaMemcpy(out, d, 12 * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+    if (reset) BOA_CUDA(cudaMemset(d, 0, 12 * sizeof(unsigned long long)));
+    return BOA_OK;
+}
+#endif
 
 int boa_device_status(boa_index* ix, int* status, void* stream)
 {

@@ -11,9 +11,17 @@
 //
 // Neighbour records (vector + attribute cells, one contiguous 32-byte-aligned row
 // each) are fetched with one bulk asynchronous copy (cp.async.bulk, the TMA engine)
-// per row into the staging area; a transaction barrier tells the warp when the bytes
-// have landed.  No register holds data in flight, so one warp keeps up to
-// `stage_rows` whole rows in flight at once.
+// per row into a two-slot ring in shared memory; one transaction barrier per slot
+// tells the warp when the bytes have landed.  No register holds data in flight, so
+// one warp keeps up to `stage_rows` whole rows in flight while it scores the rows
+// that have already arrived.
+//
+// The table of recently scored ids stores 16-bit tags in 4-way buckets.  An id is
+// first mapped by an odd multiplier modulo 2^id_bits (a bijection); the high bits
+// pick the bucket and the low bits are the tag, so bucket + tag identify the id
+// exactly: the table can forget an id, it can never report an unseen id as seen.
+// A forgotten id that is met again is scored again and then recognised by its key
+// in the pool (or rejected again by the pool's worst key), so results never change.
 //
 // Distances are accumulated in a fixed order: a row is cut into 16-byte chunks,
 // chunk c belongs to lane (c mod 8) of an 8-lane group, each lane runs
@@ -29,9 +37,21 @@ namespace boa {
 constexpr uint32_t kNoId = 0xFFFFFFFFu;
 constexpr int kThreads = 32;           // one warp per CTA
 constexpr uint64_t kKeyMax = ~0ull;
-constexpr uint32_t kWaitLimit = 1u << 22;   // bounded wait on the transaction barrier
+constexpr uint32_t kWaitLimit = 1u << 20;   // bounded wait on a transaction barrier (tries)
+constexpr uint32_t kWaitHintNs = 2000u;     // each try may block this long inside the instruction
 
 enum : uint32_t { kStatusCopyTimeout = 1u };
+
+// Optional per-section cycle counters (build with -DBOA_SECTION_TIMERS; off in the product).
+#ifdef BOA_SECTION_TIMERS
+#define BOA_T_DECL long long t_prev_ = clock64(); long long t_acc_[12] = {0}
+#define BOA_T_MARK(i) do { long long t_now_ = clock64(); t_acc_[i] += t_now_ - t_prev_; t_prev_ = t_now_; } while (0)
+#define BOA_T_FLUSH(ptr) do { if (lane == 0 && (ptr)) for (int i_ = 0; i_ < 12; ++i_) atomicAdd((unsigned long long*)(ptr) + i_, (unsigned long long)t_acc_[i_]); } while (0)
+#else
+#define BOA_T_DECL
+#define BOA_T_MARK(i)
+#define BOA_T_FLUSH(ptr)
+#endif
 
 struct SearchParams {
     // index
@@ -56,8 +76,10 @@ struct SearchParams {
     // phase
     int L;                    // beamwidth: expandable prefix of the pool
     int C;                    // pool capacity (L in restart mode, Lmax in resume mode)
-    int hash_log2;            // size of the table of recently scored ids
-    int stage_rows;           // records the staging area holds
+    int hash_log2;            // log2 of the 16-bit entries in the table of recently scored ids
+    int id_bits;              // bits of a node id (ids < 2^id_bits)
+    int tag_bits;             // id_bits - log2(buckets), at most 16
+    int stage_rows;           // records the staging ring holds (two slots of half that)
     int max_expand;           // expansions after which a phase gives up
     int first_phase;          // statistics start from zero
     int resume_in;            // load the pool a narrower phase spilled
@@ -76,6 +98,7 @@ struct SearchParams {
     uint32_t* out_list;            // survivors of this phase
     uint32_t* out_count;
     uint32_t* status;              // device status word (kStatus* bits)
+    unsigned long long* timers;    // section cycle counters (only with BOA_SECTION_TIMERS)
     // per-query state
     int32_t* final_L;
     int32_t* n_expand;
@@ -114,15 +137,16 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
                  "r"(bytes)
                  : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
+// Blocks for at most about `hint_ns` inside the instruction, then reports.
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, uint32_t hint_ns)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
         : "memory");
     return ok != 0;
 }
@@ -202,7 +226,7 @@ __host__ __device__ inline WarpSmem warp_smem_layout(int C, int hash_log2, int D
     s.pool_off = off;  off += ((C + 1) & ~1) * 8;
     s.nk_off = off;    off += 32 * RS * 8;
     s.q_off = off;     off += ((D * 4 + 15) & ~15);
-    s.hash_off = off;  off += (1 << hash_log2) * 4;
+    s.hash_off = off;  off += (1 << hash_log2) * 2;
     s.cand_off = off;  off += 32 * RS * 4;
     s.nr_off = off;    off += 32 * RS * 4;
     s.bar_off = off;   off += 16;
@@ -212,8 +236,10 @@ __host__ __device__ inline WarpSmem warp_smem_layout(int C, int hash_log2, int D
 
 // ---------------------------------------------------------------- the kernel
 // VT: 0 = float vectors, 1 = uint8 vectors.  RS: adjacency slots per lane (1: R <= 32,
-// 2: R <= 64).
-template <int VT, int RS>
+// 2: R <= 64).  CPL: 16-byte chunks of a row per lane of an 8-lane group when that is
+// at most 4 (the lane then keeps its slices of the query in registers and the chunk
+// loop is unrolled); 0 = any length, query slices read from shared memory.
+template <int VT, int RS, int CPL>
 __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams p)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -221,6 +247,8 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
     const int g = lane & 7;        // lane inside its 8-lane group
     const int gi = lane >> 3;      // group index 0..3
     const unsigned lt_mask = (1u << lane) - 1u;
+    constexpr int QF4 = (VT == 0) ? 1 : 4;          // float4 slices of the query per chunk
+    constexpr int NQ = (CPL > 0) ? CPL * QF4 : 1;
 
     const WarpSmem lay = warp_smem_layout(p.C, p.hash_log2, p.D, RS, p.stage_rows, p.rec_bytes);
     uint8_t* stage = smem_raw + lay.stage_off;
@@ -228,12 +256,14 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
     uint64_t* nk = reinterpret_cast<uint64_t*>(smem_raw + lay.nk_off);
     uint32_t* nr = reinterpret_cast<uint32_t*>(smem_raw + lay.nr_off);
     uint32_t* cand = reinterpret_cast<uint32_t*>(smem_raw + lay.cand_off);
-    uint32_t* hash = reinterpret_cast<uint32_t*>(smem_raw + lay.hash_off);
+    uint16_t* hash = reinterpret_cast<uint16_t*>(smem_raw + lay.hash_off);
     float4* qs = reinterpret_cast<float4*>(smem_raw + lay.q_off);
-    uint64_t* bar = reinterpret_cast<uint64_t*>(smem_raw + lay.bar_off);
+    uint64_t* bar = reinterpret_cast<uint64_t*>(smem_raw + lay.bar_off);   // bar[0], bar[1]
 
-    const uint32_t hmask = (1u << p.hash_log2) - 1u;
-    const int hshift = 32 - p.hash_log2;
+    const uint32_t id_mask = (p.id_bits >= 32) ? 0xFFFFFFFFu : ((1u << p.id_bits) - 1u);
+    const uint32_t tag_mask = (1u << p.tag_bits) - 1u;
+    const int n_slots = p.stage_rows >= 16 ? 2 : 1;   // ring slots of the staging area
+    const int half_rows = p.stage_rows / n_slots;      // rows per slot
 
     // work range of this launch
     const uint32_t w_begin = p.in_begin_ptr ? *p.in_begin_ptr : p.in_begin;
@@ -244,9 +274,10 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
     }
     const uint32_t n_work = w_end > w_begin ? w_end - w_begin : 0u;
 
-    if (lane == 0) mbar_init(bar, 1u);
+    if (lane == 0) { mbar_init(bar, 1u); mbar_init(bar + 1, 1u); }
     __syncwarp();
-    uint32_t bar_parity = 0;
+    uint32_t bar_parity = 0;       // bit s: parity the next wait on slot s expects
+    BOA_T_DECL;
     bool dead = false;             // a copy never completed: stop taking work
 
     while (!dead) {
@@ -260,9 +291,9 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
         {
             const float4* qsrc = reinterpret_cast<const float4*>(p.queries + (size_t)qi * p.D);
             for (int i = lane; i < p.D / 4; i += 32) qs[i] = qsrc[i];
-            uint4 ff = make_uint4(kNoId, kNoId, kNoId, kNoId);
+            const uint4 ff = make_uint4(~0u, ~0u, ~0u, ~0u);
             uint4* h4 = reinterpret_cast<uint4*>(hash);
-            for (int i = lane; i < (1 << p.hash_log2) / 4; i += 32) h4[i] = ff;
+            for (int i = lane; i < (1 << p.hash_log2) / 8; i += 32) h4[i] = ff;
         }
         int32_t my_lo = 0, my_hi = 0;
         if (g < p.m) {
@@ -271,85 +302,162 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
         }
         const bool my_float = (p.attr_float_mask >> g) & 1u;
         __syncwarp();
+        float4 qreg[NQ];           // this lane's slices of the query (CPL > 0)
+        if (CPL > 0) {
+#pragma unroll
+            for (int i = 0; i < (CPL > 0 ? CPL : 1); ++i) {
+                const int c = g + 8 * i;
+#pragma unroll
+                for (int f = 0; f < QF4; ++f)
+                    qreg[i * QF4 + f] = (c < p.nchunks) ? qs[c * QF4 + f] : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
 
-        // Scores cand[0..cnt): fetch the records, distance + violated predicates -> nk[0..cnt).
+        // squared distance contribution of this lane to one staged row
+        auto row_partial = [&](const uint8_t* row) -> float {
+            float acc = 0.0f;
+            if (CPL > 0) {
+#pragma unroll
+                for (int i = 0; i < (CPL > 0 ? CPL : 1); ++i) {
+                    const int c = g + 8 * i;
+                    if (c < p.nchunks) {
+                        if (VT == 0) {
+                            acc = sq_acc4(acc, reinterpret_cast<const float4*>(row)[c], qreg[i]);
+                        } else {
+                            const uint4 x = reinterpret_cast<const uint4*>(row)[c];
+                            acc = sq_acc_bytes(acc, x.x, qreg[4 * i + 0]);
+                            acc = sq_acc_bytes(acc, x.y, qreg[4 * i + 1]);
+                            acc = sq_acc_bytes(acc, x.z, qreg[4 * i + 2]);
+                            acc = sq_acc_bytes(acc, x.w, qreg[4 * i + 3]);
+                        }
+                    }
+                }
+            } else {
+                for (int c = g; c < p.nchunks; c += 8) {
+                    if (VT == 0) {
+                        acc = sq_acc4(acc, reinterpret_cast<const float4*>(row)[c], qs[c]);
+                    } else {
+                        const uint4 x = reinterpret_cast<const uint4*>(row)[c];
+                        acc = sq_acc_bytes(acc, x.x, qs[4 * c + 0]);
+                        acc = sq_acc_bytes(acc, x.y, qs[4 * c + 1]);
+                        acc = sq_acc_bytes(acc, x.z, qs[4 * c + 2]);
+                        acc = sq_acc_bytes(acc, x.w, qs[4 * c + 3]);
+                    }
+                }
+            }
+            return acc;
+        };
+        auto violates = [&](const uint8_t* row) -> bool {
+            const uint32_t av = *reinterpret_cast<const uint32_t*>(row + p.attr_off + 4 * g);
+            if (my_float) {
+                const float x = __uint_as_float(av);
+                return !(x >= __int_as_float(my_lo) && x <= __int_as_float(my_hi));
+            }
+            const int32_t x = (int32_t)av;
+            return x < my_lo || x > my_hi;
+        };
+
+        // Scores cand[0..cnt): fetch the records through the two-slot ring, then
+        // distance + violated predicates -> nk[0..cnt).
         auto score = [&](int cnt) {
-            for (int b0 = 0; b0 < cnt && !dead; b0 += p.stage_rows) {
-                const int nb = (cnt - b0 < p.stage_rows) ? cnt - b0 : p.stage_rows;
-                fence_async_proxy();
-                if (lane == 0) mbar_expect_tx(bar, (uint32_t)(nb * p.rec_bytes));
-                __syncwarp();
+            const int nbatch = (cnt + half_rows - 1) / half_rows;
+            auto issue = [&](int b) {
+                const int s = (n_slots == 2) ? (b & 1) : 0;
+                const int b0 = b * half_rows;
+                const int nb = (cnt - b0 < half_rows) ? cnt - b0 : half_rows;
+                if (lane == 0) mbar_expect_tx(bar + s, (uint32_t)(nb * p.rec_bytes));
+                uint8_t* dst = stage + (size_t)s * half_rows * p.rec_bytes;
                 for (int j = lane; j < nb; j += 32) {
                     const uint32_t n = cand[b0 + j];
-                    bulk_load_row(stage + (size_t)j * p.rec_bytes, p.rec + (size_t)n * p.rec_stride,
-                                  (uint32_t)p.rec_bytes, bar);
+                    bulk_load_row(dst + (size_t)j * p.rec_bytes, p.rec + (size_t)n * p.rec_stride,
+                                  (uint32_t)p.rec_bytes, bar + s);
                 }
+            };
+            BOA_T_MARK(3);
+            issue(0);
+            if (n_slots == 2 && nbatch > 1) issue(1);
+            BOA_T_MARK(4);
+            for (int b = 0; b < nbatch; ++b) {
+                const int s = (n_slots == 2) ? (b & 1) : 0;
+                const int b0 = b * half_rows;
+                const int nb = (cnt - b0 < half_rows) ? cnt - b0 : half_rows;
                 uint32_t spins = 0;
-                while (!mbar_try_wait(bar, bar_parity)) {
+                while (!mbar_try_wait(bar + s, (bar_parity >> s) & 1u, kWaitHintNs)) {
                     if (++spins > kWaitLimit) { dead = true; break; }
                 }
                 dead = __any_sync(0xffffffffu, dead);
-                bar_parity ^= 1u;
+                bar_parity ^= 1u << s;
+                BOA_T_MARK(5);
                 if (dead) {
                     if (lane == 0) atomicOr(p.status, kStatusCopyTimeout);
-                    break;
+                    return;
                 }
-                for (int r0 = 0; r0 < nb; r0 += 4) {
-                    const int j = r0 + gi;
-                    const bool act = j < nb;
-                    const uint8_t* row = stage + (size_t)(act ? j : 0) * p.rec_bytes;
-                    float acc = 0.0f;
-                    if (act) {
-                        if (VT == 0) {
-                            const float4* r4 = reinterpret_cast<const float4*>(row);
-#pragma unroll 4
-                            for (int c = g; c < p.nchunks; c += 8) acc = sq_acc4(acc, r4[c], qs[c]);
-                        } else {
-                            const uint4* r4 = reinterpret_cast<const uint4*>(row);
-                            for (int c = g; c < p.nchunks; c += 8) {
-                                const uint4 x = r4[c];
-                                acc = sq_acc_bytes(acc, x.x, qs[4 * c + 0]);
-                                acc = sq_acc_bytes(acc, x.y, qs[4 * c + 1]);
-                                acc = sq_acc_bytes(acc, x.z, qs[4 * c + 2]);
-                                acc = sq_acc_bytes(acc, x.w, qs[4 * c + 3]);
-                            }
-                        }
-                    }
-                    acc += __shfl_xor_sync(0xffffffffu, acc, 4);
-                    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
-                    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-                    bool viol = false;
-                    if (act && g < p.m) {
-                        const uint32_t av = *reinterpret_cast<const uint32_t*>(row + p.attr_off + 4 * g);
-                        if (my_float) {
-                            const float x = __uint_as_float(av);
-                            viol = !(x >= __int_as_float(my_lo) && x <= __int_as_float(my_hi));
-                        } else {
-                            const int32_t x = (int32_t)av;
-                            viol = x < my_lo || x > my_hi;
-                        }
-                    }
-                    const unsigned bal = __ballot_sync(0xffffffffu, viol);
-                    const uint32_t phi = __popc((bal >> (8 * gi)) & 0xFFu);
-                    if (act && g == 0) nk[b0 + j] = pack_key(phi, acc, cand[b0 + j]);
+                const uint8_t* src = stage + (size_t)s * half_rows * p.rec_bytes;
+                // eight rows per pass: every 8-lane group takes two, and the two partial-sum
+                // sets share one butterfly (lanes 0-3 of a group finish the first row, lanes
+                // 4-7 the second; the pairs added are the same as for a single row)
+                for (int r0 = 0; r0 < nb; r0 += 8) {
+                    const int j0 = r0 + gi, j1 = r0 + 4 + gi;
+                    const bool act0 = j0 < nb, act1 = j1 < nb;
+                    const uint8_t* row0 = src + (size_t)(act0 ? j0 : 0) * p.rec_bytes;
+                    const uint8_t* row1 = src + (size_t)(act1 ? j1 : 0) * p.rec_bytes;
+                    const float a0 = row_partial(row0);
+                    const float a1 = row_partial(row1);
+                    const bool hi4 = (lane & 4) != 0;
+                    float v = hi4 ? a1 : a0;
+                    const float w = hi4 ? a0 : a1;
+                    v += __shfl_xor_sync(0xffffffffu, w, 4);
+                    v += __shfl_xor_sync(0xffffffffu, v, 2);
+                    v += __shfl_xor_sync(0xffffffffu, v, 1);
+                    const bool v0 = act0 && g < p.m && violates(row0);
+                    const bool v1 = act1 && g < p.m && violates(row1);
+                    const unsigned bal0 = __ballot_sync(0xffffffffu, v0);
+                    const unsigned bal1 = __ballot_sync(0xffffffffu, v1);
+                    if (g == 0 && act0)
+                        nk[b0 + j0] = pack_key(__popc((bal0 >> (8 * gi)) & 0xFFu), v, cand[b0 + j0]);
+                    if (g == 4 && act1)
+                        nk[b0 + j1] = pack_key(__popc((bal1 >> (8 * gi)) & 0xFFu), v, cand[b0 + j1]);
                 }
-                __syncwarp();
+                __syncwarp();                     // every lane is done with slot s
+                BOA_T_MARK(6);
+                if (b + n_slots < nbatch) issue(b + n_slots);
             }
         };
 
         // Returns true when id was not in the table; records it either way.
         auto hash_test_and_set = [&](uint32_t id) -> bool {
-            const uint32_t h = (id * 0x9E3779B1u) >> hshift;
-            int empty = -1;
-#pragma unroll
-            for (int pr = 0; pr < 4; ++pr) {
-                const uint32_t s = (h + pr) & hmask;
-                const uint32_t v = hash[s];
-                if (v == id) return false;
-                if (v == kNoId && empty < 0) empty = (int)s;
-            }
-            hash[empty >= 0 ? (uint32_t)empty : h] = id;
+            const uint32_t h = (id * 0x9E3779B1u) & id_mask;
+            const uint32_t tag = h & tag_mask;
+            const uint32_t bucket = h >> p.tag_bits;
+            if (tag == 0xFFFFu) return true;              // would look like an empty way
+            const uint2 b = *reinterpret_cast<const uint2*>(hash + 4 * bucket);
+            const uint32_t w0 = b.x & 0xFFFFu, w1 = b.x >> 16, w2 = b.y & 0xFFFFu, w3 = b.y >> 16;
+            if (w0 == tag || w1 == tag || w2 == tag || w3 == tag) return false;
+            uint32_t way = (id ^ (id >> 7)) & 3u;
+            if (w3 == 0xFFFFu) way = 3u;
+            if (w2 == 0xFFFFu) way = 2u;
+            if (w1 == 0xFFFFu) way = 1u;
+            if (w0 == 0xFFFFu) way = 0u;
+            hash[4 * bucket + way] = (uint16_t)tag;
             return true;
+        };
+        // first unexpanded entry at or after `from` among the first `lim`, or -1
+        auto first_unexpanded = [&](int from, int lim) -> int {
+            for (int b0 = from & ~31; b0 < lim; b0 += 32) {
+                const int i = b0 + lane;
+                const bool un = (i >= from) && (i < lim) && ((pool[i] & 1ull) == 0ull);
+                const unsigned bal = __ballot_sync(0xffffffffu, un);
+                if (bal) return b0 + __ffs(bal) - 1;
+            }
+            return -1;
+        };
+        auto load_row_ids = [&](uint32_t id, uint32_t (&out)[RS]) {
+            const uint32_t* grow = p.graph + (size_t)id * p.R;
+#pragma unroll
+            for (int s = 0; s < RS; ++s) {
+                const int j = lane + 32 * s;
+                out[s] = (j < p.R) ? __ldg(grow + j) : kNoId;
+            }
         };
 
         // ---- pool: fresh from the entry point, or what a narrower phase left
@@ -379,32 +487,22 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
         }
 
         // ---- Algorithm 2 main loop
+        BOA_T_MARK(0);
+        int pos = dead ? -1 : first_unexpanded(0, n < p.L ? n : p.L);
+        uint32_t nb[RS];
+        bool have_row = false;         // nb[] already holds the adjacency row of pool[pos]
         while (!dead) {
-            // nearest unexpanded entry among the first L
-            const int lim = n < p.L ? n : p.L;
-            int pos = -1;
-            for (int b0 = cur & ~31; b0 < lim; b0 += 32) {
-                const int i = b0 + lane;
-                const bool un = (i >= cur) && (i < lim) && ((pool[i] & 1ull) == 0ull);
-                const unsigned bal = __ballot_sync(0xffffffffu, un);
-                if (bal) { pos = b0 + __ffs(bal) - 1; break; }
-            }
             if (pos < 0) break;                                   // converged
             if (n_exp >= p.max_expand) { capped = true; break; }
-            const uint32_t u_id = key_id(pool[pos]);
+            if (!have_row) load_row_ids(key_id(pool[pos]), nb);
             __syncwarp();
             if (lane == 0) pool[pos] |= 1ull;
             cur = pos + 1;
             n_exp++;
+            have_row = false;
+            BOA_T_MARK(1);
 
-            // adjacency row, drop ids scored before, compact the rest
-            uint32_t nb[RS];
-            const uint32_t* grow = p.graph + (size_t)u_id * p.R;
-#pragma unroll
-            for (int s = 0; s < RS; ++s) {
-                const int j = lane + 32 * s;
-                nb[s] = (j < p.R) ? __ldg(grow + j) : kNoId;
-            }
+            // drop ids scored before, compact the rest
             int cnt = 0;
 #pragma unroll
             for (int s = 0; s < RS; ++s) {
@@ -414,87 +512,155 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
                 cnt += __popc(bal);
             }
             __syncwarp();
-            if (cnt == 0) continue;
-            n_sc += cnt;
-
-            // gather + distance + range check (fused)
-            score(cnt);
-            if (dead) break;
-
-            // new keys that cannot enter a full pool are dropped right away; sort the rest
-            const uint64_t worst = (n == p.C) ? (pool[n - 1] >> 1) : (kKeyMax >> 1);
+            BOA_T_MARK(2);
+            int kept = 0, live = 0;
             uint64_t x[RS];
-            int live = 0;
-#pragma unroll
-            for (int s = 0; s < RS; ++s) {
-                const int j = lane + 32 * s;
-                x[s] = (j < cnt) ? nk[j] : kKeyMax;
-                if (x[s] != kKeyMax && (x[s] >> 1) >= worst) x[s] = kKeyMax;
-                live += __popc(__ballot_sync(0xffffffffu, x[s] != kKeyMax));
-            }
-            if (live == 0) continue;
-            if (live > 1) sort_keys<RS>(x, lane);
-            __syncwarp();
-
-            // rank of every new key in the pool; drop keys the pool already holds
-            int steps = 0;
-            while ((1 << steps) <= n) ++steps;
             bool keep[RS];
-            int kept = 0;
             int pos_new[RS];
+            if (cnt > 0) {
+                n_sc += cnt;
+                // gather + distance + range check (fused)
+                score(cnt);
+                if (dead) break;
+
+                // new keys that cannot enter a full pool are dropped right away
+                const uint64_t worst = (n == p.C) ? (pool[n - 1] >> 1) : (kKeyMax >> 1);
 #pragma unroll
-            for (int s = 0; s < RS; ++s) {
-                const uint64_t xs = x[s] >> 1;
-                const bool valid = x[s] != kKeyMax;
-                int lo_i = 0, hi_i = valid ? n : 0;
-                for (int it = 0; it < steps; ++it) {
-                    if (lo_i < hi_i) {
-                        const int mid = (lo_i + hi_i) >> 1;
-                        if ((pool[mid] >> 1) < xs) lo_i = mid + 1; else hi_i = mid;
-                    }
+                for (int s = 0; s < RS; ++s) {
+                    const int j = lane + 32 * s;
+                    x[s] = (j < cnt) ? nk[j] : kKeyMax;
+                    if (x[s] != kKeyMax && (x[s] >> 1) >= worst) x[s] = kKeyMax;
+                    live += __popc(__ballot_sync(0xffffffffu, x[s] != kKeyMax));
                 }
-                const bool dup = valid && (lo_i < n) && ((pool[lo_i] >> 1) == xs);
-                const bool nd = valid && !dup;
-                const unsigned bal = __ballot_sync(0xffffffffu, nd);
-                const int pidx = kept + __popc(bal & lt_mask);
-                pos_new[s] = lo_i + pidx;
-                keep[s] = nd && (pos_new[s] < p.C);
-                const unsigned kb = __ballot_sync(0xffffffffu, keep[s]);
-                if (keep[s]) nr[pidx] = (uint32_t)lo_i;
-                kept += __popc(kb);
             }
-            __syncwarp();
-            if (kept == 0) continue;
+            if (live > 0) {
+                // sort the survivors: by counting for a handful, bitonic otherwise
+                if (RS == 1 && live <= 8) {
+                    const unsigned m0 = __ballot_sync(0xffffffffu, x[0] != kKeyMax);
+                    int r = 0;
+                    for (unsigned mm = m0; mm; mm &= mm - 1) {
+                        const uint64_t y = __shfl_sync(0xffffffffu, x[0], __ffs(mm) - 1);
+                        r += (y < x[0]) ? 1 : 0;
+                    }
+                    __syncwarp();
+                    if (x[0] != kKeyMax) nk[r] = x[0];
+                    __syncwarp();
+                    x[0] = (lane < live) ? nk[lane] : kKeyMax;
+                } else if (live > 1) {
+                    sort_keys<RS>(x, lane);
+                }
+                BOA_T_MARK(7);
+
+                // rank of every new key in the pool (4-ary search); drop keys it already holds
+#pragma unroll
+                for (int s = 0; s < RS; ++s) {
+                    const uint64_t xs = x[s] >> 1;
+                    const bool valid = x[s] != kKeyMax;
+                    int lo_i = 0, hi_i = valid ? n : 0;
+                    while (__any_sync(0xffffffffu, lo_i < hi_i)) {
+                        if (lo_i < hi_i) {
+                            const int len = hi_i - lo_i;
+                            const int q1 = lo_i + (len >> 2), q2 = lo_i + (len >> 1);
+                            const int q3 = lo_i + ((3 * len) >> 2);
+                            const bool c1 = (pool[q1] >> 1) < xs;
+                            const bool c2 = (pool[q2] >> 1) < xs;
+                            const bool c3 = (pool[q3] >> 1) < xs;
+                            if (c3) lo_i = q3 + 1;
+                            else if (c2) { lo_i = q2 + 1; hi_i = q3; }
+                            else if (c1) { lo_i = q1 + 1; hi_i = q2; }
+                            else hi_i = q1;
+                        }
+                    }
+                    const bool dup = valid && (lo_i < n) && ((pool[lo_i] >> 1) == xs);
+                    const bool nd = valid && !dup;
+                    const unsigned bal = __ballot_sync(0xffffffffu, nd);
+                    const int pidx = kept + __popc(bal & lt_mask);
+                    pos_new[s] = lo_i + pidx;
+                    keep[s] = nd && (pos_new[s] < p.C);
+                    const unsigned kb = __ballot_sync(0xffffffffu, keep[s]);
+                    if (keep[s]) nr[pidx] = (uint32_t)lo_i;
+                    kept += __popc(kb);
+                }
+                __syncwarp();
+                BOA_T_MARK(8);
+            }
+            if (kept == 0) {
+                // pool unchanged: the next node is simply the next unexpanded entry
+                pos = first_unexpanded(cur, n < p.L ? n : p.L);
+                continue;
+            }
             const int rmin = (int)nr[0];
 
-            // shift pool entries right by the number of new keys ranked at or before them
-            for (int b0 = (n - 1) & ~31; b0 >= (rmin & ~31); b0 -= 32) {
-                const int i = b0 + lane;
-                uint64_t e = 0;
-                int sh = 0;
-                if (i < n && i >= rmin) {
-                    e = pool[i];
-                    if (kept <= 8) {
-                        for (int j = 0; j < kept; ++j) sh += ((int)nr[j] <= i) ? 1 : 0;
-                    } else {
-                        int a = 0, b = kept;             // upper_bound(nr, i)
-                        while (a < b) {
-                            const int mid = (a + b) >> 1;
-                            if ((int)nr[mid] <= i) a = mid + 1; else b = mid;
-                        }
-                        sh = a;
+            // ---- which node is expanded next?  Decide on the pool as it is, translate the
+            // position, and start loading that node's adjacency row before the merge.
+            {
+                const int pos_old = first_unexpanded(cur, n < p.L ? n : p.L);
+                int pos_old_new = -1;
+                if (pos_old >= 0) {
+                    int sh = 0;
+                    for (int j = 0; j < kept; ++j) sh += ((int)nr[j] <= pos_old) ? 1 : 0;
+                    pos_old_new = pos_old + sh;
+                }
+                const int n_new = (n + kept < p.C) ? n + kept : p.C;
+                const int lim_new = n_new < p.L ? n_new : p.L;
+                int next_pos;
+                uint32_t next_id;
+                if (pos_old_new < 0 || rmin < pos_old_new) {
+                    next_pos = rmin;                         // the smallest new key comes first
+                    uint64_t first_new = 0;
+#pragma unroll
+                    for (int s = RS - 1; s >= 0; --s) {
+                        const unsigned kb = __ballot_sync(0xffffffffu, keep[s]);
+                        if (kb) first_new = __shfl_sync(0xffffffffu, x[s], __ffs(kb) - 1);
+                    }
+                    next_id = key_id(first_new);
+                } else {
+                    next_pos = pos_old_new;
+                    next_id = key_id(pool[pos_old]);
+                }
+                if (next_pos >= lim_new) next_pos = -1;
+                pos = next_pos;
+                if (pos >= 0 && n_exp < p.max_expand) {
+                    load_row_ids(next_id, nb);
+                    have_row = true;
+                }
+            }
+
+            // ---- merge.  The pool entries between two consecutive new keys all move up by
+            // the same amount: segment j = [rank_j, rank_{j+1}) moves by j+1.  Segments go
+            // top first, each in 32-entry chunks from its top end; the next chunk is read
+            // before the current one is written (its slots are never a write target).
+            {
+                for (int j = kept - 1; j >= 0; --j) {
+                    const int a = (int)nr[j];
+                    const int bnd = (j == kept - 1) ? n : (int)nr[j + 1];
+                    if (bnd <= a) continue;
+                    const int sft = j + 1;
+                    int lo_c = (bnd - 32 > a) ? bnd - 32 : a;
+                    int i = lo_c + lane;
+                    bool v = i < bnd;
+                    uint64_t e = v ? pool[i] : 0ull;
+                    for (;;) {
+                        __syncwarp();
+                        const int hi2 = lo_c;
+                        const int lo2 = (hi2 - 32 > a) ? hi2 - 32 : a;
+                        const int i2 = lo2 + lane;
+                        const bool v2 = (hi2 > a) && (i2 < hi2);
+                        const uint64_t e2 = v2 ? pool[i2] : 0ull;
+                        if (v && i + sft < p.C) pool[i + sft] = e;
+                        if (hi2 <= a) break;
+                        lo_c = lo2; i = i2; v = v2; e = e2;
                     }
                 }
                 __syncwarp();
-                if (sh > 0 && i + sh < p.C) pool[i + sh] = e;
+#pragma unroll
+                for (int s = 0; s < RS; ++s)
+                    if (keep[s]) pool[pos_new[s]] = x[s];
+                n = (n + kept < p.C) ? n + kept : p.C;
+                if (rmin < cur) cur = rmin;
                 __syncwarp();
             }
-#pragma unroll
-            for (int s = 0; s < RS; ++s)
-                if (keep[s]) pool[pos_new[s]] = x[s];
-            n = (n + kept < p.C) ? n + kept : p.C;
-            if (rmin < cur) cur = rmin;
-            __syncwarp();
+            BOA_T_MARK(9);
         }
         if (dead) break;
 
@@ -552,7 +718,9 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
             }
         }
         __syncwarp();
+        BOA_T_MARK(10);
     }
+    BOA_T_FLUSH(p.timers);
 }
 
 }  // namespace boa
