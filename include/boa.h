@@ -28,7 +28,8 @@ enum {
     BOA_EINVAL = -1, /* bad argument (null, range, alignment, unsupported shape) */
     BOA_ENOMEM = -2, /* device or host allocation failed                         */
     BOA_ECUDA = -3,  /* a CUDA call failed; boa_last_cuda_error() has its code   */
-    BOA_EGRAPH = -4  /* the graph names a node id >= N                           */
+    BOA_EGRAPH = -4, /* the graph names a node id >= N                           */
+    BOA_ETOOBIG = -5 /* boa_search_noalloc: Q or Lmax beyond its fixed scratch   */
 };
 
 #define BOA_NO_ID 0xFFFFFFFFu /* "no edge" in graph rows, "no result" in out_ids */
@@ -108,6 +109,39 @@ int64_t boa_index_entry(const boa_index* index);
  */
 int boa_search(boa_index* index, const float* queries, int64_t Q, const void* lo, const void* hi,
                int k, int L0, int Lmax, uint32_t* out_ids, float* out_dists, void* stream);
+
+/*
+ * boa_search for callers that must not allocate device memory.  (The paper has no
+ * counterpart: this is a service of the library, not a step of the method.)
+ *
+ * Who needs it: a serving loop that has handed all device memory to its own pools and
+ * runs with allocation forbidden; a latency-critical caller that cannot afford the
+ * device-wide synchronisation a cudaMalloc or cudaFree may imply; code running inside a
+ * region where the CUDA runtime refuses allocation.  boa_search grows index-owned
+ * scratch with cudaMalloc the first time a batch is larger than any before; this
+ * variant never does.  Its scratch (survivor lists, counters, per-query statistics and
+ * the pools carried between phases) is a fixed array of about 4.1 MiB inside the
+ * library image, so every GPU that loads the library holds that much until the process
+ * exits.
+ *
+ * Same arguments, outputs and asynchronous behaviour as boa_search, same results, with
+ * these differences:
+ *   - Q <= BOA_NOALLOC_MAX_Q and Lmax <= BOA_NOALLOC_MAX_WIDTH, else BOA_ETOOBIG and
+ *     nothing is enqueued;
+ *   - it calls no cudaMalloc, cudaFree or other allocating routine; the first call on a
+ *     device looks up the device address of the fixed array (one cudaGetSymbolAddress),
+ *     so make that first call outside any stream capture;
+ *   - all calls on one device share the one array, whatever the index: it keeps the
+ *     previous call's contents (what must start at zero is cleared on `stream` at the
+ *     start of each call), and two calls whose GPU work overlaps in time race on it --
+ *     run them one after the other, on one stream or ordered by events;
+ *   - boa_get_stats and boa_get_phase_counts do not cover this call.
+ */
+#define BOA_NOALLOC_MAX_Q 1024
+#define BOA_NOALLOC_MAX_WIDTH 512
+int boa_search_noalloc(boa_index* index, const float* queries, int64_t Q, const void* lo,
+                       const void* hi, int k, int L0, int Lmax, uint32_t* out_ids, float* out_dists,
+                       void* stream);
 
 /* Set one parameter (keys above).  BOA_EINVAL for an unknown key or a value out of range. */
 int boa_set_param(boa_index* index, int key, double value);

@@ -55,6 +55,8 @@ def load_library():
     L.boa_index_entry.argtypes = [vp]
     L.boa_search.restype = i32
     L.boa_search.argtypes = [vp, vp, i64, vp, vp, i32, i32, i32, vp, vp, vp]
+    L.boa_search_noalloc.restype = i32
+    L.boa_search_noalloc.argtypes = [vp, vp, i64, vp, vp, i32, i32, i32, vp, vp, vp]
     L.boa_set_param.restype = i32
     L.boa_set_param.argtypes = [vp, i32, C.c_double]
     L.boa_set_schedule.restype = i32
@@ -161,6 +163,23 @@ class BoaIndex:
                                     L0, Lmax, out_ids.data_ptr(), out_dists.data_ptr(),
                                     _stream_ptr(stream)), "boa_search")
         self._last_Q = Q
+        return out_ids, out_dists
+
+    def search_noalloc(self, queries: torch.Tensor, lo: torch.Tensor, hi: torch.Tensor, k: int,
+                       L0: int, Lmax: int, out_ids: torch.Tensor, out_dists: torch.Tensor,
+                       stream: Optional[torch.cuda.Stream] = None):
+        """boa_search_noalloc: for callers that may not allocate device memory.  The caller
+        passes every buffer, outputs included; the library's scratch is a fixed array in its
+        own image (batches up to 1024 queries, widths up to 512).  Calls that overlap on the
+        GPU race on that array, so keep them ordered."""
+        for name, t in (("queries", queries), ("lo", lo), ("hi", hi), ("out_ids", out_ids),
+                        ("out_dists", out_dists)):
+            if not (t.is_cuda and t.is_contiguous()):
+                raise ValueError(f"{name} must be a contiguous CUDA tensor")
+        _check(self._lib.boa_search_noalloc(self._h, queries.data_ptr(), queries.shape[0],
+                                            lo.data_ptr(), hi.data_ptr(), k, L0, Lmax,
+                                            out_ids.data_ptr(), out_dists.data_ptr(),
+                                            _stream_ptr(stream)), "boa_search_noalloc")
         return out_ids, out_dists
 
     def stats(self, stream: Optional[torch.cuda.Stream] = None):

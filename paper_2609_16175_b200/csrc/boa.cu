@@ -189,6 +189,39 @@ constexpr int kCntTicket = 48;                        // one per launch
 constexpr int kMaxLaunches = 128;
 constexpr int kCntWords = kCntTicket + kMaxLaunches;   // 176: the 64-bit words after it stay aligned
 
+// ---- scratch of boa_search_noalloc: lives in the library image, never allocated
+constexpr int64_t kNoAllocMaxQ = BOA_NOALLOC_MAX_Q;
+constexpr int kNoAllocMaxWidth = BOA_NOALLOC_MAX_WIDTH;
+constexpr size_t kNaCounters = 0;                                             // 1 KiB
+constexpr size_t kNaLists = 1024;                                             // [phases][Q] u32
+constexpr size_t kNaStats = kNaLists + (size_t)BOA_MAX_PHASES * kNoAllocMaxQ * 4;
+constexpr size_t kNaSpillSize = kNaStats + (size_t)4 * kNoAllocMaxQ * 4;
+constexpr size_t kNaSpill = kNaSpillSize + (size_t)kNoAllocMaxQ * 4;
+constexpr size_t kNaBytes = kNaSpill + (size_t)kNoAllocMaxQ * kNoAllocMaxWidth * 8;
+static_assert(kCntWords * 4 + 12 * 8 <= 1024, "counter block must fit its slot");
+static_assert(kNaSpill % 256 == 0 && kNaStats % 256 == 0, "sub-buffers stay aligned");
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaBytes];
+
+// In host code `g_noalloc_scratch` is only a handle for the runtime, not an address a
+// kernel can use: the device address is asked for once per device and kept here.
+constexpr int kMaxDevices = 64;
+unsigned char* g_noalloc_ptr[kMaxDevices] = {nullptr};
+
+int noalloc_scratch(unsigned char** out)
+{
+    int dev = 0;
+    BOA_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return BOA_EINVAL;
+    if (!g_noalloc_ptr[dev]) {
+        void* ptr = nullptr;
+        BOA_CUDA(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+        g_noalloc_ptr[dev] = static_cast<unsigned char*>(ptr);
+    }
+    *out = g_noalloc_ptr[dev];
+    return BOA_OK;
+}
+
 typedef void (*SearchKernel)(const boa::SearchParams);
 
 struct KernelChoice {
@@ -365,6 +398,7 @@ const char* boa_strerror(int status)
         case BOA_ENOMEM: return "out of memory";
         case BOA_ECUDA: return "CUDA call failed";
         case BOA_EGRAPH: return "graph names a node id outside the index";
+        case BOA_ETOOBIG: return "batch or beamwidth beyond the fixed scratch of boa_search_noalloc";
         default: return "unknown status";
     }
 }
@@ -688,6 +722,36 @@ int boa_get_phase_counts(boa_index* ix, int64_t* active, int n, int* n_phases, v
 }
 
 int boa_last_launch_count(const boa_index* ix) { return ix ? ix->last_launches : 0; }
+
+int boa_search_noalloc(boa_index* ix, const float* queries, int64_t Q, const void* lo, const void* hi,
+                       int k, int L0, int Lmax, uint32_t* out_ids, float* out_dists, void* stream)
+{
+    if (!ix) return BOA_EINVAL;
+    if (Q > kNoAllocMaxQ || Lmax > kNoAllocMaxWidth) return BOA_ETOOBIG;
+    unsigned char* base = nullptr;
+    const int rc0 = noalloc_scratch(&base);
+    if (rc0 != BOA_OK) return rc0;
+    // Point the index at the fixed buffer for the length of this call, run the ordinary
+    // driver (which then finds its scratch large enough and allocates nothing), and put
+    // the index's own buffers back.
+    struct Saved {
+        uint32_t *lists, *counters; int32_t *stats, *spill_size; uint64_t* spill;
+        int64_t ws_Q; int ws_spill;
+    } sv = {ix->lists, ix->counters, ix->stats, ix->spill_size, ix->spill, ix->ws_Q, ix->ws_spill};
+    ix->counters = reinterpret_cast<uint32_t*>(base + kNaCounters);
+    ix->lists = reinterpret_cast<uint32_t*>(base + kNaLists);
+    ix->stats = reinterpret_cast<int32_t*>(base + kNaStats);
+    ix->spill_size = reinterpret_cast<int32_t*>(base + kNaSpillSize);
+    ix->spill = reinterpret_cast<uint64_t*>(base + kNaSpill);
+    ix->ws_Q = kNoAllocMaxQ;
+    ix->ws_spill = kNoAllocMaxWidth;
+    const int rc = boa_search(ix, queries, Q, lo, hi, k, L0, Lmax, out_ids, out_dists, stream);
+    ix->lists = sv.lists; ix->counters = sv.counters; ix->stats = sv.stats;
+    ix->spill_size = sv.spill_size; ix->spill = sv.spill; ix->ws_Q = sv.ws_Q; ix->ws_spill = sv.ws_spill;
+    ix->last_Q = 0;            // the per-query statistics of this call are not kept
+    ix->last_phases = 0;
+    return rc;
+}
 
 #ifdef BOA_SECTION_TIMERS
 // Debug builds only: cycles per kernel section, summed over warps (12 values, HOST array).
