@@ -136,6 +136,21 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(local_ms: float, device, world: int) -> float:
+    """Time of the slowest rank (all ranks get it)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(queries_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Queries per second of the whole job: every rank searched its own batch."""
+    return world * queries_per_rank / (ms_per_step / 1e3)
+
+
 def measured_peak_gbs():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -293,11 +308,8 @@ def main():
     step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
     clocks = sampler.stop() if rank == 0 else None
     launches = ix.last_launch_count * args.steps
-    tmax = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-    ms_per_step = float(tmax.item()) / args.steps
-    value = world * Q / (ms_per_step / 1e3)
+    ms_per_step = max_over_ranks(total_ms, dev, world) / args.steps
+    value = whole_job_value(Q, world, ms_per_step)
 
     # ---- statistics of the batch (outside the timed region)
     st = {kk: v.cpu().numpy() for kk, v in ix.stats().items()}
@@ -340,10 +352,7 @@ def main():
     e1.record()
     torch.cuda.synchronize()
     barrier()
-    e2e_ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
-    e2e_value = world * Q / (float(e2e_ms.item()) / args.steps / 1e3)
+    e2e_value = whole_job_value(Q, world, max_over_ranks(e0.elapsed_time(e1), dev, world) / args.steps)
     h2d = hq.numel() * 4 + hlo.numel() * 4 + hhi.numel() * 4
     d2h = h_ids.numel() * 4 + h_d2.numel() * 4
     assert (h_ids.numpy().view(np.uint32) == ids_np).all()

@@ -230,35 +230,41 @@ struct KernelChoice {
 };
 
 template <int VT, int CPL>
-KernelChoice pick_rs(int R)
+KernelChoice pick_rs(int R, bool exact)
 {
-    if (R <= 32) return {boa::boa_search_kernel<VT, 1, CPL>, 1};
-    return {boa::boa_search_kernel<VT, 2, CPL>, 2};
+    if (R <= 32) {
+        if (exact) return {boa::boa_search_kernel<VT, 1, CPL, (CPL > 0)>, 1};
+        return {boa::boa_search_kernel<VT, 1, CPL, false>, 1};
+    }
+    if (exact) return {boa::boa_search_kernel<VT, 2, CPL, (CPL > 0)>, 2};
+    return {boa::boa_search_kernel<VT, 2, CPL, false>, 2};
 }
 
 KernelChoice pick_kernel(const boa_index* ix)
 {
     const int cpl = (ix->nchunks + 7) / 8;      // 16-byte chunks per lane of an 8-lane group
+    const bool exact = ix->nchunks == 8 * cpl;
     if (ix->vec_dtype == BOA_F32) {
         switch (cpl) {
-            case 1: return pick_rs<0, 1>(ix->R);
-            case 2: return pick_rs<0, 2>(ix->R);
-            case 3: return pick_rs<0, 3>(ix->R);
-            case 4: return pick_rs<0, 4>(ix->R);
-            default: return pick_rs<0, 0>(ix->R);
+            case 1: return pick_rs<0, 1>(ix->R, exact);
+            case 2: return pick_rs<0, 2>(ix->R, exact);
+            case 3: return pick_rs<0, 3>(ix->R, exact);
+            case 4: return pick_rs<0, 4>(ix->R, exact);
+            default: return pick_rs<0, 0>(ix->R, false);
         }
     }
     switch (cpl) {
-        case 1: return pick_rs<1, 1>(ix->R);
-        case 2: return pick_rs<1, 2>(ix->R);
-        default: return pick_rs<1, 0>(ix->R);
+        case 1: return pick_rs<1, 1>(ix->R, exact);
+        case 2: return pick_rs<1, 2>(ix->R, exact);
+        default: return pick_rs<1, 0>(ix->R, false);
     }
 }
 
 int choose_hash_log2(const boa_index* ix, int L)
 {
     if (ix->hash_log2) return ix->hash_log2;
-    int lg = (L <= 32) ? 11 : 12;     // 16-bit entries: 4 KB / 8 KB per query
+    (void)L;
+    int lg = 11;                      // 2048 16-bit entries: 4 KB per query
     int id_bits = 1;
     while (((int64_t)1 << id_bits) < ix->N) ++id_bits;
     if (id_bits - (lg - 2) > 16) lg = id_bits - 14;     // tags must fit 16 bits
@@ -267,7 +273,8 @@ int choose_hash_log2(const boa_index* ix, int L)
 
 int choose_stage_rows(const boa_index* ix, int rs)
 {
-    int rows = ix->stage_rows ? ix->stage_rows : 8192 / ix->rec_bytes;
+    // default: one slot of eight rows (a full scoring pass), fewer for very long rows
+    int rows = ix->stage_rows ? ix->stage_rows : (8 * ix->rec_bytes <= 16384 ? 8 : 16384 / ix->rec_bytes);
     if (rows > 32 * rs) rows = 32 * rs;
     if (rows >= 16) rows &= ~1;       // two ring slots of equal size
     if (rows < 1) rows = 1;

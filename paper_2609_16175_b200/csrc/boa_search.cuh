@@ -10,11 +10,13 @@
 // lambda -> infinity reading of the paper's score dist + lambda*phi.
 //
 // Neighbour records (vector + attribute cells, one contiguous 32-byte-aligned row
-// each) are fetched with one bulk asynchronous copy (cp.async.bulk, the TMA engine)
-// per row into a two-slot ring in shared memory; one transaction barrier per slot
-// tells the warp when the bytes have landed.  No register holds data in flight, so
-// one warp keeps up to `stage_rows` whole rows in flight while it scores the rows
-// that have already arrived.
+// each) are fetched with 16-byte asynchronous copies (cp.async, global -> shared, L2
+// only) into a ring of one or two slots in shared memory: the 32 lanes copy 512
+// consecutive bytes of a row per instruction, one commit group per slot.  No register
+// holds data in flight, so one warp keeps up to `stage_rows` whole rows in flight
+// while it scores the rows that have already arrived.  (A bulk copy per row through
+// the TMA engine was measured first: it needs one uniform-datapath instruction
+// sequence per row, about ten instructions each, which made the kernel issue-bound.)
 //
 // The table of recently scored ids stores 16-bit tags in 4-way buckets.  An id is
 // first mapped by an odd multiplier modulo 2^id_bits (a bijection); the high bits
@@ -37,10 +39,8 @@ namespace boa {
 constexpr uint32_t kNoId = 0xFFFFFFFFu;
 constexpr int kThreads = 32;           // one warp per CTA
 constexpr uint64_t kKeyMax = ~0ull;
-constexpr uint32_t kWaitLimit = 1u << 20;   // bounded wait on a transaction barrier (tries)
-constexpr uint32_t kWaitHintNs = 2000u;     // each try may block this long inside the instruction
 
-enum : uint32_t { kStatusCopyTimeout = 1u };
+enum : uint32_t { kStatusCopyTimeout = 1u };   // reserved: no wait in the kernel can time out
 
 // Optional per-section cycle counters (build with -DBOA_SECTION_TIMERS; off in the product).
 #ifdef BOA_SECTION_TIMERS
@@ -126,43 +126,14 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p)
 {
     return (uint32_t)__cvta_generic_to_shared(p);
 }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count)
+// 16 bytes, global -> shared, cached in L2 only.
+__device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src)
 {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
 }
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
-                 "r"(bytes)
-                 : "memory");
-}
-// Blocks for at most about `hint_ns` inside the instruction, then reports.
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, uint32_t hint_ns)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
-        : "memory");
-    return ok != 0;
-}
-// One row, global -> shared, completion counted in bytes on `bar`.  No multicast.
-__device__ __forceinline__ void bulk_load_row(void* dst, const void* src, uint32_t bytes, uint64_t* bar)
-{
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-            smem_u32(dst)),
-        "l"(src), "r"(bytes), "r"(smem_u32(bar))
-        : "memory");
-}
-__device__ __forceinline__ void fence_async_proxy()
-{
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 __device__ __forceinline__ float sq_acc4(float acc, float4 x, float4 q)
 {
@@ -238,8 +209,9 @@ __host__ __device__ inline WarpSmem warp_smem_layout(int C, int hash_log2, int D
 // VT: 0 = float vectors, 1 = uint8 vectors.  RS: adjacency slots per lane (1: R <= 32,
 // 2: R <= 64).  CPL: 16-byte chunks of a row per lane of an 8-lane group when that is
 // at most 4 (the lane then keeps its slices of the query in registers and the chunk
-// loop is unrolled); 0 = any length, query slices read from shared memory.
-template <int VT, int RS, int CPL>
+// loop is unrolled); 0 = any length, query slices read from shared memory.  EXACT: the
+// row has exactly 8*CPL chunks, so no lane ever has a chunk missing.
+template <int VT, int RS, int CPL, bool EXACT>
 __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams p)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -258,7 +230,6 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
     uint32_t* cand = reinterpret_cast<uint32_t*>(smem_raw + lay.cand_off);
     uint16_t* hash = reinterpret_cast<uint16_t*>(smem_raw + lay.hash_off);
     float4* qs = reinterpret_cast<float4*>(smem_raw + lay.q_off);
-    uint64_t* bar = reinterpret_cast<uint64_t*>(smem_raw + lay.bar_off);   // bar[0], bar[1]
 
     const uint32_t id_mask = (p.id_bits >= 32) ? 0xFFFFFFFFu : ((1u << p.id_bits) - 1u);
     const uint32_t tag_mask = (1u << p.tag_bits) - 1u;
@@ -274,13 +245,13 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
     }
     const uint32_t n_work = w_end > w_begin ? w_end - w_begin : 0u;
 
-    if (lane == 0) { mbar_init(bar, 1u); mbar_init(bar + 1, 1u); }
-    __syncwarp();
-    uint32_t bar_parity = 0;       // bit s: parity the next wait on slot s expects
     BOA_T_DECL;
-    bool dead = false;             // a copy never completed: stop taking work
+    const uint32_t stage_s = smem_u32(stage);
+    const int pieces = p.rec_bytes >> 4;            // 16-byte pieces of one record
+    const int full = pieces >> 5;                   // 512-byte spans of a record
+    const int tail = pieces & 31;                   // pieces after the last full span
 
-    while (!dead) {
+    for (;;) {
         uint32_t t = 0;
         if (lane == 0) t = atomicAdd(p.ticket, 1u);
         t = __shfl_sync(0xffffffffu, t, 0);
@@ -313,51 +284,7 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
             }
         }
 
-        // squared distance contribution of this lane to one staged row
-        auto row_partial = [&](const uint8_t* row) -> float {
-            float acc = 0.0f;
-            if (CPL > 0) {
-#pragma unroll
-                for (int i = 0; i < (CPL > 0 ? CPL : 1); ++i) {
-                    const int c = g + 8 * i;
-                    if (c < p.nchunks) {
-                        if (VT == 0) {
-                            acc = sq_acc4(acc, reinterpret_cast<const float4*>(row)[c], qreg[i]);
-                        } else {
-                            const uint4 x = reinterpret_cast<const uint4*>(row)[c];
-                            acc = sq_acc_bytes(acc, x.x, qreg[4 * i + 0]);
-                            acc = sq_acc_bytes(acc, x.y, qreg[4 * i + 1]);
-                            acc = sq_acc_bytes(acc, x.z, qreg[4 * i + 2]);
-                            acc = sq_acc_bytes(acc, x.w, qreg[4 * i + 3]);
-                        }
-                    }
-                }
-            } else {
-                for (int c = g; c < p.nchunks; c += 8) {
-                    if (VT == 0) {
-                        acc = sq_acc4(acc, reinterpret_cast<const float4*>(row)[c], qs[c]);
-                    } else {
-                        const uint4 x = reinterpret_cast<const uint4*>(row)[c];
-                        acc = sq_acc_bytes(acc, x.x, qs[4 * c + 0]);
-                        acc = sq_acc_bytes(acc, x.y, qs[4 * c + 1]);
-                        acc = sq_acc_bytes(acc, x.z, qs[4 * c + 2]);
-                        acc = sq_acc_bytes(acc, x.w, qs[4 * c + 3]);
-                    }
-                }
-            }
-            return acc;
-        };
-        auto violates = [&](const uint8_t* row) -> bool {
-            const uint32_t av = *reinterpret_cast<const uint32_t*>(row + p.attr_off + 4 * g);
-            if (my_float) {
-                const float x = __uint_as_float(av);
-                return !(x >= __int_as_float(my_lo) && x <= __int_as_float(my_hi));
-            }
-            const int32_t x = (int32_t)av;
-            return x < my_lo || x > my_hi;
-        };
-
-        // Scores cand[0..cnt): fetch the records through the two-slot ring, then
+        // Scores cand[0..cnt): fetch the records through the staging ring, then
         // distance + violated predicates -> nk[0..cnt).
         auto score = [&](int cnt) {
             const int nbatch = (cnt + half_rows - 1) / half_rows;
@@ -365,13 +292,21 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
                 const int s = (n_slots == 2) ? (b & 1) : 0;
                 const int b0 = b * half_rows;
                 const int nb = (cnt - b0 < half_rows) ? cnt - b0 : half_rows;
-                if (lane == 0) mbar_expect_tx(bar + s, (uint32_t)(nb * p.rec_bytes));
-                uint8_t* dst = stage + (size_t)s * half_rows * p.rec_bytes;
-                for (int j = lane; j < nb; j += 32) {
-                    const uint32_t n = cand[b0 + j];
-                    bulk_load_row(dst + (size_t)j * p.rec_bytes, p.rec + (size_t)n * p.rec_stride,
-                                  (uint32_t)p.rec_bytes, bar + s);
+                const uint32_t dst0 = stage_s + (uint32_t)(s * half_rows * p.rec_bytes);
+                for (int j = 0; j < nb; ++j) {
+                    const uint8_t* src = p.rec + (size_t)cand[b0 + j] * p.rec_stride + 16 * lane;
+                    const uint32_t dst = dst0 + (uint32_t)(j * p.rec_bytes) + 16u * lane;
+                    for (int f = 0; f < full; ++f) cp_async16(dst + 512u * f, src + 512 * f);
                 }
+                if (tail) {
+                    // the pieces after the last full span, for all rows of the batch at once
+                    for (int t = lane; t < nb * tail; t += 32) {
+                        const int j = t / tail, pc = 32 * full + t % tail;
+                        cp_async16(dst0 + (uint32_t)(j * p.rec_bytes + 16 * pc),
+                                   p.rec + (size_t)cand[b0 + j] * p.rec_stride + 16 * pc);
+                    }
+                }
+                cp_async_commit();
             };
             BOA_T_MARK(3);
             issue(0);
@@ -381,17 +316,10 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
                 const int s = (n_slots == 2) ? (b & 1) : 0;
                 const int b0 = b * half_rows;
                 const int nb = (cnt - b0 < half_rows) ? cnt - b0 : half_rows;
-                uint32_t spins = 0;
-                while (!mbar_try_wait(bar + s, (bar_parity >> s) & 1u, kWaitHintNs)) {
-                    if (++spins > kWaitLimit) { dead = true; break; }
-                }
-                dead = __any_sync(0xffffffffu, dead);
-                bar_parity ^= 1u << s;
+                // the newest group may stay in flight only if it belongs to the batch after this one
+                if (n_slots == 2 && b + 1 < nbatch) cp_async_wait<1>(); else cp_async_wait<0>();
+                __syncwarp();
                 BOA_T_MARK(5);
-                if (dead) {
-                    if (lane == 0) atomicOr(p.status, kStatusCopyTimeout);
-                    return;
-                }
                 const uint8_t* src = stage + (size_t)s * half_rows * p.rec_bytes;
                 // eight rows per pass: every 8-lane group takes two, and the two partial-sum
                 // sets share one butterfly (lanes 0-3 of a group finish the first row, lanes
@@ -399,24 +327,76 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
                 for (int r0 = 0; r0 < nb; r0 += 8) {
                     const int j0 = r0 + gi, j1 = r0 + 4 + gi;
                     const bool act0 = j0 < nb, act1 = j1 < nb;
-                    const uint8_t* row0 = src + (size_t)(act0 ? j0 : 0) * p.rec_bytes;
-                    const uint8_t* row1 = src + (size_t)(act1 ? j1 : 0) * p.rec_bytes;
-                    const float a0 = row_partial(row0);
-                    const float a1 = row_partial(row1);
+                    const uint8_t* row0 = src + (act0 ? j0 : 0) * p.rec_bytes;
+                    const uint8_t* row1 = src + (act1 ? j1 : 0) * p.rec_bytes;
+                    float a0 = 0.0f, a1 = 0.0f;
+                    if (CPL > 0) {
+#pragma unroll
+                        for (int i = 0; i < (CPL > 0 ? CPL : 1); ++i) {
+                            const int c = g + 8 * i;
+                            if (EXACT || c < p.nchunks) {
+                                if (VT == 0) {
+                                    a0 = sq_acc4(a0, reinterpret_cast<const float4*>(row0)[c], qreg[i]);
+                                    a1 = sq_acc4(a1, reinterpret_cast<const float4*>(row1)[c], qreg[i]);
+                                } else {
+                                    const uint4 x0 = reinterpret_cast<const uint4*>(row0)[c];
+                                    const uint4 x1 = reinterpret_cast<const uint4*>(row1)[c];
+                                    a0 = sq_acc_bytes(a0, x0.x, qreg[4 * i + 0]);
+                                    a1 = sq_acc_bytes(a1, x1.x, qreg[4 * i + 0]);
+                                    a0 = sq_acc_bytes(a0, x0.y, qreg[4 * i + 1]);
+                                    a1 = sq_acc_bytes(a1, x1.y, qreg[4 * i + 1]);
+                                    a0 = sq_acc_bytes(a0, x0.z, qreg[4 * i + 2]);
+                                    a1 = sq_acc_bytes(a1, x1.z, qreg[4 * i + 2]);
+                                    a0 = sq_acc_bytes(a0, x0.w, qreg[4 * i + 3]);
+                                    a1 = sq_acc_bytes(a1, x1.w, qreg[4 * i + 3]);
+                                }
+                            }
+                        }
+                    } else {
+                        for (int c = g; c < p.nchunks; c += 8) {
+                            if (VT == 0) {
+                                const float4 qq = qs[c];
+                                a0 = sq_acc4(a0, reinterpret_cast<const float4*>(row0)[c], qq);
+                                a1 = sq_acc4(a1, reinterpret_cast<const float4*>(row1)[c], qq);
+                            } else {
+                                const uint4 x0 = reinterpret_cast<const uint4*>(row0)[c];
+                                const uint4 x1 = reinterpret_cast<const uint4*>(row1)[c];
+                                a0 = sq_acc_bytes(a0, x0.x, qs[4 * c + 0]);
+                                a1 = sq_acc_bytes(a1, x1.x, qs[4 * c + 0]);
+                                a0 = sq_acc_bytes(a0, x0.y, qs[4 * c + 1]);
+                                a1 = sq_acc_bytes(a1, x1.y, qs[4 * c + 1]);
+                                a0 = sq_acc_bytes(a0, x0.z, qs[4 * c + 2]);
+                                a1 = sq_acc_bytes(a1, x1.z, qs[4 * c + 2]);
+                                a0 = sq_acc_bytes(a0, x0.w, qs[4 * c + 3]);
+                                a1 = sq_acc_bytes(a1, x1.w, qs[4 * c + 3]);
+                            }
+                        }
+                    }
                     const bool hi4 = (lane & 4) != 0;
                     float v = hi4 ? a1 : a0;
                     const float w = hi4 ? a0 : a1;
                     v += __shfl_xor_sync(0xffffffffu, w, 4);
                     v += __shfl_xor_sync(0xffffffffu, v, 2);
                     v += __shfl_xor_sync(0xffffffffu, v, 1);
-                    const bool v0 = act0 && g < p.m && violates(row0);
-                    const bool v1 = act1 && g < p.m && violates(row1);
-                    const unsigned bal0 = __ballot_sync(0xffffffffu, v0);
-                    const unsigned bal1 = __ballot_sync(0xffffffffu, v1);
-                    if (g == 0 && act0)
-                        nk[b0 + j0] = pack_key(__popc((bal0 >> (8 * gi)) & 0xFFu), v, cand[b0 + j0]);
-                    if (g == 4 && act1)
-                        nk[b0 + j1] = pack_key(__popc((bal1 >> (8 * gi)) & 0xFFu), v, cand[b0 + j1]);
+                    // violated predicates: lane g < m tests attribute g of both rows
+                    const int ga = (g < p.m) ? g : 0;
+                    const uint32_t av0 = *reinterpret_cast<const uint32_t*>(row0 + p.attr_off + 4 * ga);
+                    const uint32_t av1 = *reinterpret_cast<const uint32_t*>(row1 + p.attr_off + 4 * ga);
+                    bool v0, v1;
+                    if (my_float) {
+                        const float l = __int_as_float(my_lo), h = __int_as_float(my_hi);
+                        v0 = !(__uint_as_float(av0) >= l && __uint_as_float(av0) <= h);
+                        v1 = !(__uint_as_float(av1) >= l && __uint_as_float(av1) <= h);
+                    } else {
+                        v0 = (int32_t)av0 < my_lo || (int32_t)av0 > my_hi;
+                        v1 = (int32_t)av1 < my_lo || (int32_t)av1 > my_hi;
+                    }
+                    const unsigned bal0 = __ballot_sync(0xffffffffu, v0 && g < p.m);
+                    const unsigned bal1 = __ballot_sync(0xffffffffu, v1 && g < p.m);
+                    const unsigned bal = (lane & 4) ? bal1 : bal0;
+                    const int jj = (lane & 4) ? j1 : j0;
+                    if ((g & 3) == 0 && jj < nb)
+                        nk[b0 + jj] = pack_key(__popc((bal >> (8 * gi)) & 0xFFu), v, cand[b0 + jj]);
                 }
                 __syncwarp();                     // every lane is done with slot s
                 BOA_T_MARK(6);
@@ -429,17 +409,18 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
             const uint32_t h = (id * 0x9E3779B1u) & id_mask;
             const uint32_t tag = h & tag_mask;
             const uint32_t bucket = h >> p.tag_bits;
-            if (tag == 0xFFFFu) return true;              // would look like an empty way
             const uint2 b = *reinterpret_cast<const uint2*>(hash + 4 * bucket);
             const uint32_t w0 = b.x & 0xFFFFu, w1 = b.x >> 16, w2 = b.y & 0xFFFFu, w3 = b.y >> 16;
-            if (w0 == tag || w1 == tag || w2 == tag || w3 == tag) return false;
+            const bool found = (w0 == tag) | (w1 == tag) | (w2 == tag) | (w3 == tag);
             uint32_t way = (id ^ (id >> 7)) & 3u;
-            if (w3 == 0xFFFFu) way = 3u;
-            if (w2 == 0xFFFFu) way = 2u;
-            if (w1 == 0xFFFFu) way = 1u;
-            if (w0 == 0xFFFFu) way = 0u;
-            hash[4 * bucket + way] = (uint16_t)tag;
-            return true;
+            way = (w3 == 0xFFFFu) ? 3u : way;
+            way = (w2 == 0xFFFFu) ? 2u : way;
+            way = (w1 == 0xFFFFu) ? 1u : way;
+            way = (w0 == 0xFFFFu) ? 0u : way;
+            // a tag of 0xFFFF would look like an empty way: such an id is never recorded
+            const bool fresh = !found | (tag == 0xFFFFu);
+            if (fresh && tag != 0xFFFFu) hash[4 * bucket + way] = (uint16_t)tag;
+            return fresh;
         };
         // first unexpanded entry at or after `from` among the first `lim`, or -1
         auto first_unexpanded = [&](int from, int lim) -> int {
@@ -488,10 +469,10 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
 
         // ---- Algorithm 2 main loop
         BOA_T_MARK(0);
-        int pos = dead ? -1 : first_unexpanded(0, n < p.L ? n : p.L);
+        int pos = first_unexpanded(0, n < p.L ? n : p.L);
         uint32_t nb[RS];
         bool have_row = false;         // nb[] already holds the adjacency row of pool[pos]
-        while (!dead) {
+        for (;;) {
             if (pos < 0) break;                                   // converged
             if (n_exp >= p.max_expand) { capped = true; break; }
             if (!have_row) load_row_ids(key_id(pool[pos]), nb);
@@ -521,7 +502,6 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
                 n_sc += cnt;
                 // gather + distance + range check (fused)
                 score(cnt);
-                if (dead) break;
 
                 // new keys that cannot enter a full pool are dropped right away
                 const uint64_t worst = (n == p.C) ? (pool[n - 1] >> 1) : (kKeyMax >> 1);
@@ -551,25 +531,28 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
                 }
                 BOA_T_MARK(7);
 
-                // rank of every new key in the pool (4-ary search); drop keys it already holds
+                // rank of every new key in the pool (4-ary search, same trip count for all
+                // lanes, selects instead of branches); drop keys the pool already holds
+                int trips = 0;
+                for (int span = n; span > 0; span >>= 2) ++trips;
 #pragma unroll
                 for (int s = 0; s < RS; ++s) {
                     const uint64_t xs = x[s] >> 1;
                     const bool valid = x[s] != kKeyMax;
                     int lo_i = 0, hi_i = valid ? n : 0;
-                    while (__any_sync(0xffffffffu, lo_i < hi_i)) {
-                        if (lo_i < hi_i) {
-                            const int len = hi_i - lo_i;
-                            const int q1 = lo_i + (len >> 2), q2 = lo_i + (len >> 1);
-                            const int q3 = lo_i + ((3 * len) >> 2);
-                            const bool c1 = (pool[q1] >> 1) < xs;
-                            const bool c2 = (pool[q2] >> 1) < xs;
-                            const bool c3 = (pool[q3] >> 1) < xs;
-                            if (c3) lo_i = q3 + 1;
-                            else if (c2) { lo_i = q2 + 1; hi_i = q3; }
-                            else if (c1) { lo_i = q1 + 1; hi_i = q2; }
-                            else hi_i = q1;
-                        }
+                    for (int it = 0; it < trips; ++it) {
+                        const int len = hi_i - lo_i;
+                        const bool on = len > 0;
+                        const int q1 = lo_i + (len >> 2), q2 = lo_i + (len >> 1);
+                        const int q3 = lo_i + ((3 * len) >> 2);
+                        const uint64_t k1 = pool[on ? q1 : 0] >> 1;
+                        const uint64_t k2 = pool[on ? q2 : 0] >> 1;
+                        const uint64_t k3 = pool[on ? q3 : 0] >> 1;
+                        const bool c1 = k1 < xs, c2 = k2 < xs, c3 = k3 < xs;
+                        const int nlo = c3 ? q3 + 1 : (c2 ? q2 + 1 : (c1 ? q1 + 1 : lo_i));
+                        const int nhi = c3 ? hi_i : (c2 ? q3 : (c1 ? q2 : q1));
+                        lo_i = on ? nlo : lo_i;
+                        hi_i = on ? nhi : hi_i;
                     }
                     const bool dup = valid && (lo_i < n) && ((pool[lo_i] >> 1) == xs);
                     const bool nd = valid && !dup;
@@ -662,8 +645,6 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
             }
             BOA_T_MARK(9);
         }
-        if (dead) break;
-
         // ---- result: the k nearest filter-valid entries (valid ones sort first)
         const int lim = n < p.L ? n : p.L;
         int nv_beam = 0;            // filter-valid entries among the first L
