@@ -32,10 +32,11 @@ if ROOT not in sys.path:
 METRIC = "queries/sec at recall@10>=0.95 (10k-query batch)"
 UNIT = "queries/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum of the search kernel, from the ncu capture
-# summarised in profiles/ (bytes per scored neighbour, measured on a smaller case and
-# scaled by the neighbours a full launch scores).  None until a capture exists.
-NCU_DRAM_BYTES_PER_SCORED = None
+# dram__bytes_read.sum + dram__bytes_write.sum of the search kernel per scored neighbour
+# record, from the full-size ncu capture summarised in
+# profiles/boa_search_kernel_c2_dram_traffic.md (48.99 GB for 99.43 M records).  It holds
+# for the default workload and table size only.
+NCU_DRAM_BYTES_PER_SCORED = {"c2": 492.7}
 
 
 def parse_args():
@@ -381,8 +382,9 @@ def main():
     kernel_ms = float(np.mean(step_ms))
     achieved = alg_bytes / (kernel_ms / 1e3) / 1e9
     traffic = None
-    if NCU_DRAM_BYTES_PER_SCORED is not None:
-        traffic = NCU_DRAM_BYTES_PER_SCORED * float(st["n_scored"].sum())
+    if (args.workload in NCU_DRAM_BYTES_PER_SCORED and not args.scale_n and not args.hash_log2
+            and not args.stage_rows):
+        traffic = NCU_DRAM_BYTES_PER_SCORED[args.workload] * float(st["n_scored"].sum())
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
