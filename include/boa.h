@@ -54,8 +54,8 @@ enum {
     BOA_PARAM_CAP_ADD = 6,  /*   expansions; defaults 8 and 64                               */
     BOA_PARAM_HASH_LOG2 = 7, /* 0 = choose per phase; else log2 of the per-query table of
                                recently scored ids (8..14).  Never changes results.          */
-    BOA_PARAM_STAGE_ROWS = 8 /* 0 = choose; else neighbour records one query keeps in flight
-                               in shared memory (2..64).  Never changes results.             */
+    BOA_PARAM_MAX_WARPS_PER_SM = 8 /* 0 = as many query warps per SM as fit; else a cap.
+                               Never changes results.                                        */
 };
 
 /*

@@ -151,7 +151,7 @@ __global__ void copy_word_kernel(uint32_t* dst, const uint32_t* src) { *dst = *s
 struct boa_index {
     int64_t N = 0;
     int D = 0, m = 0, R = 0, vec_dtype = 0;
-    int rec_stride = 0, rec_bytes = 0, nchunks = 0, attr_off = 0;
+    int rec_stride = 0, nchunks = 0, attr_off = 0;
     uint32_t attr_float_mask = 0;
     int64_t entry = 0;
     uint8_t* rec = nullptr;
@@ -159,7 +159,7 @@ struct boa_index {
     int device = 0, num_sms = 0;
     // parameters
     double eps = 0.05, growth = 4.0, tau = 0.0;
-    int mode = 0, plus_k = 0, cap_mult = 8, cap_add = 64, hash_log2 = 0, stage_rows = 0;
+    int mode = 0, plus_k = 0, cap_mult = 8, cap_add = 64, hash_log2 = 0, max_ctas = 0;
     int n_sched = 0;
     int sched[BOA_MAX_PHASES] = {0};
     // scratch
@@ -271,16 +271,6 @@ int choose_hash_log2(const boa_index* ix, int L)
     return lg;
 }
 
-int choose_stage_rows(const boa_index* ix, int rs)
-{
-    // default: one slot of eight rows (a full scoring pass), fewer for very long rows
-    int rows = ix->stage_rows ? ix->stage_rows : (8 * ix->rec_bytes <= 16384 ? 8 : 16384 / ix->rec_bytes);
-    if (rows > 32 * rs) rows = 32 * rs;
-    if (rows >= 16) rows &= ~1;       // two ring slots of equal size
-    if (rows < 1) rows = 1;
-    return rows;
-}
-
 int phase_widths(const boa_index* ix, int L0, int Lmax, int* w)
 {
     if (ix->n_sched > 0) {
@@ -354,7 +344,6 @@ int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_p
         sp.id_bits = id_bits;
         sp.tag_bits = id_bits - bucket_bits;
     }
-    sp.stage_rows = choose_stage_rows(ix, lp.kc.rs);
     sp.max_expand = ix->cap_mult * L + ix->cap_add;
     sp.first_phase = p == 0;
     sp.resume_in = (ix->mode == 1 && p > 0);
@@ -370,8 +359,7 @@ int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_p
     sp.out_list = ix->lists + (size_t)(p + 1 < BOA_MAX_PHASES ? p + 1 : p) * ix->ws_Q;
     sp.out_count = ix->counters + kCntCount + p + 1;
 
-    const boa::WarpSmem lay = boa::warp_smem_layout(sp.C, sp.hash_log2, ix->D, lp.kc.rs, sp.stage_rows,
-                                                    ix->rec_bytes);
+    const boa::WarpSmem lay = boa::warp_smem_layout(sp.C, sp.hash_log2, ix->D, lp.kc.rs);
     const size_t smem = (size_t)lay.total;
     if (smem > 48 * 1024) {
         BOA_CUDA(cudaFuncSetAttribute((const void*)lp.kc.fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -381,6 +369,7 @@ int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_p
     BOA_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, (const void*)lp.kc.fn,
                                                            boa::kThreads, smem));
     if (per_sm < 1) return BOA_EINVAL;
+    if (ix->max_ctas > 0 && per_sm > ix->max_ctas) per_sm = ix->max_ctas;
     int64_t grid = (int64_t)per_sm * ix->num_sms;
     const int64_t need = (int64_t)expected_items;
     if (need < grid) grid = need < 1 ? 1 : need;
@@ -446,7 +435,6 @@ int boa_index_create(boa_index** out, const void* vectors, int vec_dtype, int64_
     ix->nchunks = vec_bytes / 16;
     ix->attr_off = vec_bytes;
     ix->rec_stride = (vec_bytes + 4 * m + 31) & ~31;
-    ix->rec_bytes = (vec_bytes + 4 * m + 15) & ~15;
     for (int j = 0; j < m; ++j)
         if (attr_types[j] == BOA_ATTR_F32) ix->attr_float_mask |= 1u << j;
     BOA_TRY(cudaGetDevice(&ix->device));
@@ -555,9 +543,9 @@ int boa_set_param(boa_index* ix, int key, double v)
         case BOA_PARAM_HASH_LOG2:
             if (v != 0.0 && (v < 8.0 || v > 15.0 || v != floor(v))) return BOA_EINVAL;
             ix->hash_log2 = (int)v; return BOA_OK;
-        case BOA_PARAM_STAGE_ROWS:
+        case BOA_PARAM_MAX_WARPS_PER_SM:
             if (v < 0.0 || v > 64.0 || v != floor(v)) return BOA_EINVAL;
-            ix->stage_rows = (int)v; return BOA_OK;
+            ix->max_ctas = (int)v; return BOA_OK;
         default: return BOA_EINVAL;
     }
 }
@@ -609,7 +597,7 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
     boa::SearchParams& b = lp.base;
     memset(&b, 0, sizeof(b));
     b.rec = ix->rec; b.graph = ix->graph; b.N = ix->N; b.D = ix->D; b.m = ix->m; b.R = ix->R;
-    b.rec_stride = ix->rec_stride; b.rec_bytes = ix->rec_bytes; b.nchunks = ix->nchunks;
+    b.rec_stride = ix->rec_stride; b.nchunks = ix->nchunks;
     b.attr_off = ix->attr_off; b.status = ix->counters + kCntStatus;
     b.timers = reinterpret_cast<unsigned long long*>(ix->counters + kCntWords);
     b.attr_float_mask = ix->attr_float_mask; b.entry = (uint32_t)ix->entry;

@@ -10,13 +10,15 @@
 // lambda -> infinity reading of the paper's score dist + lambda*phi.
 //
 // Neighbour records (vector + attribute cells, one contiguous 32-byte-aligned row
-// each) are fetched with 16-byte asynchronous copies (cp.async, global -> shared, L2
-// only) into a ring of one or two slots in shared memory: the 32 lanes copy 512
-// consecutive bytes of a row per instruction, one commit group per slot.  No register
-// holds data in flight, so one warp keeps up to `stage_rows` whole rows in flight
-// while it scores the rows that have already arrived.  (A bulk copy per row through
-// the TMA engine was measured first: it needs one uniform-datapath instruction
-// sequence per row, about ten instructions each, which made the kernel issue-bound.)
+// each) are read with 16-byte loads that bypass L1, straight into registers: eight
+// rows per pass, 8 lanes per row, every lane issues all its loads of the pass (two
+// rows, up to four chunks each) before the first use, so a warp keeps 4 KB in flight
+// and an SM with 16 resident warps about 64 KB.  Two staged variants were measured
+// first and dropped: one cp.async.bulk (TMA) copy per row into shared memory needs a
+// uniform-datapath instruction sequence per row, and 16-byte cp.async copies spend
+// as long issuing as waiting; both were 40 % slower than register loads on the 1M x
+// 128-d workload because the kernel is bound by instruction issue and dependent
+// latency, not by the number of bytes in flight.
 //
 // The table of recently scored ids stores 16-bit tags in 4-way buckets.  An id is
 // first mapped by an odd multiplier modulo 2^id_bits (a bijection); the high bits
@@ -36,6 +38,12 @@
 
 namespace boa {
 
+// Query warps per SM the register allocation is tuned for: with fewer registers than this
+// allows the compiler stops keeping a whole scoring pass of loads in flight.
+#ifndef BOA_MIN_CTAS
+#define BOA_MIN_CTAS 16
+#endif
+
 constexpr uint32_t kNoId = 0xFFFFFFFFu;
 constexpr int kThreads = 32;           // one warp per CTA
 constexpr uint64_t kKeyMax = ~0ull;
@@ -43,6 +51,9 @@ constexpr uint64_t kKeyMax = ~0ull;
 enum : uint32_t { kStatusCopyTimeout = 1u };   // reserved: no wait in the kernel can time out
 
 // Optional per-section cycle counters (build with -DBOA_SECTION_TIMERS; off in the product).
+// Keeps the compiler from moving code across this point.
+#define BOA_SCHED_FENCE() asm volatile("" ::: "memory")
+
 #ifdef BOA_SECTION_TIMERS
 #define BOA_T_DECL long long t_prev_ = clock64(); long long t_acc_[12] = {0}
 #define BOA_T_MARK(i) do { long long t_now_ = clock64(); t_acc_[i] += t_now_ - t_prev_; t_prev_ = t_now_; } while (0)
@@ -60,7 +71,6 @@ struct SearchParams {
     int64_t N;
     int D, m, R;
     int rec_stride;           // bytes, multiple of 32
-    int rec_bytes;            // bytes of a record that are copied (vector + cells, 16-byte multiple)
     int nchunks;              // 16-byte chunks of one vector
     int attr_off;             // byte offset of the attribute cells inside a record
     uint32_t attr_float_mask; // bit j set: column j is float
@@ -79,7 +89,6 @@ struct SearchParams {
     int hash_log2;            // log2 of the 16-bit entries in the table of recently scored ids
     int id_bits;              // bits of a node id (ids < 2^id_bits)
     int tag_bits;             // id_bits - log2(buckets), at most 16
-    int stage_rows;           // records the staging ring holds (two slots of half that)
     int max_expand;           // expansions after which a phase gives up
     int first_phase;          // statistics start from zero
     int resume_in;            // load the pool a narrower phase spilled
@@ -126,14 +135,29 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p)
 {
     return (uint32_t)__cvta_generic_to_shared(p);
 }
-// 16 bytes, global -> shared, cached in L2 only.
-__device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src)
+// Predicated 16-byte / 4-byte loads that bypass L1 (each record is used once).
+__device__ __forceinline__ uint4 ldg_stream128(const void* ptr, bool pred)
 {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
+    uint4 v;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %5, 0;\n\t"
+        "mov.u32 %0, 0;\n\tmov.u32 %1, 0;\n\tmov.u32 %2, 0;\n\tmov.u32 %3, 0;\n\t"
+        "@p ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n\t}"
+        : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+        : "l"(ptr), "r"((uint32_t)pred));
+    return v;
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ uint32_t ldg_stream32(const void* ptr, bool pred)
+{
+    uint32_t v;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\tmov.u32 %0, 0;\n\t"
+        "@p ld.global.nc.L1::no_allocate.u32 %0, [%1];\n\t}"
+        : "=r"(v)
+        : "l"(ptr), "r"((uint32_t)pred));
+    return v;
+}
+__device__ __forceinline__ float sq_acc4u(float acc, uint4 x, float4 q);
 
 __device__ __forceinline__ float sq_acc4(float acc, float4 x, float4 q)
 {
@@ -143,6 +167,11 @@ __device__ __forceinline__ float sq_acc4(float acc, float4 x, float4 q)
     d = x.z - q.z; acc = fmaf(d, d, acc);
     d = x.w - q.w; acc = fmaf(d, d, acc);
     return acc;
+}
+__device__ __forceinline__ float sq_acc4u(float acc, uint4 x, float4 q)
+{
+    return sq_acc4(acc, make_float4(__uint_as_float(x.x), __uint_as_float(x.y), __uint_as_float(x.z),
+                                    __uint_as_float(x.w)), q);
 }
 __device__ __forceinline__ float sq_acc_bytes(float acc, uint32_t w, float4 q)
 {
@@ -186,21 +215,18 @@ __device__ __forceinline__ void sort_keys(uint64_t (&x)[RS], int lane)
 
 // Per-warp shared memory carve-up (bytes), shared by host and device.
 struct WarpSmem {
-    int pool_off, nk_off, nr_off, cand_off, hash_off, q_off, stage_off, bar_off, total;
+    int pool_off, nk_off, nr_off, cand_off, hash_off, q_off, total;
 };
-__host__ __device__ inline WarpSmem warp_smem_layout(int C, int hash_log2, int D, int RS,
-                                                     int stage_rows, int rec_bytes)
+__host__ __device__ inline WarpSmem warp_smem_layout(int C, int hash_log2, int D, int RS)
 {
     WarpSmem s;
     int off = 0;
-    s.stage_off = off; off += stage_rows * rec_bytes;          // 16-byte multiple
     s.pool_off = off;  off += ((C + 1) & ~1) * 8;
     s.nk_off = off;    off += 32 * RS * 8;
     s.q_off = off;     off += ((D * 4 + 15) & ~15);
     s.hash_off = off;  off += (1 << hash_log2) * 2;
     s.cand_off = off;  off += 32 * RS * 4;
     s.nr_off = off;    off += 32 * RS * 4;
-    s.bar_off = off;   off += 16;
     s.total = (off + 127) & ~127;
     return s;
 }
@@ -212,7 +238,7 @@ __host__ __device__ inline WarpSmem warp_smem_layout(int C, int hash_log2, int D
 // loop is unrolled); 0 = any length, query slices read from shared memory.  EXACT: the
 // row has exactly 8*CPL chunks, so no lane ever has a chunk missing.
 template <int VT, int RS, int CPL, bool EXACT>
-__global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams p)
+__global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(const SearchParams p)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     const int lane = threadIdx.x;
@@ -222,8 +248,7 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
     constexpr int QF4 = (VT == 0) ? 1 : 4;          // float4 slices of the query per chunk
     constexpr int NQ = (CPL > 0) ? CPL * QF4 : 1;
 
-    const WarpSmem lay = warp_smem_layout(p.C, p.hash_log2, p.D, RS, p.stage_rows, p.rec_bytes);
-    uint8_t* stage = smem_raw + lay.stage_off;
+    const WarpSmem lay = warp_smem_layout(p.C, p.hash_log2, p.D, RS);
     uint64_t* pool = reinterpret_cast<uint64_t*>(smem_raw + lay.pool_off);
     uint64_t* nk = reinterpret_cast<uint64_t*>(smem_raw + lay.nk_off);
     uint32_t* nr = reinterpret_cast<uint32_t*>(smem_raw + lay.nr_off);
@@ -233,8 +258,6 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
 
     const uint32_t id_mask = (p.id_bits >= 32) ? 0xFFFFFFFFu : ((1u << p.id_bits) - 1u);
     const uint32_t tag_mask = (1u << p.tag_bits) - 1u;
-    const int n_slots = p.stage_rows >= 16 ? 2 : 1;   // ring slots of the staging area
-    const int half_rows = p.stage_rows / n_slots;      // rows per slot
 
     // work range of this launch
     const uint32_t w_begin = p.in_begin_ptr ? *p.in_begin_ptr : p.in_begin;
@@ -246,10 +269,6 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
     const uint32_t n_work = w_end > w_begin ? w_end - w_begin : 0u;
 
     BOA_T_DECL;
-    const uint32_t stage_s = smem_u32(stage);
-    const int pieces = p.rec_bytes >> 4;            // 16-byte pieces of one record
-    const int full = pieces >> 5;                   // 512-byte spans of a record
-    const int tail = pieces & 31;                   // pieces after the last full span
 
     for (;;) {
         uint32_t t = 0;
@@ -284,124 +303,110 @@ __global__ void __launch_bounds__(kThreads) boa_search_kernel(const SearchParams
             }
         }
 
-        // Scores cand[0..cnt): fetch the records through the staging ring, then
-        // distance + violated predicates -> nk[0..cnt).
+        // Scores cand[0..cnt) straight from global memory: eight rows per pass, every lane
+        // loads its own 16-byte chunks of two rows into registers (all loads of a pass are
+        // issued before the first use), distance + violated predicates -> nk[0..cnt).
         auto score = [&](int cnt) {
-            const int nbatch = (cnt + half_rows - 1) / half_rows;
-            auto issue = [&](int b) {
-                const int s = (n_slots == 2) ? (b & 1) : 0;
-                const int b0 = b * half_rows;
-                const int nb = (cnt - b0 < half_rows) ? cnt - b0 : half_rows;
-                const uint32_t dst0 = stage_s + (uint32_t)(s * half_rows * p.rec_bytes);
-                for (int j = 0; j < nb; ++j) {
-                    const uint8_t* src = p.rec + (size_t)cand[b0 + j] * p.rec_stride + 16 * lane;
-                    const uint32_t dst = dst0 + (uint32_t)(j * p.rec_bytes) + 16u * lane;
-                    for (int f = 0; f < full; ++f) cp_async16(dst + 512u * f, src + 512 * f);
-                }
-                if (tail) {
-                    // the pieces after the last full span, for all rows of the batch at once
-                    for (int t = lane; t < nb * tail; t += 32) {
-                        const int j = t / tail, pc = 32 * full + t % tail;
-                        cp_async16(dst0 + (uint32_t)(j * p.rec_bytes + 16 * pc),
-                                   p.rec + (size_t)cand[b0 + j] * p.rec_stride + 16 * pc);
-                    }
-                }
-                cp_async_commit();
-            };
             BOA_T_MARK(3);
-            issue(0);
-            if (n_slots == 2 && nbatch > 1) issue(1);
-            BOA_T_MARK(4);
-            for (int b = 0; b < nbatch; ++b) {
-                const int s = (n_slots == 2) ? (b & 1) : 0;
-                const int b0 = b * half_rows;
-                const int nb = (cnt - b0 < half_rows) ? cnt - b0 : half_rows;
-                // the newest group may stay in flight only if it belongs to the batch after this one
-                if (n_slots == 2 && b + 1 < nbatch) cp_async_wait<1>(); else cp_async_wait<0>();
-                __syncwarp();
-                BOA_T_MARK(5);
-                const uint8_t* src = stage + (size_t)s * half_rows * p.rec_bytes;
-                // eight rows per pass: every 8-lane group takes two, and the two partial-sum
-                // sets share one butterfly (lanes 0-3 of a group finish the first row, lanes
-                // 4-7 the second; the pairs added are the same as for a single row)
-                for (int r0 = 0; r0 < nb; r0 += 8) {
-                    const int j0 = r0 + gi, j1 = r0 + 4 + gi;
-                    const bool act0 = j0 < nb, act1 = j1 < nb;
-                    const uint8_t* row0 = src + (act0 ? j0 : 0) * p.rec_bytes;
-                    const uint8_t* row1 = src + (act1 ? j1 : 0) * p.rec_bytes;
-                    float a0 = 0.0f, a1 = 0.0f;
-                    if (CPL > 0) {
+#pragma unroll 1
+            for (int r0 = 0; r0 < cnt; r0 += 8) {
+                BOA_SCHED_FENCE();
+                const int j0 = r0 + gi, j1 = r0 + 4 + gi;
+                const bool act0 = j0 < cnt, act1 = j1 < cnt;
+                const uint32_t id0 = cand[act0 ? j0 : 0], id1 = cand[act1 ? j1 : 0];
+                const uint8_t* row0 = p.rec + (size_t)id0 * p.rec_stride;
+                const uint8_t* row1 = p.rec + (size_t)id1 * p.rec_stride;
+                const int ga = (g < p.m) ? g : 0;
+                float a0 = 0.0f, a1 = 0.0f;
+                uint32_t av0, av1;
+                if (CPL > 0) {
+                    uint4 x0[CPL > 0 ? CPL : 1], x1[CPL > 0 ? CPL : 1];
 #pragma unroll
-                        for (int i = 0; i < (CPL > 0 ? CPL : 1); ++i) {
-                            const int c = g + 8 * i;
-                            if (EXACT || c < p.nchunks) {
+                    for (int i = 0; i < (CPL > 0 ? CPL : 1); ++i) {
+                        const int c = g + 8 * i;
+                        const bool in = EXACT || c < p.nchunks;
+                        x0[i] = ldg_stream128(row0 + 16 * c, act0 && in);
+                        x1[i] = ldg_stream128(row1 + 16 * c, act1 && in);
+                    }
+                    av0 = ldg_stream32(row0 + p.attr_off + 4 * ga, act0 && g < p.m);
+                    av1 = ldg_stream32(row1 + p.attr_off + 4 * ga, act1 && g < p.m);
+                    BOA_T_MARK(4);
+                    BOA_SCHED_FENCE();        // every load of the pass is issued before its first use
+#pragma unroll
+                    for (int i = 0; i < (CPL > 0 ? CPL : 1); ++i) {
+                        if (VT == 0) {
+                            a0 = sq_acc4u(a0, x0[i], qreg[i]);
+                            a1 = sq_acc4u(a1, x1[i], qreg[i]);
+                        } else {
+                            a0 = sq_acc_bytes(a0, x0[i].x, qreg[4 * i + 0]);
+                            a1 = sq_acc_bytes(a1, x1[i].x, qreg[4 * i + 0]);
+                            a0 = sq_acc_bytes(a0, x0[i].y, qreg[4 * i + 1]);
+                            a1 = sq_acc_bytes(a1, x1[i].y, qreg[4 * i + 1]);
+                            a0 = sq_acc_bytes(a0, x0[i].z, qreg[4 * i + 2]);
+                            a1 = sq_acc_bytes(a1, x1[i].z, qreg[4 * i + 2]);
+                            a0 = sq_acc_bytes(a0, x0[i].w, qreg[4 * i + 3]);
+                            a1 = sq_acc_bytes(a1, x1[i].w, qreg[4 * i + 3]);
+                        }
+                    }
+                } else {
+                    av0 = ldg_stream32(row0 + p.attr_off + 4 * ga, act0 && g < p.m);
+                    av1 = ldg_stream32(row1 + p.attr_off + 4 * ga, act1 && g < p.m);
+                    // long rows: four chunks of each row in flight per lane at a time
+                    for (int c0 = g; c0 < p.nchunks; c0 += 32) {
+                        uint4 x0[4], x1[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int c = c0 + 8 * i;
+                            x0[i] = ldg_stream128(row0 + 16 * c, act0 && c < p.nchunks);
+                            x1[i] = ldg_stream128(row1 + 16 * c, act1 && c < p.nchunks);
+                        }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int c = c0 + 8 * i;
+                            if (c < p.nchunks) {
                                 if (VT == 0) {
-                                    a0 = sq_acc4(a0, reinterpret_cast<const float4*>(row0)[c], qreg[i]);
-                                    a1 = sq_acc4(a1, reinterpret_cast<const float4*>(row1)[c], qreg[i]);
+                                    const float4 qq = qs[c];
+                                    a0 = sq_acc4u(a0, x0[i], qq);
+                                    a1 = sq_acc4u(a1, x1[i], qq);
                                 } else {
-                                    const uint4 x0 = reinterpret_cast<const uint4*>(row0)[c];
-                                    const uint4 x1 = reinterpret_cast<const uint4*>(row1)[c];
-                                    a0 = sq_acc_bytes(a0, x0.x, qreg[4 * i + 0]);
-                                    a1 = sq_acc_bytes(a1, x1.x, qreg[4 * i + 0]);
-                                    a0 = sq_acc_bytes(a0, x0.y, qreg[4 * i + 1]);
-                                    a1 = sq_acc_bytes(a1, x1.y, qreg[4 * i + 1]);
-                                    a0 = sq_acc_bytes(a0, x0.z, qreg[4 * i + 2]);
-                                    a1 = sq_acc_bytes(a1, x1.z, qreg[4 * i + 2]);
-                                    a0 = sq_acc_bytes(a0, x0.w, qreg[4 * i + 3]);
-                                    a1 = sq_acc_bytes(a1, x1.w, qreg[4 * i + 3]);
+                                    a0 = sq_acc_bytes(a0, x0[i].x, qs[4 * c + 0]);
+                                    a1 = sq_acc_bytes(a1, x1[i].x, qs[4 * c + 0]);
+                                    a0 = sq_acc_bytes(a0, x0[i].y, qs[4 * c + 1]);
+                                    a1 = sq_acc_bytes(a1, x1[i].y, qs[4 * c + 1]);
+                                    a0 = sq_acc_bytes(a0, x0[i].z, qs[4 * c + 2]);
+                                    a1 = sq_acc_bytes(a1, x1[i].z, qs[4 * c + 2]);
+                                    a0 = sq_acc_bytes(a0, x0[i].w, qs[4 * c + 3]);
+                                    a1 = sq_acc_bytes(a1, x1[i].w, qs[4 * c + 3]);
                                 }
                             }
                         }
-                    } else {
-                        for (int c = g; c < p.nchunks; c += 8) {
-                            if (VT == 0) {
-                                const float4 qq = qs[c];
-                                a0 = sq_acc4(a0, reinterpret_cast<const float4*>(row0)[c], qq);
-                                a1 = sq_acc4(a1, reinterpret_cast<const float4*>(row1)[c], qq);
-                            } else {
-                                const uint4 x0 = reinterpret_cast<const uint4*>(row0)[c];
-                                const uint4 x1 = reinterpret_cast<const uint4*>(row1)[c];
-                                a0 = sq_acc_bytes(a0, x0.x, qs[4 * c + 0]);
-                                a1 = sq_acc_bytes(a1, x1.x, qs[4 * c + 0]);
-                                a0 = sq_acc_bytes(a0, x0.y, qs[4 * c + 1]);
-                                a1 = sq_acc_bytes(a1, x1.y, qs[4 * c + 1]);
-                                a0 = sq_acc_bytes(a0, x0.z, qs[4 * c + 2]);
-                                a1 = sq_acc_bytes(a1, x1.z, qs[4 * c + 2]);
-                                a0 = sq_acc_bytes(a0, x0.w, qs[4 * c + 3]);
-                                a1 = sq_acc_bytes(a1, x1.w, qs[4 * c + 3]);
-                            }
-                        }
                     }
-                    const bool hi4 = (lane & 4) != 0;
-                    float v = hi4 ? a1 : a0;
-                    const float w = hi4 ? a0 : a1;
-                    v += __shfl_xor_sync(0xffffffffu, w, 4);
-                    v += __shfl_xor_sync(0xffffffffu, v, 2);
-                    v += __shfl_xor_sync(0xffffffffu, v, 1);
-                    // violated predicates: lane g < m tests attribute g of both rows
-                    const int ga = (g < p.m) ? g : 0;
-                    const uint32_t av0 = *reinterpret_cast<const uint32_t*>(row0 + p.attr_off + 4 * ga);
-                    const uint32_t av1 = *reinterpret_cast<const uint32_t*>(row1 + p.attr_off + 4 * ga);
-                    bool v0, v1;
-                    if (my_float) {
-                        const float l = __int_as_float(my_lo), h = __int_as_float(my_hi);
-                        v0 = !(__uint_as_float(av0) >= l && __uint_as_float(av0) <= h);
-                        v1 = !(__uint_as_float(av1) >= l && __uint_as_float(av1) <= h);
-                    } else {
-                        v0 = (int32_t)av0 < my_lo || (int32_t)av0 > my_hi;
-                        v1 = (int32_t)av1 < my_lo || (int32_t)av1 > my_hi;
-                    }
-                    const unsigned bal0 = __ballot_sync(0xffffffffu, v0 && g < p.m);
-                    const unsigned bal1 = __ballot_sync(0xffffffffu, v1 && g < p.m);
-                    const unsigned bal = (lane & 4) ? bal1 : bal0;
-                    const int jj = (lane & 4) ? j1 : j0;
-                    if ((g & 3) == 0 && jj < nb)
-                        nk[b0 + jj] = pack_key(__popc((bal >> (8 * gi)) & 0xFFu), v, cand[b0 + jj]);
+                    BOA_T_MARK(4);
                 }
-                __syncwarp();                     // every lane is done with slot s
+                const bool hi4 = (lane & 4) != 0;
+                float v = hi4 ? a1 : a0;
+                const float w = hi4 ? a0 : a1;
+                v += __shfl_xor_sync(0xffffffffu, w, 4);
+                v += __shfl_xor_sync(0xffffffffu, v, 2);
+                v += __shfl_xor_sync(0xffffffffu, v, 1);
+                bool v0, v1;
+                if (my_float) {
+                    const float l = __int_as_float(my_lo), h = __int_as_float(my_hi);
+                    v0 = !(__uint_as_float(av0) >= l && __uint_as_float(av0) <= h);
+                    v1 = !(__uint_as_float(av1) >= l && __uint_as_float(av1) <= h);
+                } else {
+                    v0 = (int32_t)av0 < my_lo || (int32_t)av0 > my_hi;
+                    v1 = (int32_t)av1 < my_lo || (int32_t)av1 > my_hi;
+                }
+                const unsigned bal0 = __ballot_sync(0xffffffffu, v0 && act0 && g < p.m);
+                const unsigned bal1 = __ballot_sync(0xffffffffu, v1 && act1 && g < p.m);
+                const unsigned bal = hi4 ? bal1 : bal0;
+                const int jj = hi4 ? j1 : j0;
+                if ((g & 3) == 0 && jj < cnt)
+                    nk[jj] = pack_key(__popc((bal >> (8 * gi)) & 0xFFu), v, hi4 ? id1 : id0);
                 BOA_T_MARK(6);
-                if (b + n_slots < nbatch) issue(b + n_slots);
             }
+            __syncwarp();
         };
 
         // Returns true when id was not in the table; records it either way.
