@@ -10,7 +10,7 @@
 // lambda -> infinity reading of the paper's score dist + lambda*phi.
 //
 // Neighbour records (vector + attribute cells, one contiguous 32-byte-aligned row
-// each) are read with 16-byte loads that bypass L1, straight into registers: eight
+// each) are read with 16-byte read-only loads straight into registers: eight
 // rows per pass, 8 lanes per row, every lane issues all its loads of the pass (two
 // rows, up to four chunks each) before the first use, so a warp keeps 4 KB in flight
 // and an SM with 16 resident warps about 64 KB.  Two staged variants were measured
@@ -135,14 +135,58 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p)
 {
     return (uint32_t)__cvta_generic_to_shared(p);
 }
-// Predicated 16-byte / 4-byte loads that bypass L1 (each record is used once).
+// Predicated read-only loads.  When the predicate is false nothing is loaded and the
+// outputs keep whatever the registers held: callers never use them in that case.
+template <int N>
+__device__ __forceinline__ void ldg_chunks(uint4 (&v)[N], const uint8_t* ptr, bool pred)
+{
+    static_assert(N >= 1 && N <= 4, "one to four 16-byte chunks, 128 bytes apart");
+    if (N == 1) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %5, 0;\n\t"
+            "@p ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];\n\t}"
+            : "=r"(v[0].x), "=r"(v[0].y), "=r"(v[0].z), "=r"(v[0].w)
+            : "l"(ptr), "r"((uint32_t)pred));
+    } else if (N == 2) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %9, 0;\n\t"
+            "@p ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%8];\n\t"
+            "@p ld.global.nc.v4.u32 {%4,%5,%6,%7}, [%8+128];\n\t}"
+            : "=r"(v[0].x), "=r"(v[0].y), "=r"(v[0].z), "=r"(v[0].w), "=r"(v[N > 1 ? 1 : 0].x),
+              "=r"(v[N > 1 ? 1 : 0].y), "=r"(v[N > 1 ? 1 : 0].z), "=r"(v[N > 1 ? 1 : 0].w)
+            : "l"(ptr), "r"((uint32_t)pred));
+    } else if (N == 3) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %13, 0;\n\t"
+            "@p ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%12];\n\t"
+            "@p ld.global.nc.v4.u32 {%4,%5,%6,%7}, [%12+128];\n\t"
+            "@p ld.global.nc.v4.u32 {%8,%9,%10,%11}, [%12+256];\n\t}"
+            : "=r"(v[0].x), "=r"(v[0].y), "=r"(v[0].z), "=r"(v[0].w), "=r"(v[N > 1 ? 1 : 0].x),
+              "=r"(v[N > 1 ? 1 : 0].y), "=r"(v[N > 1 ? 1 : 0].z), "=r"(v[N > 1 ? 1 : 0].w),
+              "=r"(v[N > 2 ? 2 : 0].x), "=r"(v[N > 2 ? 2 : 0].y), "=r"(v[N > 2 ? 2 : 0].z),
+              "=r"(v[N > 2 ? 2 : 0].w)
+            : "l"(ptr), "r"((uint32_t)pred));
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %17, 0;\n\t"
+            "@p ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%16];\n\t"
+            "@p ld.global.nc.v4.u32 {%4,%5,%6,%7}, [%16+128];\n\t"
+            "@p ld.global.nc.v4.u32 {%8,%9,%10,%11}, [%16+256];\n\t"
+            "@p ld.global.nc.v4.u32 {%12,%13,%14,%15}, [%16+384];\n\t}"
+            : "=r"(v[0].x), "=r"(v[0].y), "=r"(v[0].z), "=r"(v[0].w), "=r"(v[N > 1 ? 1 : 0].x),
+              "=r"(v[N > 1 ? 1 : 0].y), "=r"(v[N > 1 ? 1 : 0].z), "=r"(v[N > 1 ? 1 : 0].w),
+              "=r"(v[N > 2 ? 2 : 0].x), "=r"(v[N > 2 ? 2 : 0].y), "=r"(v[N > 2 ? 2 : 0].z),
+              "=r"(v[N > 2 ? 2 : 0].w), "=r"(v[N > 3 ? 3 : 0].x), "=r"(v[N > 3 ? 3 : 0].y),
+              "=r"(v[N > 3 ? 3 : 0].z), "=r"(v[N > 3 ? 3 : 0].w)
+            : "l"(ptr), "r"((uint32_t)pred));
+    }
+}
 __device__ __forceinline__ uint4 ldg_stream128(const void* ptr, bool pred)
 {
     uint4 v;
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %5, 0;\n\t"
-        "mov.u32 %0, 0;\n\tmov.u32 %1, 0;\n\tmov.u32 %2, 0;\n\tmov.u32 %3, 0;\n\t"
-        "@p ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n\t}"
+        "@p ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];\n\t}"
         : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
         : "l"(ptr), "r"((uint32_t)pred));
     return v;
@@ -151,8 +195,8 @@ __device__ __forceinline__ uint32_t ldg_stream32(const void* ptr, bool pred)
 {
     uint32_t v;
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\tmov.u32 %0, 0;\n\t"
-        "@p ld.global.nc.L1::no_allocate.u32 %0, [%1];\n\t}"
+        "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t"
+        "@p ld.global.nc.u32 %0, [%1];\n\t}"
         : "=r"(v)
         : "l"(ptr), "r"((uint32_t)pred));
     return v;
@@ -321,12 +365,17 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                 uint32_t av0, av1;
                 if (CPL > 0) {
                     uint4 x0[CPL > 0 ? CPL : 1], x1[CPL > 0 ? CPL : 1];
+                    if (EXACT) {
+                        // one predicate per row; chunk i sits 128 bytes after chunk i-1
+                        ldg_chunks<(CPL > 0 ? CPL : 1)>(x0, row0 + 16 * g, act0);
+                        ldg_chunks<(CPL > 0 ? CPL : 1)>(x1, row1 + 16 * g, act1);
+                    } else {
 #pragma unroll
-                    for (int i = 0; i < (CPL > 0 ? CPL : 1); ++i) {
-                        const int c = g + 8 * i;
-                        const bool in = EXACT || c < p.nchunks;
-                        x0[i] = ldg_stream128(row0 + 16 * c, act0 && in);
-                        x1[i] = ldg_stream128(row1 + 16 * c, act1 && in);
+                        for (int i = 0; i < (CPL > 0 ? CPL : 1); ++i) {
+                            const int c = g + 8 * i;
+                            x0[i] = ldg_stream128(row0 + 16 * c, act0 && c < p.nchunks);
+                            x1[i] = ldg_stream128(row1 + 16 * c, act1 && c < p.nchunks);
+                        }
                     }
                     av0 = ldg_stream32(row0 + p.attr_off + 4 * ga, act0 && g < p.m);
                     av1 = ldg_stream32(row1 + p.attr_off + 4 * ga, act1 && g < p.m);
@@ -334,6 +383,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                     BOA_SCHED_FENCE();        // every load of the pass is issued before its first use
 #pragma unroll
                     for (int i = 0; i < (CPL > 0 ? CPL : 1); ++i) {
+                        if (!EXACT && g + 8 * i >= p.nchunks) continue;
                         if (VT == 0) {
                             a0 = sq_acc4u(a0, x0[i], qreg[i]);
                             a1 = sq_acc4u(a1, x1[i], qreg[i]);
@@ -414,17 +464,14 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             const uint32_t h = (id * 0x9E3779B1u) & id_mask;
             const uint32_t tag = h & tag_mask;
             const uint32_t bucket = h >> p.tag_bits;
-            const uint2 b = *reinterpret_cast<const uint2*>(hash + 4 * bucket);
+            uint2* slot = reinterpret_cast<uint2*>(hash + 4 * bucket);
+            const uint2 b = *slot;
             const uint32_t w0 = b.x & 0xFFFFu, w1 = b.x >> 16, w2 = b.y & 0xFFFFu, w3 = b.y >> 16;
             const bool found = (w0 == tag) | (w1 == tag) | (w2 == tag) | (w3 == tag);
-            uint32_t way = (id ^ (id >> 7)) & 3u;
-            way = (w3 == 0xFFFFu) ? 3u : way;
-            way = (w2 == 0xFFFFu) ? 2u : way;
-            way = (w1 == 0xFFFFu) ? 1u : way;
-            way = (w0 == 0xFFFFu) ? 0u : way;
             // a tag of 0xFFFF would look like an empty way: such an id is never recorded
             const bool fresh = !found | (tag == 0xFFFFu);
-            if (fresh && tag != 0xFFFFu) hash[4 * bucket + way] = (uint16_t)tag;
+            // first in, first out: the new tag enters at way 0, the oldest way falls off
+            if (fresh && tag != 0xFFFFu) *slot = make_uint2((b.x << 16) | tag, (b.y << 16) | w1);
             return fresh;
         };
         // first unexpanded entry at or after `from` among the first `lim`, or -1
@@ -543,6 +590,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
 #pragma unroll
                 for (int s = 0; s < RS; ++s) {
                     const uint64_t xs = x[s] >> 1;
+                    const uint64_t xo = x[s] | 1ull;        // key order ignoring the expanded bit
                     const bool valid = x[s] != kKeyMax;
                     int lo_i = 0, hi_i = valid ? n : 0;
                     for (int it = 0; it < trips; ++it) {
@@ -550,10 +598,10 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                         const bool on = len > 0;
                         const int q1 = lo_i + (len >> 2), q2 = lo_i + (len >> 1);
                         const int q3 = lo_i + ((3 * len) >> 2);
-                        const uint64_t k1 = pool[on ? q1 : 0] >> 1;
-                        const uint64_t k2 = pool[on ? q2 : 0] >> 1;
-                        const uint64_t k3 = pool[on ? q3 : 0] >> 1;
-                        const bool c1 = k1 < xs, c2 = k2 < xs, c3 = k3 < xs;
+                        const uint64_t k1 = pool[on ? q1 : 0] | 1ull;
+                        const uint64_t k2 = pool[on ? q2 : 0] | 1ull;
+                        const uint64_t k3 = pool[on ? q3 : 0] | 1ull;
+                        const bool c1 = k1 < xo, c2 = k2 < xo, c3 = k3 < xo;
                         const int nlo = c3 ? q3 + 1 : (c2 ? q2 + 1 : (c1 ? q1 + 1 : lo_i));
                         const int nhi = c3 ? hi_i : (c2 ? q3 : (c1 ? q2 : q1));
                         lo_i = on ? nlo : lo_i;
