@@ -3,8 +3,8 @@
 // into its epilogue.  sm_100a only.
 //
 // One warp (one CTA of 32 threads) owns one query from start to convergence.  Its
-// candidate pool, the table of recently scored ids, the query vector and a staging
-// area for neighbour records live in shared memory.  A pool entry is one 64-bit key
+// candidate pool, the table of recently scored ids and the query vector live in
+// shared memory.  A pool entry is one 64-bit key
 //     [63:60] phi (violated predicates)  [59:29] fp32 bits of d^2  [28:1] id  [0] expanded
 // so that integer order of keys is the lexicographic order (phi, d^2, id): the
 // lambda -> infinity reading of the paper's score dist + lambda*phi.
@@ -30,8 +30,8 @@
 // Distances are accumulated in a fixed order: a row is cut into 16-byte chunks,
 // chunk c belongs to lane (c mod 8) of an 8-lane group, each lane runs
 // acc = fmaf(x-q, x-q, acc) over its chunks in ascending order, and the eight
-// partial sums meet in a butterfly (xor 4, 2, 1).  Four neighbours are scored per
-// warp round, one per 8-lane group.
+// partial sums meet in a butterfly (xor 4, 2, 1).  Eight neighbours are scored per
+// warp pass, two per 8-lane group sharing one butterfly.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -50,9 +50,10 @@ constexpr uint64_t kKeyMax = ~0ull;
 
 enum : uint32_t { kStatusCopyTimeout = 1u };   // reserved: no wait in the kernel can time out
 
-// Optional per-section cycle counters (build with -DBOA_SECTION_TIMERS; off in the product).
 // Keeps the compiler from moving code across this point.
 #define BOA_SCHED_FENCE() asm volatile("" ::: "memory")
+
+// Optional per-section cycle counters (build with -DBOA_SECTION_TIMERS; off in the product).
 
 #ifdef BOA_SECTION_TIMERS
 #define BOA_T_DECL long long t_prev_ = clock64(); long long t_acc_[12] = {0}
