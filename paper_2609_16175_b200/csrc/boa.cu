@@ -227,17 +227,18 @@ typedef void (*SearchKernel)(const boa::SearchParams);
 struct KernelChoice {
     SearchKernel fn;
     int rs;
+    bool q_in_smem;     // the generic-length kernels keep the query in shared memory
 };
 
 template <int VT, int CPL>
 KernelChoice pick_rs(int R, bool exact)
 {
     if (R <= 32) {
-        if (exact) return {boa::boa_search_kernel<VT, 1, CPL, (CPL > 0)>, 1};
-        return {boa::boa_search_kernel<VT, 1, CPL, false>, 1};
+        if (exact) return {boa::boa_search_kernel<VT, 1, CPL, (CPL > 0)>, 1, CPL == 0};
+        return {boa::boa_search_kernel<VT, 1, CPL, false>, 1, CPL == 0};
     }
-    if (exact) return {boa::boa_search_kernel<VT, 2, CPL, (CPL > 0)>, 2};
-    return {boa::boa_search_kernel<VT, 2, CPL, false>, 2};
+    if (exact) return {boa::boa_search_kernel<VT, 2, CPL, (CPL > 0)>, 2, CPL == 0};
+    return {boa::boa_search_kernel<VT, 2, CPL, false>, 2, CPL == 0};
 }
 
 KernelChoice pick_kernel(const boa_index* ix)
@@ -359,7 +360,7 @@ int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_p
     sp.out_list = ix->lists + (size_t)(p + 1 < BOA_MAX_PHASES ? p + 1 : p) * ix->ws_Q;
     sp.out_count = ix->counters + kCntCount + p + 1;
 
-    const boa::WarpSmem lay = boa::warp_smem_layout(sp.C, sp.hash_log2, ix->D, lp.kc.rs);
+    const boa::WarpSmem lay = boa::warp_smem_layout(sp.C, sp.hash_log2, ix->D, lp.kc.rs, lp.kc.q_in_smem);
     const size_t smem = (size_t)lay.total;
     if (smem > 48 * 1024) {
         BOA_CUDA(cudaFuncSetAttribute((const void*)lp.kc.fn, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -262,13 +262,15 @@ __device__ __forceinline__ void sort_keys(uint64_t (&x)[RS], int lane)
 struct WarpSmem {
     int pool_off, nk_off, nr_off, cand_off, hash_off, q_off, total;
 };
-__host__ __device__ inline WarpSmem warp_smem_layout(int C, int hash_log2, int D, int RS)
+// q_in_smem: the query vector is kept in shared memory (only when lanes do not hold their
+// slices of it in registers).
+__host__ __device__ inline WarpSmem warp_smem_layout(int C, int hash_log2, int D, int RS, bool q_in_smem)
 {
     WarpSmem s;
     int off = 0;
     s.pool_off = off;  off += ((C + 1) & ~1) * 8;
     s.nk_off = off;    off += 32 * RS * 8;
-    s.q_off = off;     off += ((D * 4 + 15) & ~15);
+    s.q_off = off;     off += q_in_smem ? ((D * 4 + 15) & ~15) : 0;
     s.hash_off = off;  off += (1 << hash_log2) * 2;
     s.cand_off = off;  off += 32 * RS * 4;
     s.nr_off = off;    off += 32 * RS * 4;
@@ -293,7 +295,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
     constexpr int QF4 = (VT == 0) ? 1 : 4;          // float4 slices of the query per chunk
     constexpr int NQ = (CPL > 0) ? CPL * QF4 : 1;
 
-    const WarpSmem lay = warp_smem_layout(p.C, p.hash_log2, p.D, RS);
+    const WarpSmem lay = warp_smem_layout(p.C, p.hash_log2, p.D, RS, CPL == 0);
     uint64_t* pool = reinterpret_cast<uint64_t*>(smem_raw + lay.pool_off);
     uint64_t* nk = reinterpret_cast<uint64_t*>(smem_raw + lay.nk_off);
     uint32_t* nr = reinterpret_cast<uint32_t*>(smem_raw + lay.nr_off);
@@ -324,8 +326,10 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
 
         // ---- load the query, its bounds; clear the table of scored ids
         {
-            const float4* qsrc = reinterpret_cast<const float4*>(p.queries + (size_t)qi * p.D);
-            for (int i = lane; i < p.D / 4; i += 32) qs[i] = qsrc[i];
+            if (CPL == 0) {
+                const float4* qsrc = reinterpret_cast<const float4*>(p.queries + (size_t)qi * p.D);
+                for (int i = lane; i < p.D / 4; i += 32) qs[i] = qsrc[i];
+            }
             const uint4 ff = make_uint4(~0u, ~0u, ~0u, ~0u);
             uint4* h4 = reinterpret_cast<uint4*>(hash);
             for (int i = lane; i < (1 << p.hash_log2) / 8; i += 32) h4[i] = ff;
@@ -339,12 +343,13 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
         __syncwarp();
         float4 qreg[NQ];           // this lane's slices of the query (CPL > 0)
         if (CPL > 0) {
+            const float4* qsrc = reinterpret_cast<const float4*>(p.queries + (size_t)qi * p.D);
 #pragma unroll
             for (int i = 0; i < (CPL > 0 ? CPL : 1); ++i) {
                 const int c = g + 8 * i;
 #pragma unroll
                 for (int f = 0; f < QF4; ++f)
-                    qreg[i * QF4 + f] = (c < p.nchunks) ? qs[c * QF4 + f] : make_float4(0.f, 0.f, 0.f, 0.f);
+                    qreg[i * QF4 + f] = (c < p.nchunks) ? __ldg(qsrc + c * QF4 + f) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
         }
 
