@@ -1,0 +1,63 @@
+"""Kernel variants the five benchmark shapes do not reach: row lengths that are not a
+multiple of eight 16-byte chunks, long generic rows, uint8 rows of odd chunk counts, the
+largest attribute count, degree and beamwidth, odd degrees.  Random small inputs, both
+modes, bit parity with the oracle's fixed-order fp32 distances."""
+import numpy as np
+import pytest
+
+from boa_synth import SENTINEL, clean_rows, exact_knn_graph
+from tests.helpers import assert_bit_parity, gpu_search, make_pair
+
+pytestmark = pytest.mark.gpu
+
+
+def _random_case(seed, N, D, dtype, m, R, Q, float_cols=()):
+    rng = np.random.default_rng(seed)
+    if dtype == "u8":
+        x = rng.integers(0, 256, size=(N, D)).astype(np.uint8)
+        q = rng.integers(0, 256, size=(Q, D)).astype(np.float32)
+    else:
+        x = rng.standard_normal((N, D)).astype(np.float32)
+        q = rng.standard_normal((Q, D)).astype(np.float32)
+    attrs = rng.integers(0, 1000, size=(N, m)).astype(np.int32)
+    types = np.zeros(m, dtype=np.int32)
+    lo = rng.integers(0, 400, size=(Q, m)).astype(np.int32)
+    hi = (lo + rng.integers(300, 900, size=(Q, m))).astype(np.int32)
+    for j in float_cols:
+        types[j] = 1
+        attrs[:, j] = rng.random(N, dtype=np.float32).view(np.int32)
+        l = (0.4 * rng.random(Q)).astype(np.float32)
+        lo[:, j] = l.view(np.int32)
+        hi[:, j] = (l + np.float32(0.5)).astype(np.float32).view(np.int32)
+    near = exact_knn_graph(x.astype(np.float32), max(1, R - 2), device="cpu")
+    far = rng.integers(0, N, size=(N, R - near.shape[1])).astype(np.uint32)
+    g = clean_rows(np.concatenate([near, far], 1)[:, :R])
+    return dict(vectors=x, attrs=attrs, attr_types=types, graph=g, queries=q, lo=lo, hi=hi)
+
+
+CASES = [
+    # name,           N,    D,  dtype, m, R,  k, widths,          float columns
+    ("f32_5chunks",   3000, 20,  "f32", 2, 16, 5,  [8, 32, 64],    ()),
+    ("f32_25chunks",  3000, 100, "f32", 3, 32, 10, [16, 64],       (1,)),
+    ("f32_50chunks",  2500, 200, "f32", 2, 24, 10, [16, 128],      ()),
+    ("f32_1chunk",    2000, 4,   "f32", 1, 7,  3,  [4, 16],        ()),
+    ("u8_3chunks",    3000, 48,  "u8",  2, 16, 10, [16, 64],       ()),
+    ("u8_17chunks",   2500, 272, "u8",  2, 40, 10, [16, 64],       ()),
+    ("u8_12chunks",   2500, 192, "u8",  4, 33, 10, [12, 100],      (3,)),
+    ("max_attrs_deg", 4000, 64,  "f32", 8, 64, 10, [16, 256, 1024], (0, 5)),
+]
+
+
+@pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
+def test_shape_variants_match_oracle(case):
+    name, N, D, dtype, m, R, k, widths, fcols = case
+    d = _random_case(sum(map(ord, name)), N, D, dtype, m, R, 48, fcols)
+    orc, gpu, g = make_pair(d)
+    assert orc.entry == gpu.entry
+    for mode in ("restart", "resume"):
+        for eps in (0.05, 0.3):
+            o = orc.search(d["queries"], d["lo"], d["hi"], k, widths, eps=eps, mode=mode, dist_mode=1)
+            r = gpu_search(gpu, g, k, widths, mode=mode, eps=eps)
+            assert_bit_parity(o, r, f"{name}/{mode}/eps={eps}")
+    assert (r["ids"] != SENTINEL).any()
+    gpu.close()
