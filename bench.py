@@ -99,7 +99,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-i", str(self.index), "-lms", "100"],
+                 "-i", str(self.index), "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
@@ -307,7 +307,6 @@ def main():
     barrier()
     total_ms = ev[0].elapsed_time(ev[-1])
     step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
-    clocks = sampler.stop() if rank == 0 else None
     launches = ix.last_launch_count * args.steps
     ms_per_step = max_over_ranks(total_ms, dev, world) / args.steps
     value = whole_job_value(Q, world, ms_per_step)
@@ -320,6 +319,7 @@ def main():
 
     if args.no_extras:
         if rank == 0:
+            sampler.stop()
             print(json.dumps({"ms_per_step": ms_per_step, "value": value, "hash_log2": args.hash_log2,
                               "schedule": widths, "mode": args.mode,
                               "plus_k": args.plus_k, "mean_scored": float(st["n_scored"].mean()),
@@ -353,6 +353,7 @@ def main():
     e1.record()
     torch.cuda.synchronize()
     barrier()
+    clocks = sampler.stop() if rank == 0 else None     # sampled over both timed regions
     e2e_value = whole_job_value(Q, world, max_over_ranks(e0.elapsed_time(e1), dev, world) / args.steps)
     h2d = hq.numel() * 4 + hlo.numel() * 4 + hhi.numel() * 4
     d2h = h_ids.numel() * 4 + h_d2.numel() * 4

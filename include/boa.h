@@ -174,9 +174,11 @@ int boa_workspace_bytes(const boa_index* index, int64_t Q, int Lmax, size_t* byt
 /* Number of kernel launches the last boa_search enqueued. */
 int boa_last_launch_count(const boa_index* index);
 
-/* Device-side status of the last search on this index (HOST int, synchronises
-   `stream`): 0 = fine; bit 0 = an asynchronous copy did not complete within its bounded
-   wait, the affected launches stopped early and their outputs are incomplete. */
+/* Device-side status word of the last search on this index (HOST int, synchronises
+   `stream`): 0 = fine.  The search kernel has no wait on a flag, barrier or peer and
+   every loop in it is bounded by the expansion cap, so no bit is raised today; the word
+   is where a kernel that has to give up would say so (bit 0 is reserved for "a wait
+   timed out, outputs of the affected launches are incomplete"). */
 int boa_device_status(boa_index* index, int* status, void* stream);
 
 /* cudaError_t of the most recent failing CUDA call made by this library (0 if none). */
