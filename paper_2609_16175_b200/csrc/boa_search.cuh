@@ -584,36 +584,42 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                     if (x[0] != kKeyMax) nk[r] = x[0];
                     __syncwarp();
                     x[0] = (lane < live) ? nk[lane] : kKeyMax;
-                } else if (live > 1) {
+                } else {   // also for a single key: it has to end up in lane 0
                     sort_keys<RS>(x, lane);
                 }
                 BOA_T_MARK(7);
 
-                // rank of every new key in the pool (4-ary search, same trip count for all
-                // lanes, selects instead of branches); drop keys the pool already holds
-                int trips = 0;
-                for (int span = n; span > 0; span >>= 2) ++trips;
+                // rank of every new key in the pool, found by the whole warp for one key at
+                // a time: lane l holds the last key of the l-th block of `stride` pool entries;
+                // one ballot finds the block, a second one the place inside it.  Keys the
+                // pool already holds (same key, expanded or not) are dropped.
+                const int stride = (n + 31) >> 5;
+                const int pend = ((lane + 1) * stride < n) ? (lane + 1) * stride : n;
+                const uint64_t piv = (lane * stride < n) ? (pool[pend - 1] | 1ull) : kKeyMax;
+                int rank_s[RS];
+                bool dup_s[RS];
+#pragma unroll
+                for (int s = 0; s < RS; ++s) { rank_s[s] = 0; dup_s[s] = false; }
+#pragma unroll 2
+                for (int j = 0; j < live; ++j) {
+                    const uint64_t xsrc = (RS == 2 && j >= 32) ? x[RS - 1] : x[0];
+                    const uint64_t xj = __shfl_sync(0xffffffffu, xsrc, j & 31) | 1ull;
+                    const int base = __popc(__ballot_sync(0xffffffffu, piv < xj)) * stride;
+                    const int idx = base + lane;
+                    const uint64_t e = (lane < stride && idx < n) ? (pool[idx] | 1ull) : kKeyMax;
+                    int r = base + __popc(__ballot_sync(0xffffffffu, e < xj));
+                    r = r < n ? r : n;
+                    const bool dj = __ballot_sync(0xffffffffu, e == xj) != 0u;
+                    if ((j & 31) == lane) {
+                        if (RS == 2 && j >= 32) { rank_s[RS - 1] = r; dup_s[RS - 1] = dj; }
+                        else { rank_s[0] = r; dup_s[0] = dj; }
+                    }
+                }
 #pragma unroll
                 for (int s = 0; s < RS; ++s) {
-                    const uint64_t xs = x[s] >> 1;
-                    const uint64_t xo = x[s] | 1ull;        // key order ignoring the expanded bit
                     const bool valid = x[s] != kKeyMax;
-                    int lo_i = 0, hi_i = valid ? n : 0;
-                    for (int it = 0; it < trips; ++it) {
-                        const int len = hi_i - lo_i;
-                        const bool on = len > 0;
-                        const int q1 = lo_i + (len >> 2), q2 = lo_i + (len >> 1);
-                        const int q3 = lo_i + ((3 * len) >> 2);
-                        const uint64_t k1 = pool[on ? q1 : 0] | 1ull;
-                        const uint64_t k2 = pool[on ? q2 : 0] | 1ull;
-                        const uint64_t k3 = pool[on ? q3 : 0] | 1ull;
-                        const bool c1 = k1 < xo, c2 = k2 < xo, c3 = k3 < xo;
-                        const int nlo = c3 ? q3 + 1 : (c2 ? q2 + 1 : (c1 ? q1 + 1 : lo_i));
-                        const int nhi = c3 ? hi_i : (c2 ? q3 : (c1 ? q2 : q1));
-                        lo_i = on ? nlo : lo_i;
-                        hi_i = on ? nhi : hi_i;
-                    }
-                    const bool dup = valid && (lo_i < n) && ((pool[lo_i] >> 1) == xs);
+                    const int lo_i = rank_s[s];
+                    const bool dup = valid && dup_s[s];
                     const bool nd = valid && !dup;
                     const unsigned bal = __ballot_sync(0xffffffffu, nd);
                     const int pidx = kept + __popc(bal & lt_mask);
@@ -673,25 +679,55 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             // top first, each in 32-entry chunks from its top end; the next chunk is read
             // before the current one is written (its slots are never a write target).
             {
-                for (int j = kept - 1; j >= 0; --j) {
-                    const int a = (int)nr[j];
-                    const int bnd = (j == kept - 1) ? n : (int)nr[j + 1];
-                    if (bnd <= a) continue;
-                    const int sft = j + 1;
-                    int lo_c = (bnd - 32 > a) ? bnd - 32 : a;
-                    int i = lo_c + lane;
-                    bool v = i < bnd;
-                    uint64_t e = v ? pool[i] : 0ull;
-                    for (;;) {
+                if (kept <= 8) {
+                    // few new keys: every moved entry counts the new ranks at or before it;
+                    // four 32-entry chunks are read, then written, top chunks first (a write
+                    // never lands below the chunk it came from)
+                    int nrr[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) nrr[j] = (j < kept) ? (int)nr[j] : 0x7FFFFFFF;
+                    const int top = (n - 1) >> 5, bot = rmin >> 5;
+                    for (int ct = top; ct >= bot; ct -= 4) {
+                        uint64_t e[4];
+                        int dst[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int c = ct - u;
+                            const int i = c * 32 + lane;
+                            const bool ok = (c >= bot) && (i < n) && (i >= rmin);
+                            e[u] = ok ? pool[i] : 0ull;
+                            int sh = 0;
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) sh += (nrr[j] <= i) ? 1 : 0;
+                            dst[u] = ok ? i + sh : p.C;
+                        }
                         __syncwarp();
-                        const int hi2 = lo_c;
-                        const int lo2 = (hi2 - 32 > a) ? hi2 - 32 : a;
-                        const int i2 = lo2 + lane;
-                        const bool v2 = (hi2 > a) && (i2 < hi2);
-                        const uint64_t e2 = v2 ? pool[i2] : 0ull;
-                        if (v && i + sft < p.C) pool[i + sft] = e;
-                        if (hi2 <= a) break;
-                        lo_c = lo2; i = i2; v = v2; e = e2;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (dst[u] < p.C) pool[dst[u]] = e[u];
+                        __syncwarp();
+                    }
+                } else {
+                    for (int j = kept - 1; j >= 0; --j) {
+                        const int a = (int)nr[j];
+                        const int bnd = (j == kept - 1) ? n : (int)nr[j + 1];
+                        if (bnd <= a) continue;
+                        const int sft = j + 1;
+                        int lo_c = (bnd - 32 > a) ? bnd - 32 : a;
+                        int i = lo_c + lane;
+                        bool v = i < bnd;
+                        uint64_t e = v ? pool[i] : 0ull;
+                        for (;;) {
+                            __syncwarp();
+                            const int hi2 = lo_c;
+                            const int lo2 = (hi2 - 32 > a) ? hi2 - 32 : a;
+                            const int i2 = lo2 + lane;
+                            const bool v2 = (hi2 > a) && (i2 < hi2);
+                            const uint64_t e2 = v2 ? pool[i2] : 0ull;
+                            if (v && i + sft < p.C) pool[i + sft] = e;
+                            if (hi2 <= a) break;
+                            lo_c = lo2; i = i2; v = v2; e = e2;
+                        }
                     }
                 }
                 __syncwarp();
