@@ -35,11 +35,25 @@ def filtered_topk(vectors: torch.Tensor, attrs: torch.Tensor, attr_types, querie
         d = (xn[None, :] + (q.double() ** 2).sum(1)[:, None]).to(torch.float64)
         d -= 2.0 * torch.mm(q, x.t()).double()
         d.masked_fill_(~ok, float("inf"))
+        # the expansion |x|^2 + |q|^2 - 2xq in fp32 loses digits on small distances: take a
+        # few candidates more than k, recompute their distances directly in double, re-rank
         kk = min(k, n)
-        top = torch.topk(d, kk, dim=1, largest=False, sorted=True)
-        fin = torch.isfinite(top.values)
-        ids[s:e, :kk] = torch.where(fin, top.indices, torch.full_like(top.indices, -1))
-        d2[s:e, :kk] = top.values
+        kc = min(k + 16, n)
+        cand = torch.topk(d, kc, dim=1, largest=False, sorted=True)
+        fin = torch.isfinite(cand.values)
+        diff = x[cand.indices].double() - q.double()[:, None, :]
+        exact = (diff * diff).sum(-1)
+        exact.masked_fill_(~fin, float("inf"))
+        # order by (distance, id)
+        order = torch.argsort(cand.indices, dim=1, stable=True)
+        exact_o = torch.gather(exact, 1, order)
+        idx_o = torch.gather(cand.indices, 1, order)
+        order2 = torch.argsort(exact_o, dim=1, stable=True)
+        exact_s = torch.gather(exact_o, 1, order2)[:, :kk]
+        idx_s = torch.gather(idx_o, 1, order2)[:, :kk]
+        fin_s = torch.isfinite(exact_s)
+        ids[s:e, :kk] = torch.where(fin_s, idx_s, torch.full_like(idx_s, -1))
+        d2[s:e, :kk] = exact_s
         nvalid[s:e] = ok.sum(1)
     return ids, d2, nvalid
 

@@ -416,3 +416,25 @@ def test_expansion_cap_is_honoured(small):
     w, d, ix = small
     r = ix.search(d["queries"], d["lo"], d["hi"], 10, [64], cap=(0, 5))
     assert (r["n_expand"] <= 5).all() and (r["flags"] & 1).any()
+
+
+# ----------------------------------------------------------------------------
+# the harness's blocked brute force (used for recall on large batches) against the oracle's
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("which", ["small", "small_float"])
+def test_harness_ground_truth_equals_oracle_bruteforce(which, request):
+    from boa_synth.groundtruth import filtered_topk, recall_against
+    w, d, ix = request.getfixturevalue(which)
+    t = {k: torch.from_numpy(d[k]) for k in ("vectors", "attrs", "queries", "lo", "hi")}
+    ids, d2, nv = filtered_topk(t["vectors"], t["attrs"], d["attr_types"], t["queries"], t["lo"],
+                                t["hi"], 10, block=16)
+    o_ids, o_d2, o_nv = ix.bruteforce(d["queries"], d["lo"], d["hi"], 10)
+    assert (nv.numpy() == o_nv).all()
+    fin = o_ids != SENTINEL
+    np.testing.assert_allclose(d2.numpy()[fin], o_d2[fin], rtol=1e-12)
+    assert (ids.numpy()[fin] == o_ids[fin].astype(np.int64)).all()
+    # an exact answer scores recall 1, a shifted one less
+    rec = recall_against(o_ids, o_d2.astype(np.float32), d2.numpy(), nv.numpy(), 10, rel=1e-5)
+    assert np.nanmin(rec) == 1.0
+    worse = recall_against(o_ids, (o_d2 * 4.0 + 1.0).astype(np.float32), d2.numpy(), nv.numpy(), 10)
+    assert np.nanmean(worse) < 0.5
