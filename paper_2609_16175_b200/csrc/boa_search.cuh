@@ -476,8 +476,12 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             const bool found = (w0 == tag) | (w1 == tag) | (w2 == tag) | (w3 == tag);
             // a tag of 0xFFFF would look like an empty way: such an id is never recorded
             const bool fresh = !found | (tag == 0xFFFFu);
-            // first in, first out: the new tag enters at way 0, the oldest way falls off
-            if (fresh && tag != 0xFFFFu) *slot = make_uint2((b.x << 16) | tag, (b.y << 16) | w1);
+            // least recently met first out: the tag moves (or enters) to way 0, the ways
+            // before its old place move up by one, a new tag pushes the last way out
+            if (tag != 0xFFFFu && w0 != tag) {
+                const uint32_t hi = (w1 == tag) ? b.y : (w1 | (((w2 == tag) ? w3 : w2) << 16));
+                *slot = make_uint2(tag | (w0 << 16), hi);
+            }
             return fresh;
         };
         // first unexpanded entry at or after `from` among the first `lim`, or -1
@@ -620,6 +624,9 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                     const bool valid = x[s] != kKeyMax;
                     const int lo_i = rank_s[s];
                     const bool dup = valid && dup_s[s];
+#ifdef BOA_SECTION_TIMERS
+                    t_acc_[11] += __popc(__ballot_sync(0xffffffffu, dup));   // keys found again in the pool
+#endif
                     const bool nd = valid && !dup;
                     const unsigned bal = __ballot_sync(0xffffffffu, nd);
                     const int pidx = kept + __popc(bal & lt_mask);
