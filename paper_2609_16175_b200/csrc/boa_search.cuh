@@ -560,6 +560,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             uint64_t x[RS];
             bool keep[RS];
             int pos_new[RS];
+            int rank_s[RS];
             if (cnt > 0) {
                 n_sc += cnt;
                 // gather + distance + range check (fused)
@@ -597,26 +598,49 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                 // a time: lane l holds the last key of the l-th block of `stride` pool entries;
                 // one ballot finds the block, a second one the place inside it.  Keys the
                 // pool already holds (same key, expanded or not) are dropped.
-                const int stride = (n + 31) >> 5;
-                const int pend = ((lane + 1) * stride < n) ? (lane + 1) * stride : n;
-                const uint64_t piv = (lane * stride < n) ? (pool[pend - 1] | 1ull) : kKeyMax;
-                int rank_s[RS];
                 bool dup_s[RS];
 #pragma unroll
                 for (int s = 0; s < RS; ++s) { rank_s[s] = 0; dup_s[s] = false; }
+                if (live <= 10) {
+                    const int stride = (n + 31) >> 5;
+                    const int pend = ((lane + 1) * stride < n) ? (lane + 1) * stride : n;
+                    const uint64_t piv = (lane * stride < n) ? (pool[pend - 1] | 1ull) : kKeyMax;
 #pragma unroll 2
-                for (int j = 0; j < live; ++j) {
-                    const uint64_t xsrc = (RS == 2 && j >= 32) ? x[RS - 1] : x[0];
-                    const uint64_t xj = __shfl_sync(0xffffffffu, xsrc, j & 31) | 1ull;
-                    const int base = __popc(__ballot_sync(0xffffffffu, piv < xj)) * stride;
-                    const int idx = base + lane;
-                    const uint64_t e = (lane < stride && idx < n) ? (pool[idx] | 1ull) : kKeyMax;
-                    int r = base + __popc(__ballot_sync(0xffffffffu, e < xj));
-                    r = r < n ? r : n;
-                    const bool dj = __ballot_sync(0xffffffffu, e == xj) != 0u;
-                    if ((j & 31) == lane) {
-                        if (RS == 2 && j >= 32) { rank_s[RS - 1] = r; dup_s[RS - 1] = dj; }
-                        else { rank_s[0] = r; dup_s[0] = dj; }
+                    for (int j = 0; j < live; ++j) {
+                        const uint64_t xj = __shfl_sync(0xffffffffu, x[0], j) | 1ull;
+                        const int base = __popc(__ballot_sync(0xffffffffu, piv < xj)) * stride;
+                        const int idx = base + lane;
+                        const uint64_t e = (lane < stride && idx < n) ? (pool[idx] | 1ull) : kKeyMax;
+                        int r = base + __popc(__ballot_sync(0xffffffffu, e < xj));
+                        r = r < n ? r : n;
+                        const bool dj = __ballot_sync(0xffffffffu, e == xj) != 0u;
+                        if (j == lane) { rank_s[0] = r; dup_s[0] = dj; }
+                    }
+                } else {
+                    // many keys: every lane searches for its own (4-ary, same trip count for
+                    // all lanes, selects instead of branches)
+                    int trips = 0;
+                    for (int span = n; span > 0; span >>= 2) ++trips;
+#pragma unroll
+                    for (int s = 0; s < RS; ++s) {
+                        const uint64_t xo = x[s] | 1ull;
+                        int lo_i = 0, hi_i = (x[s] != kKeyMax) ? n : 0;
+                        for (int it = 0; it < trips; ++it) {
+                            const int len = hi_i - lo_i;
+                            const bool on = len > 0;
+                            const int q1 = lo_i + (len >> 2), q2 = lo_i + (len >> 1);
+                            const int q3 = lo_i + ((3 * len) >> 2);
+                            const uint64_t k1 = pool[on ? q1 : 0] | 1ull;
+                            const uint64_t k2 = pool[on ? q2 : 0] | 1ull;
+                            const uint64_t k3 = pool[on ? q3 : 0] | 1ull;
+                            const bool c1 = k1 < xo, c2 = k2 < xo, c3 = k3 < xo;
+                            const int nlo = c3 ? q3 + 1 : (c2 ? q2 + 1 : (c1 ? q1 + 1 : lo_i));
+                            const int nhi = c3 ? hi_i : (c2 ? q3 : (c1 ? q2 : q1));
+                            lo_i = on ? nlo : lo_i;
+                            hi_i = on ? nhi : hi_i;
+                        }
+                        rank_s[s] = lo_i;
+                        dup_s[s] = (lo_i < n) && ((pool[lo_i] | 1ull) == xo);
                     }
                 }
 #pragma unroll
@@ -632,11 +656,8 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                     const int pidx = kept + __popc(bal & lt_mask);
                     pos_new[s] = lo_i + pidx;
                     keep[s] = nd && (pos_new[s] < p.C);
-                    const unsigned kb = __ballot_sync(0xffffffffu, keep[s]);
-                    if (keep[s]) nr[pidx] = (uint32_t)lo_i;
-                    kept += __popc(kb);
+                    kept += __popc(__ballot_sync(0xffffffffu, keep[s]));
                 }
-                __syncwarp();
                 BOA_T_MARK(8);
             }
             if (kept == 0) {
@@ -644,7 +665,17 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                 pos = first_unexpanded(cur, n < p.L ? n : p.L);
                 continue;
             }
-            const int rmin = (int)nr[0];
+            // smallest rank among the kept keys = rank of the first kept key; and that key
+            int rmin = 0;
+            uint64_t first_new = 0;
+#pragma unroll
+            for (int s = RS - 1; s >= 0; --s) {
+                const unsigned kb = __ballot_sync(0xffffffffu, keep[s]);
+                if (kb) {
+                    rmin = __shfl_sync(0xffffffffu, rank_s[s], __ffs(kb) - 1);
+                    first_new = __shfl_sync(0xffffffffu, x[s], __ffs(kb) - 1);
+                }
+            }
 
             // ---- which node is expanded next?  Decide on the pool as it is, translate the
             // position, and start loading that node's adjacency row before the merge.
@@ -652,8 +683,10 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                 const int pos_old = first_unexpanded(cur, n < p.L ? n : p.L);
                 int pos_old_new = -1;
                 if (pos_old >= 0) {
-                    int sh = 0;
-                    for (int j = 0; j < kept; ++j) sh += ((int)nr[j] <= pos_old) ? 1 : 0;
+                    int sh = 0;                       // kept keys ranked at or before it
+#pragma unroll
+                    for (int s = 0; s < RS; ++s)
+                        sh += __popc(__ballot_sync(0xffffffffu, keep[s] && rank_s[s] <= pos_old));
                     pos_old_new = pos_old + sh;
                 }
                 const int n_new = (n + kept < p.C) ? n + kept : p.C;
@@ -662,12 +695,6 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                 uint32_t next_id;
                 if (pos_old_new < 0 || rmin < pos_old_new) {
                     next_pos = rmin;                         // the smallest new key comes first
-                    uint64_t first_new = 0;
-#pragma unroll
-                    for (int s = RS - 1; s >= 0; --s) {
-                        const unsigned kb = __ballot_sync(0xffffffffu, keep[s]);
-                        if (kb) first_new = __shfl_sync(0xffffffffu, x[s], __ffs(kb) - 1);
-                    }
                     next_id = key_id(first_new);
                 } else {
                     next_pos = pos_old_new;
@@ -681,67 +708,55 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                 }
             }
 
-            // ---- merge.  The pool entries between two consecutive new keys all move up by
-            // the same amount: segment j = [rank_j, rank_{j+1}) moves by j+1.  Segments go
-            // top first, each in 32-entry chunks from its top end; the next chunk is read
-            // before the current one is written (its slots are never a write target).
+            // ---- merge.  A bitmap marks the places the new keys take in the merged pool;
+            // every other place d receives the old entry d - (new places before d).  Places
+            // are filled four 32-entry chunks at a time, top chunks first, all reads of a
+            // group before its writes (a source never lies above its destination).
             {
-                if (kept <= 8) {
-                    // few new keys: every moved entry counts the new ranks at or before it;
-                    // four 32-entry chunks are read, then written, top chunks first (a write
-                    // never lands below the chunk it came from)
-                    int nrr[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) nrr[j] = (j < kept) ? (int)nr[j] : 0x7FFFFFFF;
-                    const int top = (n - 1) >> 5, bot = rmin >> 5;
-                    for (int ct = top; ct >= bot; ct -= 4) {
-                        uint64_t e[4];
-                        int dst[4];
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int c = ct - u;
-                            const int i = c * 32 + lane;
-                            const bool ok = (c >= bot) && (i < n) && (i >= rmin);
-                            e[u] = ok ? pool[i] : 0ull;
-                            int sh = 0;
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) sh += (nrr[j] <= i) ? 1 : 0;
-                            dst[u] = ok ? i + sh : p.C;
-                        }
-                        __syncwarp();
-#pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            if (dst[u] < p.C) pool[dst[u]] = e[u];
-                        __syncwarp();
-                    }
-                } else {
-                    for (int j = kept - 1; j >= 0; --j) {
-                        const int a = (int)nr[j];
-                        const int bnd = (j == kept - 1) ? n : (int)nr[j + 1];
-                        if (bnd <= a) continue;
-                        const int sft = j + 1;
-                        int lo_c = (bnd - 32 > a) ? bnd - 32 : a;
-                        int i = lo_c + lane;
-                        bool v = i < bnd;
-                        uint64_t e = v ? pool[i] : 0ull;
-                        for (;;) {
-                            __syncwarp();
-                            const int hi2 = lo_c;
-                            const int lo2 = (hi2 - 32 > a) ? hi2 - 32 : a;
-                            const int i2 = lo2 + lane;
-                            const bool v2 = (hi2 > a) && (i2 < hi2);
-                            const uint64_t e2 = v2 ? pool[i2] : 0ull;
-                            if (v && i + sft < p.C) pool[i + sft] = e;
-                            if (hi2 <= a) break;
-                            lo_c = lo2; i = i2; v = v2; e = e2;
-                        }
-                    }
-                }
+                uint32_t* occ = cand;                    // 32 words: places < 1024
+                uint32_t* pre = nr;                      // new places before each word
+                occ[lane] = 0u;
                 __syncwarp();
 #pragma unroll
                 for (int s = 0; s < RS; ++s)
+                    if (keep[s]) atomicOr(&occ[pos_new[s] >> 5], 1u << (pos_new[s] & 31));
+                __syncwarp();
+                {
+                    const int c_l = __popc(occ[lane]);
+                    int inc = c_l;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const int t = __shfl_up_sync(0xffffffffu, inc, o);
+                        if (lane >= o) inc += t;
+                    }
+                    pre[lane] = (uint32_t)(inc - c_l);
+                }
+                __syncwarp();
+                const int n_new = (n + kept < p.C) ? n + kept : p.C;
+                const int top = (n_new - 1) >> 5, bot = rmin >> 5;
+                for (int ct = top; ct >= bot; ct -= 4) {
+                    uint64_t e[4];
+                    bool wr[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int c = ct - u;
+                        const int cc = c >= bot ? c : bot;
+                        const int d = cc * 32 + lane;
+                        const uint32_t w = occ[cc];
+                        const int src = d - (int)pre[cc] - __popc(w & lt_mask);
+                        wr[u] = (c >= bot) && !((w >> lane) & 1u) && (d >= rmin) && (d < n_new) && (src != d);
+                        e[u] = wr[u] ? pool[src] : 0ull;
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (wr[u]) pool[(ct - u) * 32 + lane] = e[u];
+                    __syncwarp();
+                }
+#pragma unroll
+                for (int s = 0; s < RS; ++s)
                     if (keep[s]) pool[pos_new[s]] = x[s];
-                n = (n + kept < p.C) ? n + kept : p.C;
+                n = n_new;
                 if (rmin < cur) cur = rmin;
                 __syncwarp();
             }
