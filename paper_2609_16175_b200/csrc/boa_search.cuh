@@ -356,21 +356,51 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
         // Scores cand[0..cnt) straight from global memory: eight rows per pass, every lane
         // loads its own 16-byte chunks of two rows into registers (all loads of a pass are
         // issued before the first use), distance + violated predicates -> nk[0..cnt).
+        // reduce the two partial-sum sets of a pass, count violated predicates, write the keys
+        auto finish_pass = [&](int cnt, float a0, float a1, uint32_t av0, uint32_t av1, uint32_t id0,
+                               uint32_t id1, int j0, int j1, bool act0, bool act1) {
+            const bool hi4 = (lane & 4) != 0;
+            float v = hi4 ? a1 : a0;
+            const float w = hi4 ? a0 : a1;
+            v += __shfl_xor_sync(0xffffffffu, w, 4);
+            v += __shfl_xor_sync(0xffffffffu, v, 2);
+            v += __shfl_xor_sync(0xffffffffu, v, 1);
+            bool v0, v1;
+            if (my_float) {
+                const float l = __int_as_float(my_lo), h = __int_as_float(my_hi);
+                v0 = !(__uint_as_float(av0) >= l && __uint_as_float(av0) <= h);
+                v1 = !(__uint_as_float(av1) >= l && __uint_as_float(av1) <= h);
+            } else {
+                v0 = (int32_t)av0 < my_lo || (int32_t)av0 > my_hi;
+                v1 = (int32_t)av1 < my_lo || (int32_t)av1 > my_hi;
+            }
+            const unsigned bal0 = __ballot_sync(0xffffffffu, v0 && act0 && g < p.m);
+            const unsigned bal1 = __ballot_sync(0xffffffffu, v1 && act1 && g < p.m);
+            const unsigned bal = hi4 ? bal1 : bal0;
+            const int jj = hi4 ? j1 : j0;
+            if ((g & 3) == 0 && jj < cnt)
+                nk[jj] = pack_key(__popc((bal >> (8 * gi)) & 0xFFu), v, hi4 ? id1 : id0);
+        };
+
+        // Scores cand[0..cnt) straight from global memory: eight rows per pass, every lane
+        // loads its own 16-byte chunks of two rows into registers (all loads of a pass are
+        // issued before the first use), distance + violated predicates -> nk[0..cnt).  For
+        // short rows the loads of the next pass are issued as soon as the multiply-adds of
+        // this pass have freed the registers, before its reduction.
         auto score = [&](int cnt) {
             BOA_T_MARK(3);
-#pragma unroll 1
-            for (int r0 = 0; r0 < cnt; r0 += 8) {
-                BOA_SCHED_FENCE();
-                const int j0 = r0 + gi, j1 = r0 + 4 + gi;
-                const bool act0 = j0 < cnt, act1 = j1 < cnt;
-                const uint32_t id0 = cand[act0 ? j0 : 0], id1 = cand[act1 ? j1 : 0];
-                const uint8_t* row0 = p.rec + (size_t)id0 * p.rec_stride;
-                const uint8_t* row1 = p.rec + (size_t)id1 * p.rec_stride;
-                const int ga = (g < p.m) ? g : 0;
-                float a0 = 0.0f, a1 = 0.0f;
-                uint32_t av0, av1;
-                if (CPL > 0) {
-                    uint4 x0[CPL > 0 ? CPL : 1], x1[CPL > 0 ? CPL : 1];
+            const int ga = (g < p.m) ? g : 0;
+            if (CPL > 0) {
+                uint4 x0[CPL > 0 ? CPL : 1], x1[CPL > 0 ? CPL : 1];
+                uint32_t av0, av1, id0, id1;
+                bool act0, act1;
+                int j0, j1;
+                auto issue_pass = [&](int r0) {
+                    j0 = r0 + gi; j1 = r0 + 4 + gi;
+                    act0 = j0 < cnt; act1 = j1 < cnt;
+                    id0 = cand[act0 ? j0 : 0]; id1 = cand[act1 ? j1 : 0];
+                    const uint8_t* row0 = p.rec + (size_t)id0 * p.rec_stride;
+                    const uint8_t* row1 = p.rec + (size_t)id1 * p.rec_stride;
                     if (EXACT) {
                         // one predicate per row; chunk i sits 128 bytes after chunk i-1
                         ldg_chunks<(CPL > 0 ? CPL : 1)>(x0, row0 + 16 * g, act0);
@@ -385,8 +415,13 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                     }
                     av0 = ldg_stream32(row0 + p.attr_off + 4 * ga, act0 && g < p.m);
                     av1 = ldg_stream32(row1 + p.attr_off + 4 * ga, act1 && g < p.m);
+                };
+                issue_pass(0);
+#pragma unroll 1
+                for (int r0 = 0; r0 < cnt; r0 += 8) {
                     BOA_T_MARK(4);
                     BOA_SCHED_FENCE();        // every load of the pass is issued before its first use
+                    float a0 = 0.0f, a1 = 0.0f;
 #pragma unroll
                     for (int i = 0; i < (CPL > 0 ? CPL : 1); ++i) {
                         if (!EXACT && g + 8 * i >= p.nchunks) continue;
@@ -404,9 +439,26 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                             a1 = sq_acc_bytes(a1, x1[i].w, qreg[4 * i + 3]);
                         }
                     }
-                } else {
-                    av0 = ldg_stream32(row0 + p.attr_off + 4 * ga, act0 && g < p.m);
-                    av1 = ldg_stream32(row1 + p.attr_off + 4 * ga, act1 && g < p.m);
+                    const uint32_t c_av0 = av0, c_av1 = av1, c_id0 = id0, c_id1 = id1;
+                    const int c_j0 = j0, c_j1 = j1;
+                    const bool c_act0 = act0, c_act1 = act1;
+                    BOA_SCHED_FENCE();
+                    if (r0 + 8 < cnt) issue_pass(r0 + 8);
+                    BOA_SCHED_FENCE();
+                    finish_pass(cnt, a0, a1, c_av0, c_av1, c_id0, c_id1, c_j0, c_j1, c_act0, c_act1);
+                    BOA_T_MARK(6);
+                }
+            } else {
+#pragma unroll 1
+                for (int r0 = 0; r0 < cnt; r0 += 8) {
+                    const int j0 = r0 + gi, j1 = r0 + 4 + gi;
+                    const bool act0 = j0 < cnt, act1 = j1 < cnt;
+                    const uint32_t id0 = cand[act0 ? j0 : 0], id1 = cand[act1 ? j1 : 0];
+                    const uint8_t* row0 = p.rec + (size_t)id0 * p.rec_stride;
+                    const uint8_t* row1 = p.rec + (size_t)id1 * p.rec_stride;
+                    float a0 = 0.0f, a1 = 0.0f;
+                    const uint32_t av0 = ldg_stream32(row0 + p.attr_off + 4 * ga, act0 && g < p.m);
+                    const uint32_t av1 = ldg_stream32(row1 + p.attr_off + 4 * ga, act1 && g < p.m);
                     // long rows: four chunks of each row in flight per lane at a time
                     for (int c0 = g; c0 < p.nchunks; c0 += 32) {
                         uint4 x0[4], x1[4];
@@ -438,29 +490,9 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                         }
                     }
                     BOA_T_MARK(4);
+                    finish_pass(cnt, a0, a1, av0, av1, id0, id1, j0, j1, act0, act1);
+                    BOA_T_MARK(6);
                 }
-                const bool hi4 = (lane & 4) != 0;
-                float v = hi4 ? a1 : a0;
-                const float w = hi4 ? a0 : a1;
-                v += __shfl_xor_sync(0xffffffffu, w, 4);
-                v += __shfl_xor_sync(0xffffffffu, v, 2);
-                v += __shfl_xor_sync(0xffffffffu, v, 1);
-                bool v0, v1;
-                if (my_float) {
-                    const float l = __int_as_float(my_lo), h = __int_as_float(my_hi);
-                    v0 = !(__uint_as_float(av0) >= l && __uint_as_float(av0) <= h);
-                    v1 = !(__uint_as_float(av1) >= l && __uint_as_float(av1) <= h);
-                } else {
-                    v0 = (int32_t)av0 < my_lo || (int32_t)av0 > my_hi;
-                    v1 = (int32_t)av1 < my_lo || (int32_t)av1 > my_hi;
-                }
-                const unsigned bal0 = __ballot_sync(0xffffffffu, v0 && act0 && g < p.m);
-                const unsigned bal1 = __ballot_sync(0xffffffffu, v1 && act1 && g < p.m);
-                const unsigned bal = hi4 ? bal1 : bal0;
-                const int jj = hi4 ? j1 : j0;
-                if ((g & 3) == 0 && jj < cnt)
-                    nk[jj] = pack_key(__popc((bal >> (8 * gi)) & 0xFFu), v, hi4 ? id1 : id0);
-                BOA_T_MARK(6);
             }
             __syncwarp();
         };
