@@ -52,7 +52,7 @@ def parse_args():
     ap.add_argument("--mode", default="resume", choices=["restart", "resume"])
     ap.add_argument("--schedule", default="16,512")
     ap.add_argument("--plus-k", type=int, default=0)
-    ap.add_argument("--hash-log2", type=int, default=0)
+    ap.add_argument("--table-kb", type=int, default=0)
     ap.add_argument("--max-warps", type=int, default=0)
     ap.add_argument("--no-extras", action="store_true", help="debug: skip recall/e2e/cpu legs")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
@@ -274,7 +274,7 @@ def main():
     ix.set_param("mode", 1 if args.mode == "resume" else 0)
     ix.set_param("eps", args.eps)
     ix.set_param("plus_k", args.plus_k)
-    ix.set_param("hash_log2", args.hash_log2)
+    ix.set_param("table_kb", args.table_kb)
     ix.set_param("max_warps_per_sm", args.max_warps)
     ix.set_schedule(widths)
     Q, k = w.Q, w.k
@@ -320,7 +320,7 @@ def main():
     if args.no_extras:
         if rank == 0:
             sampler.stop()
-            print(json.dumps({"ms_per_step": ms_per_step, "value": value, "hash_log2": args.hash_log2,
+            print(json.dumps({"ms_per_step": ms_per_step, "value": value, "table_kb": args.table_kb,
                               "schedule": widths, "mode": args.mode,
                               "plus_k": args.plus_k, "mean_scored": float(st["n_scored"].mean()),
                               "status": ix.device_status()}))
@@ -383,7 +383,7 @@ def main():
     kernel_ms = float(np.mean(step_ms))
     achieved = alg_bytes / (kernel_ms / 1e3) / 1e9
     traffic = None
-    if (args.workload in NCU_DRAM_BYTES_PER_SCORED and not args.scale_n and not args.hash_log2):
+    if (args.workload in NCU_DRAM_BYTES_PER_SCORED and not args.scale_n and not args.table_kb):
         traffic = NCU_DRAM_BYTES_PER_SCORED[args.workload] * float(st["n_scored"].sum())
 
     line = {

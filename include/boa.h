@@ -52,8 +52,9 @@ enum {
                                Multiple Batches")                                            */
     BOA_PARAM_CAP_MULT = 5, /* a phase at width L gives up after CAP_MULT*L + CAP_ADD        */
     BOA_PARAM_CAP_ADD = 6,  /*   expansions; defaults 8 and 64                               */
-    BOA_PARAM_HASH_LOG2 = 7, /* 0 = choose per phase; else log2 of the per-query table of
-                               recently scored ids (8..14).  Never changes results.          */
+    BOA_PARAM_TABLE_KB = 7, /* 0 = default (6); else KB of shared memory per query for the
+                               table of recently scored ids: 1, 2, 3, 4, 6, 8, 12, 16 or 24.
+                               Never changes results.                                        */
     BOA_PARAM_MAX_WARPS_PER_SM = 8 /* 0 = as many query warps per SM as fit; else a cap.
                                Never changes results.                                        */
 };

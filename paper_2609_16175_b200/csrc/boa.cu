@@ -159,7 +159,7 @@ struct boa_index {
     int device = 0, num_sms = 0;
     // parameters
     double eps = 0.05, growth = 4.0, tau = 0.0;
-    int mode = 0, plus_k = 0, cap_mult = 8, cap_add = 64, hash_log2 = 0, max_ctas = 0;
+    int mode = 0, plus_k = 0, cap_mult = 8, cap_add = 64, table_kb = 0, max_ctas = 0;
     int n_sched = 0;
     int sched[BOA_MAX_PHASES] = {0};
     // scratch
@@ -261,15 +261,29 @@ KernelChoice pick_kernel(const boa_index* ix)
     }
 }
 
-int choose_hash_log2(const boa_index* ix, int L)
+// Table of recently scored ids: size in KB (a power of two, or three times one) -> bucket
+// count, bucket-group bits and the bits left for group-local addressing.  Tags are 16 bits.
+struct TableShape { int buckets, mul3, id_bits, low_bits; };
+TableShape choose_table(const boa_index* ix)
 {
-    if (ix->hash_log2) return ix->hash_log2;
-    (void)L;
-    int lg = 11;                      // 2048 16-bit entries: 4 KB per query
-    int id_bits = 1;
-    while (((int64_t)1 << id_bits) < ix->N) ++id_bits;
-    if (id_bits - (lg - 2) > 16) lg = id_bits - 14;     // tags must fit 16 bits
-    return lg;
+    int kb_size = ix->table_kb ? ix->table_kb : 6;     // default: 768 buckets, 3072 tags
+    TableShape t;
+    t.id_bits = 1;
+    while (((int64_t)1 << t.id_bits) < ix->N) ++t.id_bits;
+    for (;;) {
+        t.mul3 = (kb_size % 3 == 0) ? 1 : 0;
+        const int groups = (t.mul3 ? kb_size / 3 : kb_size) * 128;     // 2^kb
+        int kb = 0;
+        while ((1 << kb) < groups) ++kb;
+        if (kb > t.id_bits) kb = t.id_bits;
+        t.low_bits = t.id_bits - kb;
+        t.buckets = (t.mul3 ? 3 : 1) << kb;
+        // the largest tag must stay below 0xFFFF (the empty mark)
+        const uint32_t max_tag = ((1u << t.low_bits) - 1u) / (t.mul3 ? 3u : 1u);
+        if (max_tag < 0xFFFFu || kb_size >= 1024) break;
+        kb_size *= 2;
+    }
+    return t;
 }
 
 int phase_widths(const boa_index* ix, int L0, int Lmax, int* w)
@@ -335,15 +349,10 @@ int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_p
     const int Lmax = lp.widths[lp.n_phases - 1];
     sp.L = L;
     sp.C = ix->mode == 1 ? Lmax : L;
-    sp.hash_log2 = choose_hash_log2(ix, L);
     {
-        int id_bits = 1;
-        while (((int64_t)1 << id_bits) < ix->N) ++id_bits;
-        if (id_bits - (sp.hash_log2 - 2) > 16) sp.hash_log2 = id_bits - 14;
-        int bucket_bits = sp.hash_log2 - 2;
-        if (bucket_bits > id_bits) bucket_bits = id_bits;
-        sp.id_bits = id_bits;
-        sp.tag_bits = id_bits - bucket_bits;
+        const TableShape t = choose_table(ix);
+        sp.table_buckets = t.buckets; sp.table_mul3 = t.mul3;
+        sp.id_bits = t.id_bits; sp.low_bits = t.low_bits;
     }
     sp.max_expand = ix->cap_mult * L + ix->cap_add;
     sp.first_phase = p == 0;
@@ -360,7 +369,7 @@ int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_p
     sp.out_list = ix->lists + (size_t)(p + 1 < BOA_MAX_PHASES ? p + 1 : p) * ix->ws_Q;
     sp.out_count = ix->counters + kCntCount + p + 1;
 
-    const boa::WarpSmem lay = boa::warp_smem_layout(sp.C, sp.hash_log2, ix->D, lp.kc.rs, lp.kc.q_in_smem);
+    const boa::WarpSmem lay = boa::warp_smem_layout(sp.C, sp.table_buckets, ix->D, lp.kc.rs, lp.kc.q_in_smem);
     const size_t smem = (size_t)lay.total;
     if (smem > 48 * 1024) {
         BOA_CUDA(cudaFuncSetAttribute((const void*)lp.kc.fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -541,9 +550,16 @@ int boa_set_param(boa_index* ix, int key, double v)
         case BOA_PARAM_CAP_ADD:
             if (v < 0.0 || v > 1e6 || v != floor(v)) return BOA_EINVAL;
             ix->cap_add = (int)v; return BOA_OK;
-        case BOA_PARAM_HASH_LOG2:
-            if (v != 0.0 && (v < 8.0 || v > 15.0 || v != floor(v))) return BOA_EINVAL;
-            ix->hash_log2 = (int)v; return BOA_OK;
+        case BOA_PARAM_TABLE_KB: {
+            const int kb = (int)v;
+            bool ok = v == floor(v) && kb >= 0 && kb <= 24;
+            if (ok && kb > 0) {
+                int t = (kb % 3 == 0) ? kb / 3 : kb;
+                ok = (t & (t - 1)) == 0;               // a power of two, or three times one
+            }
+            if (!ok) return BOA_EINVAL;
+            ix->table_kb = kb; return BOA_OK;
+        }
         case BOA_PARAM_MAX_WARPS_PER_SM:
             if (v < 0.0 || v > 64.0 || v != floor(v)) return BOA_EINVAL;
             ix->max_ctas = (int)v; return BOA_OK;

@@ -20,10 +20,12 @@
 // 128-d workload because the kernel is bound by instruction issue and dependent
 // latency, not by the number of bytes in flight.
 //
-// The table of recently scored ids stores 16-bit tags in 4-way buckets.  An id is
-// first mapped by an odd multiplier modulo 2^id_bits (a bijection); the high bits
-// pick the bucket and the low bits are the tag, so bucket + tag identify the id
-// exactly: the table can forget an id, it can never report an unseen id as seen.
+// The table of recently scored ids stores 16-bit tags in 4-way buckets (least recently
+// met way replaced).  An id is first mapped by an odd multiplier modulo 2^id_bits (a
+// bijection); the high bits pick the bucket (with 3*2^kb buckets: the bucket group, and
+// the low part modulo 3 the bucket inside it) and the rest is the tag, so bucket + tag
+// identify the id exactly: the table can forget an id, it can never report an unseen id
+// as seen.
 // A forgotten id that is met again is scored again and then recognised by its key
 // in the pool (or rejected again by the pool's worst key), so results never change.
 //
@@ -87,9 +89,10 @@ struct SearchParams {
     // phase
     int L;                    // beamwidth: expandable prefix of the pool
     int C;                    // pool capacity (L in restart mode, Lmax in resume mode)
-    int hash_log2;            // log2 of the 16-bit entries in the table of recently scored ids
+    int table_buckets;        // 4-way buckets in the table of recently scored ids: 2^kb or 3*2^kb
+    int table_mul3;           // 1 when the bucket count is 3*2^kb
     int id_bits;              // bits of a node id (ids < 2^id_bits)
-    int tag_bits;             // id_bits - log2(buckets), at most 16
+    int low_bits;             // id_bits - kb: bits of a mapped id below its bucket group
     int max_expand;           // expansions after which a phase gives up
     int first_phase;          // statistics start from zero
     int resume_in;            // load the pool a narrower phase spilled
@@ -264,14 +267,14 @@ struct WarpSmem {
 };
 // q_in_smem: the query vector is kept in shared memory (only when lanes do not hold their
 // slices of it in registers).
-__host__ __device__ inline WarpSmem warp_smem_layout(int C, int hash_log2, int D, int RS, bool q_in_smem)
+__host__ __device__ inline WarpSmem warp_smem_layout(int C, int table_buckets, int D, int RS, bool q_in_smem)
 {
     WarpSmem s;
     int off = 0;
     s.pool_off = off;  off += ((C + 1) & ~1) * 8;
     s.nk_off = off;    off += 32 * RS * 8;
     s.q_off = off;     off += q_in_smem ? ((D * 4 + 15) & ~15) : 0;
-    s.hash_off = off;  off += (1 << hash_log2) * 2;
+    s.hash_off = off;  off += table_buckets * 8;
     s.cand_off = off;  off += 32 * RS * 4;
     s.nr_off = off;    off += 32 * RS * 4;
     s.total = (off + 127) & ~127;
@@ -295,7 +298,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
     constexpr int QF4 = (VT == 0) ? 1 : 4;          // float4 slices of the query per chunk
     constexpr int NQ = (CPL > 0) ? CPL * QF4 : 1;
 
-    const WarpSmem lay = warp_smem_layout(p.C, p.hash_log2, p.D, RS, CPL == 0);
+    const WarpSmem lay = warp_smem_layout(p.C, p.table_buckets, p.D, RS, CPL == 0);
     uint64_t* pool = reinterpret_cast<uint64_t*>(smem_raw + lay.pool_off);
     uint64_t* nk = reinterpret_cast<uint64_t*>(smem_raw + lay.nk_off);
     uint32_t* nr = reinterpret_cast<uint32_t*>(smem_raw + lay.nr_off);
@@ -304,7 +307,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
     float4* qs = reinterpret_cast<float4*>(smem_raw + lay.q_off);
 
     const uint32_t id_mask = (p.id_bits >= 32) ? 0xFFFFFFFFu : ((1u << p.id_bits) - 1u);
-    const uint32_t tag_mask = (1u << p.tag_bits) - 1u;
+    const uint32_t low_mask = (1u << p.low_bits) - 1u;
 
     // work range of this launch
     const uint32_t w_begin = p.in_begin_ptr ? *p.in_begin_ptr : p.in_begin;
@@ -332,7 +335,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             }
             const uint4 ff = make_uint4(~0u, ~0u, ~0u, ~0u);
             uint4* h4 = reinterpret_cast<uint4*>(hash);
-            for (int i = lane; i < (1 << p.hash_log2) / 8; i += 32) h4[i] = ff;
+            for (int i = lane; i < p.table_buckets / 2; i += 32) h4[i] = ff;
         }
         int32_t my_lo = 0, my_hi = 0;
         if (g < p.m) {
@@ -500,8 +503,12 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
         // Returns true when id was not in the table; records it either way.
         auto hash_test_and_set = [&](uint32_t id) -> bool {
             const uint32_t h = (id * 0x9E3779B1u) & id_mask;
-            const uint32_t tag = h & tag_mask;
-            const uint32_t bucket = h >> p.tag_bits;
+            // (high part, low part) -> (bucket, tag), one to one: with 3*2^kb buckets the low
+            // part picks one of three buckets of its group and its third is the tag
+            const uint32_t top = h >> p.low_bits, low = h & low_mask;
+            const uint32_t third = __umulhi(low, 0xAAAAAAABu) >> 1;        // low / 3
+            const uint32_t tag = p.table_mul3 ? third : low;
+            const uint32_t bucket = p.table_mul3 ? top * 3u + (low - 3u * third) : top;
             uint2* slot = reinterpret_cast<uint2*>(hash + 4 * bucket);
             const uint2 b = *slot;
             const uint32_t w0 = b.x & 0xFFFFu, w1 = b.x >> 16, w2 = b.y & 0xFFFFu, w3 = b.y >> 16;
