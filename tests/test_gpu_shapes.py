@@ -61,3 +61,22 @@ def test_shape_variants_match_oracle(case):
             assert_bit_parity(o, r, f"{name}/{mode}/eps={eps}")
     assert (r["ids"] != SENTINEL).any()
     gpu.close()
+
+
+def test_degenerate_sizes():
+    """One point, two points, one query, every neighbour slot empty."""
+    for N in (1, 2, 5):
+        x = np.arange(N * 8, dtype=np.float32).reshape(N, 8)
+        g = np.full((N, 3), SENTINEL, dtype=np.uint32)
+        if N > 1:
+            g[:, 0] = (np.arange(N) + 1) % N
+        d = dict(vectors=x, attrs=np.arange(N, dtype=np.int32)[:, None], attr_types=np.zeros(1, np.int32),
+                 graph=g, queries=np.ones((1, 8), np.float32), lo=np.array([[0]], np.int32),
+                 hi=np.array([[3]], np.int32))
+        orc, gpu, gg = make_pair(d)
+        for mode in ("restart", "resume"):
+            o = orc.search(d["queries"], d["lo"], d["hi"], 2, [2, 8], mode=mode, dist_mode=1)
+            r = gpu_search(gpu, gg, 2, [2, 8], mode=mode)
+            assert_bit_parity(o, r, f"N={N}/{mode}")
+        assert r["ids"][0, 0] == 0
+        gpu.close()
