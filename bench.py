@@ -54,6 +54,8 @@ def parse_args():
     ap.add_argument("--plus-k", type=int, default=0)
     ap.add_argument("--table-kb", type=int, default=0)
     ap.add_argument("--max-warps", type=int, default=0)
+    ap.add_argument("--fixed-L", type=int, default=0,
+                    help="the paper's Fixed-L baseline: one phase at this beamwidth for every query")
     ap.add_argument("--no-extras", action="store_true", help="debug: skip recall/e2e/cpu legs")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--seed", type=int, default=0)
@@ -78,6 +80,8 @@ def get_workload(args):
 
 
 def schedule_of(args, w):
+    if getattr(args, "fixed_L", 0):
+        return [int(args.fixed_L)]
     s = [int(x) for x in args.schedule.split(",") if x]
     if s[0] != w.L0 or s[-1] != w.Lmax:
         s = [w.L0] + [x for x in s[1:-1] if w.L0 < x < w.Lmax] + [w.Lmax]
