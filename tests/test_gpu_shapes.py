@@ -80,3 +80,28 @@ def test_degenerate_sizes():
             assert_bit_parity(o, r, f"N={N}/{mode}")
         assert r["ids"][0, 0] == 0
         gpu.close()
+
+
+def test_many_random_small_cases():
+    """Thirty seeded random shapes (dimension, element type, attribute count and types,
+    degree, k, widths, ε, mode, BOA+), each against the oracle bit for bit."""
+    rng = np.random.default_rng(2024)
+    for case in range(30):
+        dtype = "u8" if rng.random() < 0.4 else "f32"
+        D = int(rng.integers(1, 9)) * (16 if dtype == "u8" else 4)
+        m = int(rng.integers(1, 9))
+        R = int(rng.integers(2, 65))
+        N = int(rng.integers(R + 2, 1500))
+        fcols = tuple(j for j in range(m) if rng.random() < 0.3)
+        d = _random_case(1000 + case, N, D, dtype, m, R, 24, fcols)
+        k = int(rng.integers(1, 12))
+        L0 = int(rng.integers(k, k + 20))
+        widths = sorted({L0, L0 + int(rng.integers(1, 100)), L0 + int(rng.integers(100, 600))})
+        mode = "resume" if rng.random() < 0.5 else "restart"
+        eps = float(rng.choice([0.02, 0.1, 0.4]))
+        plus_k = int(rng.choice([0, 0, 3]))
+        orc, gpu, g = make_pair(d)
+        o = orc.search(d["queries"], d["lo"], d["hi"], k, widths, eps=eps, mode=mode, dist_mode=1)
+        r = gpu_search(gpu, g, k, widths, mode=mode, eps=eps, plus_k=plus_k)
+        assert_bit_parity(o, r, f"case {case}: {dtype} D={D} m={m} R={R} N={N} k={k} {widths} {mode}")
+        gpu.close()

@@ -438,3 +438,43 @@ def test_harness_ground_truth_equals_oracle_bruteforce(which, request):
     assert np.nanmin(rec) == 1.0
     worse = recall_against(o_ids, (o_d2 * 4.0 + 1.0).astype(np.float32), d2.numpy(), nv.numpy(), 10)
     assert np.nanmean(worse) < 0.5
+
+
+# ----------------------------------------------------------------------------
+# the same closed forms on many random tiny inputs
+# ----------------------------------------------------------------------------
+def test_random_tiny_graphs_full_width_is_exact_and_narrow_is_valid():
+    from hypothesis import given, settings, strategies as st
+
+    @settings(max_examples=60, deadline=None)
+    @given(st.integers(0, 10 ** 6), st.integers(8, 60), st.integers(2, 5), st.integers(1, 3))
+    def check(seed, N, R, m):
+        rng = np.random.default_rng(seed)
+        x = rng.integers(0, 16, size=(N, 4)).astype(np.float32)
+        attrs = rng.integers(0, 10, size=(N, m)).astype(np.int32)
+        g = rng.integers(0, N, size=(N, R)).astype(np.uint32)
+        g[:, 0] = (np.arange(N) + 1) % N                       # a ring keeps it strongly connected
+        g[rng.random((N, R)) < 0.2] = SENTINEL
+        g[:, 0] = (np.arange(N) + 1) % N
+        ix = OracleIndex(x, attrs, np.zeros(m, np.int32), g, entry=int(rng.integers(N)))
+        q = rng.integers(0, 16, size=(3, 4)).astype(np.float32)
+        lo = rng.integers(0, 6, size=(3, m)).astype(np.int32)
+        hi = (lo + rng.integers(0, 8, size=(3, m))).astype(np.int32)
+        k = int(rng.integers(1, 6))
+        gt_ids, gt_d2, nvalid = ix.bruteforce(q, lo, hi, k)
+        for mode in ("restart", "resume"):
+            full = ix.search(q, lo, hi, k, [max(k, 4), N], eps=-1.0, mode=mode)
+            assert (full["ids"] == gt_ids).all()
+            narrow = ix.search(q, lo, hi, k, [max(k, 4)], mode=mode)
+            for i in range(3):
+                ids = narrow["ids"][i]
+                n = int((ids != SENTINEL).sum())
+                assert n <= min(k, nvalid[i]) and (ids[n:] == SENTINEL).all()
+                a = attrs[ids[:n].astype(np.int64)]
+                assert ((a >= lo[i]) & (a <= hi[i])).all()
+                keys = list(zip(narrow["d2"][i][:n].tolist(), ids[:n].tolist()))
+                assert keys == sorted(keys) and len(set(ids[:n].tolist())) == n
+                # what the narrow search returns can never beat the exact answer
+                assert (narrow["d2"][i][:n].astype(np.float64) >= gt_d2[i][:n]).all()
+
+    check()
