@@ -53,8 +53,10 @@ enum {
     BOA_PARAM_CAP_MULT = 5, /* a phase at width L gives up after CAP_MULT*L + CAP_ADD        */
     BOA_PARAM_CAP_ADD = 6,  /*   expansions; defaults 8 and 64                               */
     BOA_PARAM_TABLE_KB = 7, /* 0 = default (6); else KB of shared memory per query for the
-                               table of recently scored ids: 1, 2, 3, 4, 6, 8, 12, 16 or 24.
-                               Never changes results.                                        */
+                               table of recently scored ids: 1, 2, 3, 4, 6, 8, 12, 16 or 24
+                               (doubled automatically while an index of more than 2^25
+                               points needs tags wider than 16 bits).  Never changes
+                               results.                                                      */
     BOA_PARAM_MAX_WARPS_PER_SM = 8 /* 0 = as many query warps per SM as fit; else a cap.
                                Never changes results.                                        */
 };
