@@ -165,7 +165,7 @@ struct boa_index {
     // scratch
     int64_t ws_Q = 0;
     int ws_spill = 0;
-    uint32_t* lists = nullptr;     // [BOA_MAX_PHASES][ws_Q]
+    uint32_t* lists = nullptr;     // [2][BOA_MAX_PHASES][ws_Q]: survivor lists (second set: BOA+ pool 2)
     uint32_t* counters = nullptr;  // see enum below
     int32_t* stats = nullptr;      // [4][ws_Q]
     uint64_t* spill = nullptr;     // [ws_Q][ws_spill]
@@ -182,7 +182,7 @@ struct boa_index {
 namespace {
 // layout of boa_index::counters (uint32 words)
 constexpr int kCntCount = 0;                          // [P+1] survivors entering phase p (p>=1)
-constexpr int kCntConsumed = 16;                      // [P+1] list positions already searched
+constexpr int kCntCount2 = 16;                        // [P+1] the same for the second pool of BOA+ (p>=2)
 constexpr int kCntSnap = 32;                          // [pool] frozen end of phase 1's list
 constexpr int kCntStatus = 47;                        // device status bits
 constexpr int kCntTicket = 48;                        // one per launch
@@ -194,7 +194,7 @@ constexpr int64_t kNoAllocMaxQ = BOA_NOALLOC_MAX_Q;
 constexpr int kNoAllocMaxWidth = BOA_NOALLOC_MAX_WIDTH;
 constexpr size_t kNaCounters = 0;                                             // 1 KiB
 constexpr size_t kNaLists = 1024;                                             // [phases][Q] u32
-constexpr size_t kNaStats = kNaLists + (size_t)BOA_MAX_PHASES * kNoAllocMaxQ * 4;
+constexpr size_t kNaStats = kNaLists + (size_t)2 * BOA_MAX_PHASES * kNoAllocMaxQ * 4;
 constexpr size_t kNaSpillSize = kNaStats + (size_t)4 * kNoAllocMaxQ * 4;
 constexpr size_t kNaSpill = kNaSpillSize + (size_t)kNoAllocMaxQ * 4;
 constexpr size_t kNaBytes = kNaSpill + (size_t)kNoAllocMaxQ * kNoAllocMaxWidth * 8;
@@ -319,7 +319,7 @@ int ensure_workspace(boa_index* ix, int64_t Q, int Lmax)
         cudaFree(ix->lists); cudaFree(ix->stats); cudaFree(ix->spill); cudaFree(ix->spill_size);
         ix->lists = nullptr; ix->stats = nullptr; ix->spill = nullptr; ix->spill_size = nullptr;
         ix->ws_Q = 0; ix->ws_spill = 0;
-        BOA_CUDA(cudaMalloc(&ix->lists, (size_t)BOA_MAX_PHASES * nq * sizeof(uint32_t)));
+        BOA_CUDA(cudaMalloc(&ix->lists, (size_t)2 * BOA_MAX_PHASES * nq * sizeof(uint32_t)));
         BOA_CUDA(cudaMalloc(&ix->stats, (size_t)4 * nq * sizeof(int32_t)));
         BOA_CUDA(cudaMalloc(&ix->spill_size, (size_t)nq * sizeof(int32_t)));
         if (ns > 0) BOA_CUDA(cudaMalloc(&ix->spill, (size_t)nq * ns * sizeof(uint64_t)));
@@ -339,8 +339,11 @@ struct LaunchPlan {
 };
 
 // One launch of Algorithm 2 over positions [begin, end) of phase p's work list.
+// `chain` picks the set of survivor lists and counters (0 everywhere except the second
+// pooled escalation of BOA+); phase 1 always reads the one list the first phase wrote.
 int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_ptr,
-                 const uint32_t* end_ptr, uint32_t begin, uint32_t end, uint32_t expected_items)
+                 const uint32_t* end_ptr, uint32_t begin, uint32_t end, uint32_t expected_items,
+                 int chain = 0, bool use_active_count = true)
 {
     boa_index* ix = lp.ix;
     if (lp.launches >= kMaxLaunches) return BOA_EINVAL;
@@ -359,15 +362,17 @@ int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_p
     sp.resume_in = (ix->mode == 1 && p > 0);
     sp.last_phase = p == lp.n_phases - 1;
     sp.spill_out = (ix->mode == 1 && !sp.last_phase);
-    sp.in_list = p == 0 ? nullptr : ix->lists + (size_t)p * ix->ws_Q;
+    uint32_t* lists_c = ix->lists + (size_t)chain * BOA_MAX_PHASES * ix->ws_Q;
+    uint32_t* cnt_c = ix->counters + (chain == 0 ? kCntCount : kCntCount2);
+    sp.in_list = p == 0 ? nullptr : (p == 1 ? ix->lists : lists_c) + (size_t)p * ix->ws_Q;
     sp.in_begin_ptr = begin_ptr;
     sp.in_end_ptr = end_ptr;
     sp.in_begin = begin;
     sp.in_end = end;
-    sp.active_count = p == 0 ? nullptr : ix->counters + kCntCount + p;
+    sp.active_count = (p == 0 || !use_active_count) ? nullptr : ix->counters + kCntCount + p;
     sp.ticket = ix->counters + kCntTicket + lp.launches;
-    sp.out_list = ix->lists + (size_t)(p + 1 < BOA_MAX_PHASES ? p + 1 : p) * ix->ws_Q;
-    sp.out_count = ix->counters + kCntCount + p + 1;
+    sp.out_list = lists_c + (size_t)(p + 1 < BOA_MAX_PHASES ? p + 1 : p) * ix->ws_Q;
+    sp.out_count = cnt_c + p + 1;
 
     const boa::WarpSmem lay = boa::warp_smem_layout(sp.C, sp.table_buckets, ix->D, lp.kc.rs, lp.kc.q_in_smem);
     const size_t smem = (size_t)lay.total;
@@ -583,7 +588,7 @@ int boa_workspace_bytes(const boa_index* ix, int64_t Q, int Lmax, size_t* bytes)
 {
     if (!ix || !bytes || Q < 0 || Lmax < 1 || Lmax > BOA_MAX_WIDTH) return BOA_EINVAL;
     size_t b = kCntWords * sizeof(uint32_t);
-    b += (size_t)BOA_MAX_PHASES * Q * sizeof(uint32_t) + (size_t)5 * Q * sizeof(int32_t);
+    b += (size_t)2 * BOA_MAX_PHASES * Q * sizeof(uint32_t) + (size_t)5 * Q * sizeof(int32_t);
     if (ix->mode == 1) b += (size_t)Q * ((Lmax + 1) & ~1) * sizeof(uint64_t);
     *bytes = b;
     return BOA_OK;
@@ -652,9 +657,7 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
 
     const int K = (ix->plus_k >= 2 && lp.n_phases > 1 && ix->tau == 0.0) ? ix->plus_k : 1;
     uint32_t* cnt = ix->counters + kCntCount;
-    uint32_t* consumed = ix->counters + kCntConsumed;
     uint32_t* snap = ix->counters + kCntSnap;
-    int n_pools = 0;
     if (K == 1) {
         // BOA: one launch per phase, each over the survivors of the one before
         rc = launch_phase(lp, 0, st, nullptr, nullptr, 0u, (uint32_t)Q, (uint32_t)Q);
@@ -664,10 +667,11 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
             if (rc != BOA_OK) return rc;
         }
     } else {
-        // BOA+: the first phase goes out as K sub-batches on the caller's stream.  After
-        // the sub-batch in the middle and after the last one the survivors gathered so
-        // far are escalated together through all wider phases on the side stream, so
-        // the wide searches of the first pool overlap the remaining narrow sub-batches.
+        // BOA+: the first phase goes out as K sub-batches on the caller's stream.  The
+        // survivors gathered up to the middle sub-batch are escalated together through all
+        // wider phases on the side stream while the remaining narrow sub-batches run; the
+        // survivors of the second half follow as a second pool on the caller's stream,
+        // concurrently with the first pool.  Each pool has its own lists from phase 2 on.
         const int mid = (K + 1) / 2;
         for (int j = 0; j < K; ++j) {
             const uint32_t b0 = (uint32_t)((Q * j) / K), b1 = (uint32_t)((Q * (j + 1)) / K);
@@ -676,24 +680,30 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
                 if (rc != BOA_OK) return rc;
             }
             if (j + 1 == mid || j + 1 == K) {
-                uint32_t* my_snap = snap + n_pools++;     // one word per pooled escalation
-                copy_word_kernel<<<1, 1, 0, st>>>(my_snap, cnt + 1);
+                const int chain = (j + 1 == K && mid != K) ? 1 : 0;
+                // freeze the end of the phase-1 list at this point of the caller's stream
+                copy_word_kernel<<<1, 1, 0, st>>>(snap + chain, cnt + 1);
                 extra_launches++;
                 BOA_CUDA(cudaGetLastError());
-                BOA_CUDA(cudaEventRecord(ix->ev_fork, st));
-                BOA_CUDA(cudaStreamWaitEvent(ix->side, ix->ev_fork, 0));
+                cudaStream_t cs = st;
+                if (chain == 0 && mid != K) {
+                    BOA_CUDA(cudaEventRecord(ix->ev_fork, st));
+                    BOA_CUDA(cudaStreamWaitEvent(ix->side, ix->ev_fork, 0));
+                    cs = ix->side;
+                }
+                uint32_t* cnt_c = ix->counters + (chain == 0 ? kCntCount : kCntCount2);
                 for (int p = 1; p < lp.n_phases; ++p) {
-                    const uint32_t* endp = (p == 1) ? my_snap : cnt + p;
-                    rc = launch_phase(lp, p, ix->side, consumed + p, endp, 0u, 0u, (uint32_t)Q);
+                    const uint32_t* beginp = (p == 1 && chain == 1) ? snap + 0 : nullptr;
+                    const uint32_t* endp = (p == 1) ? snap + chain : cnt_c + p;
+                    rc = launch_phase(lp, p, cs, beginp, endp, 0u, 0u, (uint32_t)Q, chain, false);
                     if (rc != BOA_OK) return rc;
-                    copy_word_kernel<<<1, 1, 0, ix->side>>>(consumed + p, endp);
-                    extra_launches++;
-                    BOA_CUDA(cudaGetLastError());
                 }
             }
         }
-        BOA_CUDA(cudaEventRecord(ix->ev_join, ix->side));
-        BOA_CUDA(cudaStreamWaitEvent(st, ix->ev_join, 0));
+        if (mid != K) {
+            BOA_CUDA(cudaEventRecord(ix->ev_join, ix->side));
+            BOA_CUDA(cudaStreamWaitEvent(st, ix->ev_join, 0));
+        }
     }
     ix->last_launches = lp.launches + extra_launches;
     return BOA_OK;
@@ -721,12 +731,14 @@ int boa_get_phase_counts(boa_index* ix, int64_t* active, int n, int* n_phases, v
     if (n_phases) *n_phases = ix->last_phases;
     if (ix->last_Q == 0 || ix->last_phases == 0) return BOA_OK;
     uint32_t h[BOA_MAX_PHASES + 1] = {0};
+    uint32_t h2[BOA_MAX_PHASES + 1] = {0};
     BOA_CUDA(cudaMemcpyAsync(h, ix->counters + kCntCount, sizeof(h), cudaMemcpyDeviceToHost, st));
+    BOA_CUDA(cudaMemcpyAsync(h2, ix->counters + kCntCount2, sizeof(h2), cudaMemcpyDeviceToHost, st));
     BOA_CUDA(cudaStreamSynchronize(st));
     const double tau_q = ix->tau * (double)ix->last_Q;
     bool stopped = false;
     for (int p = 0; p < n && p < ix->last_phases; ++p) {
-        const int64_t a = p == 0 ? ix->last_Q : (int64_t)h[p];
+        const int64_t a = p == 0 ? ix->last_Q : (int64_t)h[p] + (p >= 2 ? (int64_t)h2[p] : 0);
         if (!((double)a > tau_q)) stopped = true;
         active[p] = stopped ? 0 : a;
     }
