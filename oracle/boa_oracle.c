@@ -30,6 +30,8 @@
  *     resume mode keeps pool, flags and seen set, pool capacity Lmax, and only
  *     lengthens the expandable prefix (reading of "redundancy avoidance")
  *   - a phase stops after cap_mult*L + cap_add expansions at the latest
+ *   - expansion width W (nodes expanded per iteration) is 1 as in the paper unless a
+ *     caller asks for more; see orc_beam_run_w
  *
  * parity pins: tests/test_oracle_pins.py (brute force vs. an independent sort,
  * g == 1 vs. a library k-NN, the ring-graph hand trace, full-graph search ==
@@ -43,6 +45,7 @@
 #include <string.h>
 
 #define ORC_SENTINEL 0xFFFFFFFFu
+#define ORC_MAX_W 64            /* largest expansion width (nodes per iteration) */
 #define ORC_F32 0
 #define ORC_U8 1
 #define ORC_ATTR_I32 0
@@ -235,7 +238,7 @@ orc_state *orc_state_new(const orc_index *ix, int C)
 {
     orc_state *st = (orc_state *)calloc(1, sizeof(orc_state));
     st->ix = ix; st->C = C;
-    st->pool = (orc_entry_t *)calloc((size_t)(C + ix->R + 1), sizeof(orc_entry_t));
+    st->pool = (orc_entry_t *)calloc((size_t)C + (size_t)ORC_MAX_W * ix->R + 1, sizeof(orc_entry_t));
     st->seen = (uint8_t *)calloc((size_t)ix->N, 1);
     st->touched_cap = 1024;
     st->touched = (uint32_t *)malloc((size_t)st->touched_cap * sizeof(uint32_t));
@@ -281,36 +284,58 @@ void orc_beam_init(orc_state *st, int C, const float *q, const int32_t *lo, cons
 
 /* run the loop of Algorithm 2 at beamwidth L until every one of the first L
    pool entries is expanded; gives up (hit_cap) when an unexpanded entry is left
-   after max_expand expansions of this call */
-void orc_beam_run(orc_state *st, int L, const float *q, const int32_t *lo, const int32_t *hi,
-                  int dist_mode, int64_t max_expand)
+   after max_expand expansions of this call.
+
+   W is the expansion width.  The paper expands one node per iteration (W = 1).
+   With W > 1 (an extension: the step widening of multi-node expansion in GPU
+   graph search) an iteration takes the first W unexpanded entries of the beam,
+   fewer when the beam or the expansion cap leaves fewer, marks them expanded,
+   and then scores their rows in that order before the pool is looked at again. */
+void orc_beam_run_w(orc_state *st, int L, const float *q, const int32_t *lo, const int32_t *hi,
+                    int dist_mode, int64_t max_expand, int W)
 {
     const orc_index *ix = st->ix;
     int64_t done = 0;
     st->hit_cap = 0;
+    if (W < 1) W = 1;
+    if (W > ORC_MAX_W) W = ORC_MAX_W;
     for (;;) {
         int lim = st->size < L ? st->size : L;
-        int u = -1;
+        uint32_t picked[ORC_MAX_W];
+        int np = 0, any = 0;
         for (int t = 0; t < lim; ++t)
-            if (!st->pool[t].expanded) { u = t; break; }
-        if (u < 0) break;                               /* converged */
+            if (!st->pool[t].expanded) { any = 1; break; }
+        if (!any) break;                                /* converged */
         if (done >= max_expand) { st->hit_cap = 1; break; }
-        st->pool[u].expanded = 1;
-        st->n_expand++; done++;
-        uint32_t uid = st->pool[u].id;
-        for (int j = 0; j < ix->R; ++j) {
-            uint32_t n = ix->graph[(int64_t)uid * ix->R + j];
-            if (n == ORC_SENTINEL || st->seen[n]) continue;
-            orc_mark_seen(st, n);
-            st->n_scored++;
-            orc_entry_t e;
-            e.id = n; e.expanded = 0;
-            e.phi = orc_phi(ix, lo, hi, n);
-            e.d2 = orc_dist2(ix, q, n, dist_mode);
-            orc_pool_insert(st, e);
+        for (int t = 0; t < lim && np < W && done + np < max_expand; ++t)
+            if (!st->pool[t].expanded) {
+                st->pool[t].expanded = 1;
+                picked[np++] = st->pool[t].id;
+            }
+        st->n_expand += np; done += np;
+        for (int a = 0; a < np; ++a) {
+            uint32_t uid = picked[a];
+            for (int j = 0; j < ix->R; ++j) {
+                uint32_t n = ix->graph[(int64_t)uid * ix->R + j];
+                if (n == ORC_SENTINEL || st->seen[n]) continue;
+                orc_mark_seen(st, n);
+                st->n_scored++;
+                orc_entry_t e;
+                e.id = n; e.expanded = 0;
+                e.phi = orc_phi(ix, lo, hi, n);
+                e.d2 = orc_dist2(ix, q, n, dist_mode);
+                orc_pool_insert(st, e);
+            }
         }
         if (st->size > st->C) st->size = st->C;          /* keep the C best */
     }
+}
+
+/* Algorithm 2 as printed: one node per iteration */
+void orc_beam_run(orc_state *st, int L, const float *q, const int32_t *lo, const int32_t *hi,
+                  int dist_mode, int64_t max_expand)
+{
+    orc_beam_run_w(st, L, q, lo, hi, dist_mode, max_expand, 1);
 }
 
 /* K_i <- the k nearest filter-valid pool entries; returns how many there are */
@@ -406,13 +431,13 @@ static void orc_restore(orc_state *st, const orc_saved *sv, int C)
  * add up over the phases a query ran; flags bit 0 = some phase hit its
  * expansion cap.
  */
-void orc_boa_search(const orc_index *ix, const float *queries, int64_t Q,
-                    const int32_t *lo, const int32_t *hi, int k,
-                    const int32_t *widths, int n_widths, double eps, double tau,
-                    int mode, int dist_mode, int cap_mult, int cap_add,
-                    uint32_t *out_ids, float *out_d2,
-                    int32_t *final_L, int32_t *n_expand, int32_t *n_scored, int32_t *flags,
-                    int64_t *phase_active)
+void orc_boa_search_w(const orc_index *ix, const float *queries, int64_t Q,
+                      const int32_t *lo, const int32_t *hi, int k,
+                      const int32_t *widths, int n_widths, double eps, double tau,
+                      int mode, int dist_mode, int cap_mult, int cap_add, int W,
+                      uint32_t *out_ids, float *out_d2,
+                      int32_t *final_L, int32_t *n_expand, int32_t *n_scored, int32_t *flags,
+                      int64_t *phase_active)
 {
     int Cmax = 0;
     for (int p = 0; p < n_widths; ++p) if (widths[p] > Cmax) Cmax = widths[p];
@@ -441,7 +466,7 @@ void orc_boa_search(const orc_index *ix, const float *queries, int64_t Q,
             } else {
                 orc_beam_init(st, mode == 1 ? Cmax : L, q, l, h, dist_mode);
             }
-            orc_beam_run(st, L, q, l, h, dist_mode, cap);
+            orc_beam_run_w(st, L, q, l, h, dist_mode, cap, W);
             orc_beam_result(st, k, out_ids + i * k, out_d2 + i * k);    /* scatter */
             final_L[i] = L;
             n_expand[i] += (int32_t)st->n_expand;
@@ -458,4 +483,18 @@ void orc_boa_search(const orc_index *ix, const float *queries, int64_t Q,
     free(saved);
     free(active);
     orc_state_free(st);
+}
+
+/* the paper's setting: expansion width 1 */
+void orc_boa_search(const orc_index *ix, const float *queries, int64_t Q,
+                    const int32_t *lo, const int32_t *hi, int k,
+                    const int32_t *widths, int n_widths, double eps, double tau,
+                    int mode, int dist_mode, int cap_mult, int cap_add,
+                    uint32_t *out_ids, float *out_d2,
+                    int32_t *final_L, int32_t *n_expand, int32_t *n_scored, int32_t *flags,
+                    int64_t *phase_active)
+{
+    orc_boa_search_w(ix, queries, Q, lo, hi, k, widths, n_widths, eps, tau, mode, dist_mode,
+                     cap_mult, cap_add, 1, out_ids, out_d2, final_L, n_expand, n_scored, flags,
+                     phase_active);
 }

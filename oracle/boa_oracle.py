@@ -39,6 +39,7 @@ def lib():
         L.orc_state_free.argtypes = [vp]
         L.orc_beam_init.argtypes = [vp, i32, vp, vp, vp, i32]
         L.orc_beam_run.argtypes = [vp, i32, vp, vp, vp, i32, i64]
+        L.orc_beam_run_w.argtypes = [vp, i32, vp, vp, vp, i32, i64, i32]
         L.orc_beam_result.restype = i32
         L.orc_beam_result.argtypes = [vp, i32, vp, vp]
         L.orc_state_size.restype = i32
@@ -54,6 +55,8 @@ def lib():
         L.orc_uncertain.argtypes = [vp, i32, i32, dbl]
         L.orc_boa_search.argtypes = [vp, vp, i64, vp, vp, i32, vp, i32, dbl, dbl, i32, i32,
                                      i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.orc_boa_search_w.argtypes = [vp, vp, i64, vp, vp, i32, vp, i32, dbl, dbl, i32, i32,
+                                       i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -127,12 +130,13 @@ class OracleIndex:
         return ids, d2, nvalid
 
     # --- one beam search, step-wise ------------------------------------------
-    def beam(self, q, lo, hi, L, C=None, dist_mode=0, max_expand=1 << 40):
-        return OracleBeam(self, q, lo, hi, L, C if C is not None else L, dist_mode, max_expand)
+    def beam(self, q, lo, hi, L, C=None, dist_mode=0, max_expand=1 << 40, expand_w=1):
+        return OracleBeam(self, q, lo, hi, L, C if C is not None else L, dist_mode, max_expand,
+                          expand_w)
 
     # --- the multi-phase batch driver ----------------------------------------
     def search(self, queries, lo, hi, k, widths, eps=0.05, tau=0.0, mode="restart",
-               dist_mode=0, cap=DEFAULT_CAP):
+               dist_mode=0, cap=DEFAULT_CAP, expand_w=1):
         queries = np.ascontiguousarray(queries, dtype=np.float32)
         lo = np.ascontiguousarray(lo, dtype=np.int32)
         hi = np.ascontiguousarray(hi, dtype=np.int32)
@@ -145,10 +149,10 @@ class OracleIndex:
         n_scored = np.empty(Q, dtype=np.int32)
         flags = np.empty(Q, dtype=np.int32)
         phase_active = np.zeros(len(w), dtype=np.int64)
-        lib().orc_boa_search(self.h, _p(queries), Q, _p(lo), _p(hi), k, _p(w), len(w),
-                             float(eps), float(tau), 1 if mode == "resume" else 0, int(dist_mode),
-                             int(cap[0]), int(cap[1]), _p(ids), _p(d2), _p(final_L), _p(n_expand),
-                             _p(n_scored), _p(flags), _p(phase_active))
+        lib().orc_boa_search_w(self.h, _p(queries), Q, _p(lo), _p(hi), k, _p(w), len(w),
+                               float(eps), float(tau), 1 if mode == "resume" else 0, int(dist_mode),
+                               int(cap[0]), int(cap[1]), int(expand_w), _p(ids), _p(d2), _p(final_L),
+                               _p(n_expand), _p(n_scored), _p(flags), _p(phase_active))
         return dict(ids=ids, d2=d2, final_L=final_L, n_expand=n_expand, n_scored=n_scored,
                     flags=flags, phase_active=phase_active)
 
@@ -156,8 +160,9 @@ class OracleIndex:
 class OracleBeam:
     """One query's Algorithm-2 state, for tests that look inside a search."""
 
-    def __init__(self, index, q, lo, hi, L, C, dist_mode, max_expand):
+    def __init__(self, index, q, lo, hi, L, C, dist_mode, max_expand, expand_w=1):
         self.ix = index
+        self.expand_w = int(expand_w)
         self.q = np.ascontiguousarray(q, dtype=np.float32)
         self.lo = np.ascontiguousarray(lo, dtype=np.int32)
         self.hi = np.ascontiguousarray(hi, dtype=np.int32)
@@ -168,8 +173,8 @@ class OracleBeam:
 
     def run(self, L, max_expand=1 << 40):
         self.L = int(L)
-        lib().orc_beam_run(self.st, int(L), _p(self.q), _p(self.lo), _p(self.hi), self.dist_mode,
-                           int(max_expand))
+        lib().orc_beam_run_w(self.st, int(L), _p(self.q), _p(self.lo), _p(self.hi), self.dist_mode,
+                             int(max_expand), self.expand_w)
         return self
 
     def result(self, k):

@@ -228,6 +228,77 @@ def test_ring_walk_passes_through_invalid_nodes():
 
 
 # ----------------------------------------------------------------------------
+# expansion width W > 1 (an extension of Algorithm 2): a second hand trace
+# ----------------------------------------------------------------------------
+def _stride_line():
+    n = 16
+    x = np.arange(n, dtype=np.float32)[:, None]
+    attrs = np.zeros((n, 1), dtype=np.int32)
+    g = np.full((n, 4), SENTINEL, dtype=np.uint32)
+    for i in range(n):
+        for c, o in enumerate((-2, -1, 1, 2)):
+            if 0 <= i + o < n:
+                g[i, c] = i + o
+    return OracleIndex(x, attrs, np.zeros(1, np.int32), g, entry=0)
+
+
+def test_stride_line_hand_trace_width_1_and_2():
+    gold = {r[0]: [int(v) for v in r[1:]] for r in _read_golden("stride_trace_width2.txt")}
+    ix = _stride_line()
+    q = np.array([10.1], dtype=np.float32)
+    z = np.zeros(1, dtype=np.int32)
+    for w, tag in ((1, "w1"), (2, "w2"), (3, "w2")):     # the beam holds two entries: W = 3 picks two
+        b = ix.beam(q, z, z, L=2, C=8, expand_w=w)
+        ids, d2, phi, ex = b.pool()
+        assert [int(i) for i in ids] == gold["final_pool"]
+        assert [int(e) for e in ex] == gold[tag + "_expanded_flags"]
+        assert b.n_expand == len(gold[tag + "_expansions"])
+        assert b.n_scored == len(gold["scored_order"])
+        assert not b.hit_cap
+        assert [int(i) for i in b.result(2)[0]] == [10, 11]
+    # the cap is counted in nodes, not in iterations
+    b = ix.beam(q, z, z, L=2, C=8, expand_w=2, max_expand=4)
+    ids, d2, phi, ex = b.pool()
+    assert b.n_expand == 4 and b.hit_cap
+    assert [int(i) for i in ids] == gold["w2_cap4_pool"]
+    assert [int(e) for e in ex] == gold["w2_cap4_flags"]
+    # the order in which nodes become expanded: a cap of c nodes leaves exactly the first c
+    # of the hand-derived order expanded (capacity 16 keeps every scored node in the pool)
+    for c in range(1, 13):
+        b = ix.beam(q, z, z, L=2, C=16, expand_w=2, max_expand=c)
+        ids, _, _, ex = b.pool()
+        assert sorted(int(i) for i, e in zip(ids, ex) if e) == sorted(gold["w2_expansions"][:c])
+        assert b.hit_cap == (c < 12)
+
+
+@pytest.mark.parametrize("w", [2, 3, 7])
+def test_any_expansion_width_at_full_beam_equals_bruteforce(w):
+    rng = np.random.default_rng(11)
+    N, D, R, k = 200, 6, 5, 8
+    x = rng.integers(0, 32, size=(N, D)).astype(np.float32)
+    attrs = rng.integers(0, 100, size=(N, 2)).astype(np.int32)
+    g = rng.integers(0, N, size=(N, R)).astype(np.uint32)
+    g[:, 0] = (np.arange(N) + 1) % N
+    ix = OracleIndex(x, attrs, np.zeros(2, np.int32), g)
+    q = rng.integers(0, 32, size=(10, D)).astype(np.float32)
+    lo = rng.integers(0, 50, size=(10, 2)).astype(np.int32)
+    hi = (lo + rng.integers(20, 60, size=(10, 2))).astype(np.int32)
+    gt_ids, gt_d2, nvalid = ix.bruteforce(q, lo, hi, k)
+    for i in range(10):
+        b = ix.beam(q[i], lo[i], hi[i], L=N, C=N, expand_w=w)
+        assert b.n_expand == N and b.n_scored == N - 1      # every node once, whatever W
+        assert (b.result(k)[0] == gt_ids[i]).all()
+    r1 = ix.search(q, lo, hi, k, [8, 32], eps=0.05, mode="resume", expand_w=1)
+    rw = ix.search(q, lo, hi, k, [8, 32], eps=0.05, mode="resume", expand_w=w)
+    # narrow beams: whatever W, answers are no better than exact and the cap holds per phase
+    for r in (r1, rw):
+        for i in range(10):
+            n = int((r["ids"][i] != SENTINEL).sum())
+            assert (r["d2"][i][:n].astype(np.float64) >= gt_d2[i][:n]).all()
+            assert (r["n_expand"][i] <= 2 * (8 * 32 + 64)).all()
+
+
+# ----------------------------------------------------------------------------
 # P4: on a graph connected from s with L = C >= N the search sees every node,
 #     so its answer is the exact filtered top-k
 # ----------------------------------------------------------------------------
