@@ -57,8 +57,14 @@ enum {
                                (doubled automatically while an index of more than 2^25
                                points needs tags wider than 16 bits).  Never changes
                                results.                                                      */
-    BOA_PARAM_MAX_WARPS_PER_SM = 8 /* 0 = as many query warps per SM as fit; else a cap.
+    BOA_PARAM_MAX_WARPS_PER_SM = 8, /* 0 = as many query warps per SM as fit; else a cap.
                                Never changes results.                                        */
+    BOA_PARAM_EXPAND_W = 9  /* nodes expanded per iteration of Algorithm 2.  1 (default) is
+                               the algorithm as printed ("each iteration expands one
+                               node").  2 is an extension: the first two unexpanded beam
+                               entries are marked and their rows scored together (first
+                               node's row first), at most as many as the expansion cap
+                               leaves.  Changes which nodes get expanded, hence results.  */
 };
 
 /*

@@ -159,7 +159,7 @@ struct boa_index {
     int device = 0, num_sms = 0;
     // parameters
     double eps = 0.05, growth = 4.0, tau = 0.0;
-    int mode = 0, plus_k = 0, cap_mult = 8, cap_add = 64, table_kb = 0, max_ctas = 0;
+    int mode = 0, plus_k = 0, cap_mult = 8, cap_add = 64, table_kb = 0, max_ctas = 0, expand_w = 1;
     int n_sched = 0;
     int sched[BOA_MAX_PHASES] = {0};
     // scratch
@@ -230,15 +230,20 @@ struct KernelChoice {
     bool q_in_smem;     // the generic-length kernels keep the query in shared memory
 };
 
-template <int VT, int CPL>
-KernelChoice pick_rs(int R, bool exact)
+template <int VT, int CPL, int W>
+KernelChoice pick_rn(int R, bool exact)
 {
     if (R <= 32) {
-        if (exact) return {boa::boa_search_kernel<VT, 1, CPL, (CPL > 0)>, 1, CPL == 0};
-        return {boa::boa_search_kernel<VT, 1, CPL, false>, 1, CPL == 0};
+        if (exact) return {boa::boa_search_kernel<VT, 1, W, CPL, (CPL > 0)>, W, CPL == 0};
+        return {boa::boa_search_kernel<VT, 1, W, CPL, false>, W, CPL == 0};
     }
-    if (exact) return {boa::boa_search_kernel<VT, 2, CPL, (CPL > 0)>, 2, CPL == 0};
-    return {boa::boa_search_kernel<VT, 2, CPL, false>, 2, CPL == 0};
+    if (exact) return {boa::boa_search_kernel<VT, 2, W, CPL, (CPL > 0)>, 2 * W, CPL == 0};
+    return {boa::boa_search_kernel<VT, 2, W, CPL, false>, 2 * W, CPL == 0};
+}
+template <int VT, int CPL>
+KernelChoice pick_rs(int R, bool exact, int expand_w)
+{
+    return expand_w == 2 ? pick_rn<VT, CPL, 2>(R, exact) : pick_rn<VT, CPL, 1>(R, exact);
 }
 
 KernelChoice pick_kernel(const boa_index* ix)
@@ -247,17 +252,17 @@ KernelChoice pick_kernel(const boa_index* ix)
     const bool exact = ix->nchunks == 8 * cpl;
     if (ix->vec_dtype == BOA_F32) {
         switch (cpl) {
-            case 1: return pick_rs<0, 1>(ix->R, exact);
-            case 2: return pick_rs<0, 2>(ix->R, exact);
-            case 3: return pick_rs<0, 3>(ix->R, exact);
-            case 4: return pick_rs<0, 4>(ix->R, exact);
-            default: return pick_rs<0, 0>(ix->R, false);
+            case 1: return pick_rs<0, 1>(ix->R, exact, ix->expand_w);
+            case 2: return pick_rs<0, 2>(ix->R, exact, ix->expand_w);
+            case 3: return pick_rs<0, 3>(ix->R, exact, ix->expand_w);
+            case 4: return pick_rs<0, 4>(ix->R, exact, ix->expand_w);
+            default: return pick_rs<0, 0>(ix->R, false, ix->expand_w);
         }
     }
     switch (cpl) {
-        case 1: return pick_rs<1, 1>(ix->R, exact);
-        case 2: return pick_rs<1, 2>(ix->R, exact);
-        default: return pick_rs<1, 0>(ix->R, false);
+        case 1: return pick_rs<1, 1>(ix->R, exact, ix->expand_w);
+        case 2: return pick_rs<1, 2>(ix->R, exact, ix->expand_w);
+        default: return pick_rs<1, 0>(ix->R, false, ix->expand_w);
     }
 }
 
@@ -568,6 +573,9 @@ int boa_set_param(boa_index* ix, int key, double v)
         case BOA_PARAM_MAX_WARPS_PER_SM:
             if (v < 0.0 || v > 64.0 || v != floor(v)) return BOA_EINVAL;
             ix->max_ctas = (int)v; return BOA_OK;
+        case BOA_PARAM_EXPAND_W:
+            if (v != 1.0 && v != 2.0) return BOA_EINVAL;
+            ix->expand_w = (int)v; return BOA_OK;
         default: return BOA_EINVAL;
     }
 }

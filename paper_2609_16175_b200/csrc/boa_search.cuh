@@ -240,10 +240,17 @@ __device__ __forceinline__ void sort_keys(uint64_t (&x)[RS], int lane)
 #pragma unroll
         for (int j = k >> 1; j > 0; j >>= 1) {
             if (j >= 32) {
-                if (RS == 2) {
-                    uint64_t a = x[0], b = x[RS - 1];
-                    x[0] = a < b ? a : b;
-                    x[RS - 1] = a < b ? b : a;
+                // partners sit in the same lane, t slots apart
+                const int t = j >> 5;
+#pragma unroll
+                for (int s = 0; s < RS; ++s) {
+                    if ((s & t) == 0 && (s | t) < RS) {
+                        const uint64_t a = x[s], b = x[s | t];
+                        const bool up = ((32 * s) & k) == 0;
+                        const uint64_t mn = a < b ? a : b, mx = a < b ? b : a;
+                        x[s] = up ? mn : mx;
+                        x[s | t] = up ? mx : mn;
+                    }
                 }
             } else {
 #pragma unroll
@@ -282,14 +289,17 @@ __host__ __device__ inline WarpSmem warp_smem_layout(int C, int table_buckets, i
 }
 
 // ---------------------------------------------------------------- the kernel
-// VT: 0 = float vectors, 1 = uint8 vectors.  RS: adjacency slots per lane (1: R <= 32,
-// 2: R <= 64).  CPL: 16-byte chunks of a row per lane of an 8-lane group when that is
+// VT: 0 = float vectors, 1 = uint8 vectors.  RN: adjacency slots per lane and node (1:
+// R <= 32, 2: R <= 64).  W: nodes expanded per iteration (1 = Algorithm 2 as printed; 2 =
+// the first two unexpanded beam entries together, an extension).  CPL: 16-byte chunks of a row per lane of an 8-lane group when that is
 // at most 4 (the lane then keeps its slices of the query in registers and the chunk
 // loop is unrolled); 0 = any length, query slices read from shared memory.  EXACT: the
 // row has exactly 8*CPL chunks, so no lane ever has a chunk missing.
-template <int VT, int RS, int CPL, bool EXACT>
+template <int VT, int RN, int W, int CPL, bool EXACT>
 __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(const SearchParams p)
 {
+    static_assert(W == 1 || W == 2, "expansion width 1 or 2");
+    constexpr int RS = RN * W;                      // adjacency slots per lane and iteration
     extern __shared__ __align__(128) uint8_t smem_raw[];
     const int lane = threadIdx.x;
     const int g = lane & 7;        // lane inside its 8-lane group
@@ -533,12 +543,13 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             }
             return -1;
         };
-        auto load_row_ids = [&](uint32_t id, uint32_t (&out)[RS]) {
-            const uint32_t* grow = p.graph + (size_t)id * p.R;
+        // adjacency row of node `id` into slots [base, base + RN); id == kNoId: an empty row
+        auto load_row_ids = [&](uint32_t id, uint32_t (&out)[RS], int base) {
+            const uint32_t* grow = p.graph + (size_t)(id == kNoId ? 0u : id) * p.R;
 #pragma unroll
-            for (int s = 0; s < RS; ++s) {
+            for (int s = 0; s < RN; ++s) {
                 const int j = lane + 32 * s;
-                out[s] = (j < p.R) ? __ldg(grow + j) : kNoId;
+                out[base + s] = (id != kNoId && j < p.R) ? __ldg(grow + j) : kNoId;
             }
         };
 
@@ -571,16 +582,26 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
         // ---- Algorithm 2 main loop
         BOA_T_MARK(0);
         int pos = first_unexpanded(0, n < p.L ? n : p.L);
+        int pos2 = -1;                 // W == 2: the second node of this iteration, or -1
         uint32_t nb[RS];
-        bool have_row = false;         // nb[] already holds the adjacency row of pool[pos]
+        bool have_row = false;         // nb[] already holds the adjacency rows of this iteration
         for (;;) {
             if (pos < 0) break;                                   // converged
             if (n_exp >= p.max_expand) { capped = true; break; }
-            if (!have_row) load_row_ids(key_id(pool[pos]), nb);
+            if (!have_row) {
+                load_row_ids(key_id(pool[pos]), nb, 0);
+                if (W > 1) {
+                    pos2 = (n_exp + 1 < p.max_expand) ? first_unexpanded(pos + 1, n < p.L ? n : p.L) : -1;
+                    load_row_ids(pos2 >= 0 ? key_id(pool[pos2]) : kNoId, nb, RN);
+                }
+            }
             __syncwarp();
-            if (lane == 0) pool[pos] |= 1ull;
-            cur = pos + 1;
-            n_exp++;
+            if (lane == 0) {
+                pool[pos] |= 1ull;
+                if (W > 1 && pos2 >= 0) pool[pos2] |= 1ull;
+            }
+            cur = ((W > 1 && pos2 >= 0) ? pos2 : pos) + 1;
+            n_exp += (W > 1 && pos2 >= 0) ? 2 : 1;
             have_row = false;
             BOA_T_MARK(1);
 
@@ -588,6 +609,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             int cnt = 0;
 #pragma unroll
             for (int s = 0; s < RS; ++s) {
+                if (W > 1 && s == RN) __syncwarp();   // the second row sees what the first recorded
                 const bool fresh = (nb[s] != kNoId) && hash_test_and_set(nb[s]);
                 const unsigned bal = __ballot_sync(0xffffffffu, fresh);
                 if (fresh) cand[cnt + __popc(bal & lt_mask)] = nb[s];
@@ -640,6 +662,20 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                 bool dup_s[RS];
 #pragma unroll
                 for (int s = 0; s < RS; ++s) { rank_s[s] = 0; dup_s[s] = false; }
+                if (W > 1) {
+                    // two rows of one iteration can hold the same id, and the table may have
+                    // forgotten it in between: equal keys are neighbours after the sort, the
+                    // later one is dropped
+#pragma unroll
+                    for (int s = 0; s < RS; ++s) {
+                        uint64_t pv = __shfl_up_sync(0xffffffffu, x[s], 1);
+                        if (s > 0) {
+                            const uint64_t last = __shfl_sync(0xffffffffu, x[s - 1], 31);
+                            if (lane == 0) pv = last;
+                        }
+                        dup_s[s] = (s > 0 || lane > 0) && x[s] != kKeyMax && pv == x[s];
+                    }
+                }
                 if (live <= 10) {
                     const int stride = (n + 31) >> 5;
                     const int pend = ((lane + 1) * stride < n) ? (lane + 1) * stride : n;
@@ -653,7 +689,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                         int r = base + __popc(__ballot_sync(0xffffffffu, e < xj));
                         r = r < n ? r : n;
                         const bool dj = __ballot_sync(0xffffffffu, e == xj) != 0u;
-                        if (j == lane) { rank_s[0] = r; dup_s[0] = dj; }
+                        if (j == lane) { rank_s[0] = r; dup_s[0] = dup_s[0] || dj; }
                     }
                 } else {
                     // many keys: every lane searches for its own (4-ary, same trip count for
@@ -679,7 +715,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                             hi_i = on ? nhi : hi_i;
                         }
                         rank_s[s] = lo_i;
-                        dup_s[s] = (lo_i < n) && ((pool[lo_i] | 1ull) == xo);
+                        dup_s[s] = dup_s[s] || ((lo_i < n) && ((pool[lo_i] | 1ull) == xo));
                     }
                 }
 #pragma unroll
@@ -719,7 +755,8 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             // ---- which node is expanded next?  Decide on the pool as it is, translate the
             // position, and start loading that node's adjacency row before the merge.
             {
-                const int pos_old = first_unexpanded(cur, n < p.L ? n : p.L);
+                const int lim_old = n < p.L ? n : p.L;
+                const int pos_old = first_unexpanded(cur, lim_old);
                 int pos_old_new = -1;
                 if (pos_old >= 0) {
                     int sh = 0;                       // kept keys ranked at or before it
@@ -730,20 +767,76 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                 }
                 const int n_new = (n + kept < p.C) ? n + kept : p.C;
                 const int lim_new = n_new < p.L ? n_new : p.L;
-                int next_pos;
-                uint32_t next_id;
-                if (pos_old_new < 0 || rmin < pos_old_new) {
-                    next_pos = rmin;                         // the smallest new key comes first
-                    next_id = key_id(first_new);
+                if (W == 1) {
+                    int next_pos;
+                    uint32_t next_id;
+                    if (pos_old_new < 0 || rmin < pos_old_new) {
+                        next_pos = rmin;                         // the smallest new key comes first
+                        next_id = key_id(first_new);
+                    } else {
+                        next_pos = pos_old_new;
+                        next_id = key_id(pool[pos_old]);
+                    }
+                    if (next_pos >= lim_new) next_pos = -1;
+                    pos = next_pos;
+                    if (pos >= 0 && n_exp < p.max_expand) {
+                        load_row_ids(next_id, nb, 0);
+                        have_row = true;
+                    }
                 } else {
-                    next_pos = pos_old_new;
-                    next_id = key_id(pool[pos_old]);
-                }
-                if (next_pos >= lim_new) next_pos = -1;
-                pos = next_pos;
-                if (pos >= 0 && n_exp < p.max_expand) {
-                    load_row_ids(next_id, nb);
-                    have_row = true;
+                    // the next two nodes are the two smallest merged places among: the first
+                    // two unexpanded old entries and the first two kept new keys
+                    constexpr int kNone = 0x7fffffff;
+                    const int a0 = pos_old_new >= 0 ? pos_old_new : kNone;
+                    const uint32_t a0id = pos_old >= 0 ? key_id(pool[pos_old]) : kNoId;
+                    int a1 = kNone;
+                    uint32_t a1id = kNoId;
+                    if (pos_old >= 0) {
+                        const int o2 = first_unexpanded(pos_old + 1, lim_old);
+                        if (o2 >= 0) {
+                            int sh = 0;
+#pragma unroll
+                            for (int s = 0; s < RS; ++s)
+                                sh += __popc(__ballot_sync(0xffffffffu, keep[s] && rank_s[s] <= o2));
+                            a1 = o2 + sh;
+                            a1id = key_id(pool[o2]);
+                        }
+                    }
+                    const int b0 = rmin;
+                    const uint32_t b0id = key_id(first_new);
+                    int b1 = kNone;
+                    uint32_t b1id = kNoId;
+                    {
+                        bool skipped = false;
+#pragma unroll
+                        for (int s = 0; s < RS; ++s) {
+                            unsigned mk = __ballot_sync(0xffffffffu, keep[s]);
+                            if (!skipped && mk) { mk &= mk - 1; skipped = true; }
+                            if (b1 == kNone && mk) {
+                                const int src = __ffs(mk) - 1;
+                                b1 = __shfl_sync(0xffffffffu, pos_new[s], src);
+                                b1id = key_id(__shfl_sync(0xffffffffu, x[s], src));
+                            }
+                        }
+                    }
+                    int p1, p2;
+                    uint32_t id1, id2;
+                    if (a0 < b0) {
+                        p1 = a0; id1 = a0id;
+                        if (a1 < b0) { p2 = a1; id2 = a1id; } else { p2 = b0; id2 = b0id; }
+                    } else {
+                        p1 = b0; id1 = b0id;
+                        if (a0 < b1) { p2 = a0; id2 = a0id; } else { p2 = b1; id2 = b1id; }
+                    }
+                    if (p1 >= lim_new) p1 = -1;
+                    if (p1 < 0 || p2 >= lim_new || !(n_exp + 1 < p.max_expand)) p2 = -1;
+                    pos = p1;
+                    pos2 = p2;
+                    if (pos >= 0 && n_exp < p.max_expand) {
+                        load_row_ids(id1, nb, 0);
+                        load_row_ids(pos2 >= 0 ? id2 : kNoId, nb, RN);
+                        have_row = true;
+                    }
                 }
             }
 

@@ -30,13 +30,14 @@ def make_pair(d, entry=-1):
 
 
 def gpu_search(gpu, g, k, widths, mode="restart", eps=0.05, tau=0.0, plus_k=0, cap=(8, 64),
-               sel=None):
+               sel=None, expand_w=1):
     gpu.set_param("mode", 1 if mode == "resume" else 0)
     gpu.set_param("eps", eps)
     gpu.set_param("tau", tau)
     gpu.set_param("plus_k", plus_k)
     gpu.set_param("cap_mult", cap[0])
     gpu.set_param("cap_add", cap[1])
+    gpu.set_param("expand_w", expand_w)
     gpu.set_schedule(list(widths))
     q, lo, hi = g["queries"], g["lo"], g["hi"]
     if sel is not None:

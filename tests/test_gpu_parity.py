@@ -47,6 +47,54 @@ def test_boa_matches_oracle_bit_for_bit(name, mode):
     assert len(set(o["final_L"].tolist())) > 1 or name == "c1"
 
 
+@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c5"])
+@pytest.mark.parametrize("mode", ["restart", "resume"])
+def test_expansion_width_2_matches_oracle_bit_for_bit(name, mode):
+    """Two nodes per iteration (an extension of Algorithm 2): same picks, same row order,
+    same cap accounting as the oracle run at the same width."""
+    w, d, orc, gpu, g = _get(name)
+    widths = default_widths(w.L0, min(w.Lmax, 256))
+    eps = {"c4": 0.2}.get(name, 0.05)
+    o = orc.search(d["queries"], d["lo"], d["hi"], w.k, widths, eps=eps, mode=mode, dist_mode=1,
+                   expand_w=2)
+    r = gpu_search(gpu, g, w.k, widths, eps=eps, mode=mode, expand_w=2)
+    assert_bit_parity(o, r, f"{name}/{mode}/W=2")
+    o1 = orc.search(d["queries"], d["lo"], d["hi"], w.k, widths, eps=eps, mode=mode, dist_mode=1)
+    assert (o1["n_expand"] != o["n_expand"]).any()        # the width does change the search
+
+
+def test_expansion_width_2_cap_and_boa_plus():
+    w, d, orc, gpu, g = _get("c2")
+    o = orc.search(d["queries"], d["lo"], d["hi"], w.k, [16, 64], cap=(1, 3), dist_mode=1, expand_w=2)
+    r = gpu_search(gpu, g, w.k, [16, 64], cap=(1, 3), expand_w=2)
+    assert (o["flags"] & 1).any() and (o["n_expand"] % 2 == 1).any()
+    assert_bit_parity(o, r, "cap/W=2")
+    o = orc.search(d["queries"], d["lo"], d["hi"], w.k, [16, 128], mode="resume", dist_mode=1, expand_w=2)
+    r = gpu_search(gpu, g, w.k, [16, 128], mode="resume", plus_k=3, expand_w=2)
+    assert_bit_parity(o, r, "BOA+/W=2")
+
+
+def test_stride_line_hand_trace_width_2_on_gpu():
+    """The width-2 hand trace of tests/golden/stride_trace_width2.txt, on the GPU."""
+    n = 16
+    x = np.zeros((n, 4), dtype=np.float32)
+    x[:, 0] = np.arange(n)
+    graph = np.full((n, 4), SENTINEL, dtype=np.uint32)
+    for i in range(n):
+        for c, o in enumerate((-2, -1, 1, 2)):
+            if 0 <= i + o < n:
+                graph[i, c] = i + o
+    d = dict(vectors=x, attrs=np.zeros((n, 1), np.int32), attr_types=np.zeros(1, np.int32), graph=graph,
+             queries=np.array([[10.1, 0, 0, 0]], dtype=np.float32),
+             lo=np.array([[0]], np.int32), hi=np.array([[0]], np.int32))
+    orc, gpu, g = make_pair(d, entry=0)
+    for w, n_exp in ((1, 7), (2, 12)):
+        r = gpu_search(gpu, g, 2, [2], expand_w=w)
+        assert r["ids"][0].tolist() == [10, 11]
+        assert r["n_expand"][0] == n_exp and r["n_scored"][0] == 13
+    gpu.close()
+
+
 @pytest.mark.parametrize("name", ["c2", "c4"])
 def test_integer_data_matches_double_accumulation_too(name):
     """Every partial sum of integer-valued rows is below 2^24, so the fp32 order cannot

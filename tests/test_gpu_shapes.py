@@ -59,6 +59,9 @@ def test_shape_variants_match_oracle(case):
             o = orc.search(d["queries"], d["lo"], d["hi"], k, widths, eps=eps, mode=mode, dist_mode=1)
             r = gpu_search(gpu, g, k, widths, mode=mode, eps=eps)
             assert_bit_parity(o, r, f"{name}/{mode}/eps={eps}")
+        o = orc.search(d["queries"], d["lo"], d["hi"], k, widths, mode=mode, dist_mode=1, expand_w=2)
+        r = gpu_search(gpu, g, k, widths, mode=mode, expand_w=2)
+        assert_bit_parity(o, r, f"{name}/{mode}/W=2")
     assert (r["ids"] != SENTINEL).any()
     gpu.close()
 
@@ -101,7 +104,12 @@ def test_many_random_small_cases():
         eps = float(rng.choice([0.02, 0.1, 0.4]))
         plus_k = int(rng.choice([0, 0, 3]))
         orc, gpu, g = make_pair(d)
-        o = orc.search(d["queries"], d["lo"], d["hi"], k, widths, eps=eps, mode=mode, dist_mode=1)
-        r = gpu_search(gpu, g, k, widths, mode=mode, eps=eps, plus_k=plus_k)
-        assert_bit_parity(o, r, f"case {case}: {dtype} D={D} m={m} R={R} N={N} k={k} {widths} {mode}")
+        for ew in (1, 2):
+            if ew == 2:
+                gpu.set_param("table_kb", int(rng.choice([0, 1])))   # a 1 KB table forgets at once
+            o = orc.search(d["queries"], d["lo"], d["hi"], k, widths, eps=eps, mode=mode, dist_mode=1,
+                           expand_w=ew)
+            r = gpu_search(gpu, g, k, widths, mode=mode, eps=eps, plus_k=plus_k, expand_w=ew)
+            assert_bit_parity(o, r, f"case {case}: {dtype} D={D} m={m} R={R} N={N} k={k} {widths} "
+                                    f"{mode} W={ew}")
         gpu.close()
