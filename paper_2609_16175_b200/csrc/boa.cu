@@ -269,9 +269,9 @@ KernelChoice pick_kernel(const boa_index* ix)
 // Table of recently scored ids: size in KB (a power of two, or three times one) -> bucket
 // count, bucket-group bits and the bits left for group-local addressing.  Tags are 16 bits.
 struct TableShape { int buckets, mul3, id_bits, low_bits; };
-TableShape choose_table(const boa_index* ix)
+TableShape choose_table(const boa_index* ix, int default_kb)
 {
-    int kb_size = ix->table_kb ? ix->table_kb : 6;     // default: 768 buckets, 3072 tags
+    int kb_size = ix->table_kb ? ix->table_kb : default_kb;
     TableShape t;
     t.id_bits = 1;
     while (((int64_t)1 << t.id_bits) < ix->N) ++t.id_bits;
@@ -289,6 +289,23 @@ TableShape choose_table(const boa_index* ix)
         kb_size *= 2;
     }
     return t;
+}
+
+// Default table size of a launch.  The register allocation lets 20 query warps live on an
+// SM; their shared memory (plus the 1 KB the system reserves per CTA) has to stay within
+// 196 KB, the largest carve-out that still leaves the L1 cache about 60 KB for the rows in
+// flight: with the next carve-out step (28 KB of L1) the same kernel ran 35 % slower on the
+// 1M x 128-d workload.  So: 6 KB (768 buckets, 3072 tags) when that fits, else 4 KB when
+// that fits; when neither does (long pools with R > 32, query vector in shared memory) fewer
+// warps fit anyway and the larger table wins.
+int default_table_kb(const boa_index* ix, const KernelChoice& kc, int C)
+{
+    const int sizes[2] = {6, 4};
+    for (int i = 0; i < 2; ++i) {
+        const boa::WarpSmem lay = boa::warp_smem_layout(C, sizes[i] * 128, ix->D, kc.rs, kc.q_in_smem);
+        if ((int64_t)BOA_MIN_CTAS * (lay.total + 1024) <= 196 * 1024) return sizes[i];
+    }
+    return 6;
 }
 
 int phase_widths(const boa_index* ix, int L0, int Lmax, int* w)
@@ -358,7 +375,7 @@ int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_p
     sp.L = L;
     sp.C = ix->mode == 1 ? Lmax : L;
     {
-        const TableShape t = choose_table(ix);
+        const TableShape t = choose_table(ix, default_table_kb(ix, lp.kc, sp.C));
         sp.table_buckets = t.buckets; sp.table_mul3 = t.mul3;
         sp.id_bits = t.id_bits; sp.low_bits = t.low_bits;
     }
