@@ -55,6 +55,7 @@ def parse_args():
     ap.add_argument("--expand-w", type=int, default=1, choices=[1, 2],
                     help="nodes expanded per iteration: 1 = Algorithm 2 as printed, 2 = extension")
     ap.add_argument("--table-kb", type=int, default=0)
+    ap.add_argument("--table-tags", type=int, default=0, choices=[0, 16])
     ap.add_argument("--max-warps", type=int, default=0)
     ap.add_argument("--fixed-L", type=int, default=0,
                     help="the paper's Fixed-L baseline: one phase at this beamwidth for every query")
@@ -283,6 +284,7 @@ def main():
     ix.set_param("plus_k", args.plus_k)
     ix.set_param("expand_w", args.expand_w)
     ix.set_param("table_kb", args.table_kb)
+    ix.set_param("table_tags", args.table_tags)
     ix.set_param("max_warps_per_sm", args.max_warps)
     ix.set_schedule(widths)
     Q, k = w.Q, w.k
@@ -391,7 +393,8 @@ def main():
     kernel_ms = float(np.mean(step_ms))
     achieved = alg_bytes / (kernel_ms / 1e3) / 1e9
     traffic = None
-    if (args.workload in NCU_DRAM_BYTES_PER_SCORED and not args.scale_n and not args.table_kb):
+    if (args.workload in NCU_DRAM_BYTES_PER_SCORED and not args.scale_n and not args.table_kb and not args.table_tags
+            and args.expand_w == 1):
         traffic = NCU_DRAM_BYTES_PER_SCORED[args.workload] * float(st["n_scored"].sum())
 
     line = {

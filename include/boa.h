@@ -52,13 +52,19 @@ enum {
                                Multiple Batches")                                            */
     BOA_PARAM_CAP_MULT = 5, /* a phase at width L gives up after CAP_MULT*L + CAP_ADD        */
     BOA_PARAM_CAP_ADD = 6,  /*   expansions; defaults 8 and 64                               */
-    BOA_PARAM_TABLE_KB = 7, /* 0 = default (6); else KB of shared memory per query for the
-                               table of recently scored ids: 1, 2, 3, 4, 6, 8, 12, 16 or 24
-                               (doubled automatically while an index of more than 2^25
-                               points needs tags wider than 16 bits).  Never changes
-                               results.                                                      */
+    BOA_PARAM_TABLE_KB = 7, /* 0 = default (6 or 4, whichever keeps 20 query warps per SM
+                               within 196 KB of shared memory); else KB of shared memory
+                               per query for the table of recently scored ids: 1, 2, 3, 4,
+                               6, 8, 12, 16 or 24 (doubled automatically while an index of
+                               more than 2^25 points needs tags wider than 16 bits).  Never
+                               changes results.                                              */
     BOA_PARAM_MAX_WARPS_PER_SM = 8, /* 0 = as many query warps per SM as fit; else a cap.
                                Never changes results.                                        */
+    BOA_PARAM_TABLE_TAGS = 10, /* 0 (default) = the table keeps 10-bit tags, three to a 4-byte
+                               bucket, when the index is small enough for that (up to 2^20
+                               points with the default 4 KB), else 16-bit tags, four to an
+                               8-byte bucket; 16 = always the latter.  Never changes
+                               results.                                                      */
     BOA_PARAM_EXPAND_W = 9  /* nodes expanded per iteration of Algorithm 2.  1 (default) is
                                the algorithm as printed ("each iteration expands one
                                node").  2 is an extension: the first two unexpanded beam

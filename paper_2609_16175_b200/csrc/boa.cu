@@ -159,7 +159,7 @@ struct boa_index {
     int device = 0, num_sms = 0;
     // parameters
     double eps = 0.05, growth = 4.0, tau = 0.0;
-    int mode = 0, plus_k = 0, cap_mult = 8, cap_add = 64, table_kb = 0, max_ctas = 0, expand_w = 1;
+    int mode = 0, plus_k = 0, cap_mult = 8, cap_add = 64, table_kb = 0, max_ctas = 0, expand_w = 1, table_tags = 0;
     int n_sched = 0;
     int sched[BOA_MAX_PHASES] = {0};
     // scratch
@@ -267,8 +267,10 @@ KernelChoice pick_kernel(const boa_index* ix)
 }
 
 // Table of recently scored ids: size in KB (a power of two, or three times one) -> bucket
-// count, bucket-group bits and the bits left for group-local addressing.  Tags are 16 bits.
-struct TableShape { int buckets, mul3, id_bits, low_bits; };
+// count, bucket-group bits and the bits left for group-local addressing.  Buckets are 4
+// bytes (three 10-bit tags) when the tags of this index fit 10 bits at that bucket count,
+// else 8 bytes (four 16-bit tags).  `tags` forces the wide form when it is 16.
+struct TableShape { int bytes, narrow, mul3, id_bits, low_bits; };
 TableShape choose_table(const boa_index* ix, int default_kb)
 {
     int kb_size = ix->table_kb ? ix->table_kb : default_kb;
@@ -277,18 +279,22 @@ TableShape choose_table(const boa_index* ix, int default_kb)
     while (((int64_t)1 << t.id_bits) < ix->N) ++t.id_bits;
     for (;;) {
         t.mul3 = (kb_size % 3 == 0) ? 1 : 0;
-        const int groups = (t.mul3 ? kb_size / 3 : kb_size) * 128;     // 2^kb
-        int kb = 0;
-        while ((1 << kb) < groups) ++kb;
-        if (kb > t.id_bits) kb = t.id_bits;
-        t.low_bits = t.id_bits - kb;
-        t.buckets = (t.mul3 ? 3 : 1) << kb;
-        // the largest tag must stay below 0xFFFF (the empty mark)
-        const uint32_t max_tag = ((1u << t.low_bits) - 1u) / (t.mul3 ? 3u : 1u);
-        if (max_tag < 0xFFFFu || kb_size >= 1024) break;
+        t.bytes = kb_size * 1024;
+        for (t.narrow = (ix->table_tags == 16 ? 0 : 1); t.narrow >= 0; --t.narrow) {
+            const int groups = (t.mul3 ? kb_size / 3 : kb_size) * (t.narrow ? 256 : 128);   // 2^kb
+            int kb = 0;
+            while ((1 << kb) < groups) ++kb;
+            if (kb > t.id_bits) kb = t.id_bits;
+            t.low_bits = t.id_bits - kb;
+            // tags must fit; an id whose tag is all ones (the empty mark) is simply never
+            // recorded, which the narrow form accepts for one id in 1024
+            const uint32_t max_tag = ((1u << t.low_bits) - 1u) / (t.mul3 ? 3u : 1u);
+            if (t.narrow ? max_tag <= 0x3FFu : max_tag < 0xFFFFu) return t;
+        }
+        t.narrow = 0;
+        if (kb_size >= 1024) return t;
         kb_size *= 2;
     }
-    return t;
 }
 
 // Default table size of a launch.  The register allocation lets 20 query warps live on an
@@ -302,7 +308,7 @@ int default_table_kb(const boa_index* ix, const KernelChoice& kc, int C)
 {
     const int sizes[2] = {6, 4};
     for (int i = 0; i < 2; ++i) {
-        const boa::WarpSmem lay = boa::warp_smem_layout(C, sizes[i] * 128, ix->D, kc.rs, kc.q_in_smem);
+        const boa::WarpSmem lay = boa::warp_smem_layout(C, sizes[i] * 1024, ix->D, kc.rs, kc.q_in_smem);
         if ((int64_t)BOA_MIN_CTAS * (lay.total + 1024) <= 196 * 1024) return sizes[i];
     }
     return 6;
@@ -376,7 +382,7 @@ int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_p
     sp.C = ix->mode == 1 ? Lmax : L;
     {
         const TableShape t = choose_table(ix, default_table_kb(ix, lp.kc, sp.C));
-        sp.table_buckets = t.buckets; sp.table_mul3 = t.mul3;
+        sp.table_bytes = t.bytes; sp.table_narrow = t.narrow; sp.table_mul3 = t.mul3;
         sp.id_bits = t.id_bits; sp.low_bits = t.low_bits;
     }
     sp.max_expand = ix->cap_mult * L + ix->cap_add;
@@ -396,7 +402,7 @@ int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_p
     sp.out_list = lists_c + (size_t)(p + 1 < BOA_MAX_PHASES ? p + 1 : p) * ix->ws_Q;
     sp.out_count = cnt_c + p + 1;
 
-    const boa::WarpSmem lay = boa::warp_smem_layout(sp.C, sp.table_buckets, ix->D, lp.kc.rs, lp.kc.q_in_smem);
+    const boa::WarpSmem lay = boa::warp_smem_layout(sp.C, sp.table_bytes, ix->D, lp.kc.rs, lp.kc.q_in_smem);
     const size_t smem = (size_t)lay.total;
     if (smem > 48 * 1024) {
         BOA_CUDA(cudaFuncSetAttribute((const void*)lp.kc.fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -590,6 +596,9 @@ int boa_set_param(boa_index* ix, int key, double v)
         case BOA_PARAM_MAX_WARPS_PER_SM:
             if (v < 0.0 || v > 64.0 || v != floor(v)) return BOA_EINVAL;
             ix->max_ctas = (int)v; return BOA_OK;
+        case BOA_PARAM_TABLE_TAGS:
+            if (v != 0.0 && v != 16.0) return BOA_EINVAL;
+            ix->table_tags = (int)v; return BOA_OK;
         case BOA_PARAM_EXPAND_W:
             if (v != 1.0 && v != 2.0) return BOA_EINVAL;
             ix->expand_w = (int)v; return BOA_OK;

@@ -20,8 +20,9 @@
 // 128-d workload because the kernel is bound by instruction issue and dependent
 // latency, not by the number of bytes in flight.
 //
-// The table of recently scored ids stores 16-bit tags in 4-way buckets (least recently
-// met way replaced).  An id is first mapped by an odd multiplier modulo 2^id_bits (a
+// The table of recently scored ids stores 16-bit tags in 4-way buckets of 8 bytes or, when
+// the index is small enough for 10-bit tags, 10-bit tags in 3-way buckets of 4 bytes (half
+// again as many ids in the same shared memory); the least recently met way is replaced.  An id is first mapped by an odd multiplier modulo 2^id_bits (a
 // bijection); the high bits pick the bucket (with 3*2^kb buckets: the bucket group, and
 // the low part modulo 3 the bucket inside it) and the rest is the tag, so bucket + tag
 // identify the id exactly: the table can forget an id, it can never report an unseen id
@@ -91,8 +92,9 @@ struct SearchParams {
     // phase
     int L;                    // beamwidth: expandable prefix of the pool
     int C;                    // pool capacity (L in restart mode, Lmax in resume mode)
-    int table_buckets;        // 4-way buckets in the table of recently scored ids: 2^kb or 3*2^kb
-    int table_mul3;           // 1 when the bucket count is 3*2^kb
+    int table_bytes;          // shared memory of the table of recently scored ids (multiple of 16)
+    int table_narrow;         // 0: 8-byte buckets of four 16-bit tags; 1: 4-byte buckets of three 10-bit tags
+    int table_mul3;           // 1 when the bucket count is 3*2^kb, 0 when it is 2^kb
     int id_bits;              // bits of a node id (ids < 2^id_bits)
     int low_bits;             // id_bits - kb: bits of a mapped id below its bucket group
     int max_expand;           // expansions after which a phase gives up
@@ -276,14 +278,14 @@ struct WarpSmem {
 };
 // q_in_smem: the query vector is kept in shared memory (only when lanes do not hold their
 // slices of it in registers).
-__host__ __device__ inline WarpSmem warp_smem_layout(int C, int table_buckets, int D, int RS, bool q_in_smem)
+__host__ __device__ inline WarpSmem warp_smem_layout(int C, int table_bytes, int D, int RS, bool q_in_smem)
 {
     WarpSmem s;
     int off = 0;
     s.pool_off = off;  off += ((C + 1) & ~1) * 8;
     s.nk_off = off;    off += 32 * RS * 8;
     s.q_off = off;     off += q_in_smem ? ((D * 4 + 15) & ~15) : 0;
-    s.hash_off = off;  off += table_buckets * 8;
+    s.hash_off = off;  off += table_bytes;
     s.cand_off = off;  off += 32 * RS * 4;
     s.nr_off = off;    off += 32 * RS * 4;
     s.total = (off + 127) & ~127;
@@ -310,7 +312,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
     constexpr int QF4 = (VT == 0) ? 1 : 4;          // float4 slices of the query per chunk
     constexpr int NQ = (CPL > 0) ? CPL * QF4 : 1;
 
-    const WarpSmem lay = warp_smem_layout(p.C, p.table_buckets, p.D, RS, CPL == 0);
+    const WarpSmem lay = warp_smem_layout(p.C, p.table_bytes, p.D, RS, CPL == 0);
     uint64_t* pool = reinterpret_cast<uint64_t*>(smem_raw + lay.pool_off);
     uint64_t* nk = reinterpret_cast<uint64_t*>(smem_raw + lay.nk_off);
     uint32_t* nr = reinterpret_cast<uint32_t*>(smem_raw + lay.nr_off);
@@ -347,7 +349,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             }
             const uint4 ff = make_uint4(~0u, ~0u, ~0u, ~0u);
             uint4* h4 = reinterpret_cast<uint4*>(hash);
-            for (int i = lane; i < p.table_buckets / 2; i += 32) h4[i] = ff;
+            for (int i = lane; i < p.table_bytes / 16; i += 32) h4[i] = ff;
         }
         int32_t my_lo = 0, my_hi = 0;
         if (g < p.m) {
@@ -521,14 +523,24 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             const uint32_t third = __umulhi(low, 0xAAAAAAABu) >> 1;        // low / 3
             const uint32_t tag = p.table_mul3 ? third : low;
             const uint32_t bucket = p.table_mul3 ? top * 3u + (low - 3u * third) : top;
+            // least recently met first out: the tag moves (or enters) to way 0, the ways
+            // before its old place move up by one, a new tag pushes the last way out.  The
+            // all-ones tag marks an empty way: an id with that tag is never recorded.
+            if (p.table_narrow) {
+                uint32_t* slot = reinterpret_cast<uint32_t*>(hash) + bucket;
+                const uint32_t b = *slot;
+                const uint32_t w0 = b & 0x3FFu, w1 = (b >> 10) & 0x3FFu, w2 = (b >> 20) & 0x3FFu;
+                const bool found = (w0 == tag) | (w1 == tag) | (w2 == tag);
+                const bool fresh = !found | (tag == 0x3FFu);
+                if (tag != 0x3FFu && w0 != tag)
+                    *slot = tag | (w0 << 10) | (((w1 == tag) ? w2 : w1) << 20) | 0xC0000000u;
+                return fresh;
+            }
             uint2* slot = reinterpret_cast<uint2*>(hash + 4 * bucket);
             const uint2 b = *slot;
             const uint32_t w0 = b.x & 0xFFFFu, w1 = b.x >> 16, w2 = b.y & 0xFFFFu, w3 = b.y >> 16;
             const bool found = (w0 == tag) | (w1 == tag) | (w2 == tag) | (w3 == tag);
-            // a tag of 0xFFFF would look like an empty way: such an id is never recorded
             const bool fresh = !found | (tag == 0xFFFFu);
-            // least recently met first out: the tag moves (or enters) to way 0, the ways
-            // before its old place move up by one, a new tag pushes the last way out
             if (tag != 0xFFFFu && w0 != tag) {
                 const uint32_t hi = (w1 == tag) ? b.y : (w1 | (((w2 == tag) ? w3 : w2) << 16));
                 *slot = make_uint2(tag | (w0 << 16), hi);

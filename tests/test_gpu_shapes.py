@@ -104,6 +104,7 @@ def test_many_random_small_cases():
         eps = float(rng.choice([0.02, 0.1, 0.4]))
         plus_k = int(rng.choice([0, 0, 3]))
         orc, gpu, g = make_pair(d)
+        gpu.set_param("table_tags", 16 if case % 2 else 0)       # both bucket formats
         for ew in (1, 2):
             if ew == 2:
                 gpu.set_param("table_kb", int(rng.choice([0, 1])))   # a 1 KB table forgets at once
