@@ -301,13 +301,14 @@ TableShape choose_table(const boa_index* ix, int default_kb)
 // SM; their shared memory (plus the 1 KB the system reserves per CTA) has to stay within
 // 196 KB, the largest carve-out that still leaves the L1 cache about 60 KB for the rows in
 // flight: with the next carve-out step (28 KB of L1) the same kernel ran 35 % slower on the
-// 1M x 128-d workload.  So: 6 KB (768 buckets, 3072 tags) when that fits, else 4 KB when
-// that fits; when neither does (long pools with R > 32, query vector in shared memory) fewer
-// warps fit anyway and the larger table wins.
+// 1M x 128-d workload.  So: the largest of 6, 4, 3, 2 KB that fits.  Rows shorter than 256
+// bytes need little L1 and take 6 KB; so does a launch that no size fits (query vector in
+// shared memory): fewer warps are resident then anyway.
 int default_table_kb(const boa_index* ix, const KernelChoice& kc, int C)
 {
-    const int sizes[2] = {6, 4};
-    for (int i = 0; i < 2; ++i) {
+    if (ix->rec_stride < 256) return 6;
+    const int sizes[4] = {6, 4, 3, 2};
+    for (int i = 0; i < 4; ++i) {
         const boa::WarpSmem lay = boa::warp_smem_layout(C, sizes[i] * 1024, ix->D, kc.rs, kc.q_in_smem);
         if ((int64_t)BOA_MIN_CTAS * (lay.total + 1024) <= 196 * 1024) return sizes[i];
     }

@@ -274,7 +274,7 @@ __device__ __forceinline__ void sort_keys(uint64_t (&x)[RS], int lane)
 
 // Per-warp shared memory carve-up (bytes), shared by host and device.
 struct WarpSmem {
-    int pool_off, nk_off, nr_off, cand_off, hash_off, q_off, total;
+    int pool_off, nk_off, cand_off, hash_off, q_off, total;
 };
 // q_in_smem: the query vector is kept in shared memory (only when lanes do not hold their
 // slices of it in registers).
@@ -287,7 +287,6 @@ __host__ __device__ inline WarpSmem warp_smem_layout(int C, int table_bytes, int
     s.q_off = off;     off += q_in_smem ? ((D * 4 + 15) & ~15) : 0;
     s.hash_off = off;  off += table_bytes;
     s.cand_off = off;  off += 32 * RS * 4;
-    s.nr_off = off;    off += 32 * RS * 4;
     s.total = (off + 127) & ~127;
     return s;
 }
@@ -315,7 +314,6 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
     const WarpSmem lay = warp_smem_layout(p.C, p.table_bytes, p.D, RS, CPL == 0);
     uint64_t* pool = reinterpret_cast<uint64_t*>(smem_raw + lay.pool_off);
     uint64_t* nk = reinterpret_cast<uint64_t*>(smem_raw + lay.nk_off);
-    uint32_t* nr = reinterpret_cast<uint32_t*>(smem_raw + lay.nr_off);
     uint32_t* cand = reinterpret_cast<uint32_t*>(smem_raw + lay.cand_off);
     uint16_t* hash = reinterpret_cast<uint16_t*>(smem_raw + lay.hash_off);
     float4* qs = reinterpret_cast<float4*>(smem_raw + lay.q_off);
@@ -860,7 +858,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             // group before its writes (a source never lies above its destination).
             {
                 uint32_t* occ = cand;                    // 32 words: places < 1024
-                uint32_t* pre = nr;                      // new places before each word
+                uint32_t* pre = reinterpret_cast<uint32_t*>(nk);   // new places before each word (nk is free here)
                 occ[lane] = 0u;
                 __syncwarp();
 #pragma unroll
