@@ -17,8 +17,9 @@
  *   orc_boa_search     multi-phase driver (Algorithm 1)
  *
  * Readings of points the paper leaves open (each is listed in the design notes):
- *   - the score dist + lambda*phi is taken in its lambda -> infinity limit: keys
- *     order by (phi, d2, id) lexicographically; id breaks every tie
+ *   - the score dist + lambda*phi is taken in its lambda -> infinity limit by default:
+ *     keys order by (phi, d2, id) lexicographically; id breaks every tie.  A finite
+ *     lambda can be set: score = d2 + lambda*phi on squared distances, order (score, id)
  *   - "visited" means two things in Algorithm 2: a node already scored ("seen",
  *     the Bloom filter line, here an exact set) and a node already expanded (a
  *     flag on the worklist entry, the convergence line)
@@ -211,6 +212,7 @@ int64_t orc_bruteforce(const orc_index *ix, const float *q, const int32_t *lo, c
 typedef struct {
     int phi;
     float d2;
+    float score;         /* d2 + lambda*phi (finite lambda only) */
     uint32_t id;
     int expanded;
 } orc_entry_t;
@@ -219,7 +221,8 @@ typedef struct {
     const orc_index *ix;
     int C;               /* pool capacity */
     int size;
-    orc_entry_t *pool;   /* C + R slots, ascending by (phi, d2, id) */
+    orc_entry_t *pool;   /* ascending by (phi, d2, id), or by (score, id) with a finite lambda */
+    float lambda;        /* weight of the filter penalty; INFINITY = lexicographic order */
     uint8_t *seen;       /* [N] */
     uint32_t *touched;   /* ids set in seen, for a cheap reset */
     int64_t ntouched, touched_cap;
@@ -227,23 +230,33 @@ typedef struct {
     int hit_cap;
 } orc_state;
 
-static int orc_less(const orc_entry_t *a, const orc_entry_t *b)
+/* The order the search works by.  The paper's score is dist + lambda*phi with one lambda
+   for all attributes.  lambda = INFINITY is its limit: any violated predicate outweighs
+   any distance, so keys compare by (phi, d2).  A finite lambda gives score = d2 +
+   lambda*phi, one fused multiply-add in fp32.  The node id breaks ties either way. */
+static int orc_less(const orc_state *st, const orc_entry_t *a, const orc_entry_t *b)
 {
-    if (a->phi != b->phi) return a->phi < b->phi;
-    if (a->d2 != b->d2) return a->d2 < b->d2;
+    if (isinf(st->lambda)) {
+        if (a->phi != b->phi) return a->phi < b->phi;
+        if (a->d2 != b->d2) return a->d2 < b->d2;
+    } else {
+        if (a->score != b->score) return a->score < b->score;
+    }
     return a->id < b->id;
 }
 
 orc_state *orc_state_new(const orc_index *ix, int C)
 {
     orc_state *st = (orc_state *)calloc(1, sizeof(orc_state));
-    st->ix = ix; st->C = C;
+    st->ix = ix; st->C = C; st->lambda = INFINITY;
     st->pool = (orc_entry_t *)calloc((size_t)C + (size_t)ORC_MAX_W * ix->R + 1, sizeof(orc_entry_t));
     st->seen = (uint8_t *)calloc((size_t)ix->N, 1);
     st->touched_cap = 1024;
     st->touched = (uint32_t *)malloc((size_t)st->touched_cap * sizeof(uint32_t));
     return st;
 }
+/* set before orc_beam_init; lambda >= 0, INFINITY for the lexicographic order */
+void orc_state_set_lambda(orc_state *st, float lambda) { st->lambda = lambda; }
 void orc_state_free(orc_state *st)
 {
     free(st->pool); free(st->seen); free(st->touched); free(st);
@@ -262,7 +275,8 @@ static void orc_mark_seen(orc_state *st, uint32_t id)
 static void orc_pool_insert(orc_state *st, orc_entry_t e)
 {
     int pos = st->size;
-    while (pos > 0 && orc_less(&e, &st->pool[pos - 1])) { st->pool[pos] = st->pool[pos - 1]; pos--; }
+    e.score = isinf(st->lambda) ? e.d2 : fmaf(st->lambda, (float)e.phi, e.d2);
+    while (pos > 0 && orc_less(st, &e, &st->pool[pos - 1])) { st->pool[pos] = st->pool[pos - 1]; pos--; }
     st->pool[pos] = e;
     st->size++;
 }
@@ -431,10 +445,10 @@ static void orc_restore(orc_state *st, const orc_saved *sv, int C)
  * add up over the phases a query ran; flags bit 0 = some phase hit its
  * expansion cap.
  */
-void orc_boa_search_w(const orc_index *ix, const float *queries, int64_t Q,
+void orc_boa_search_wl(const orc_index *ix, const float *queries, int64_t Q,
                       const int32_t *lo, const int32_t *hi, int k,
                       const int32_t *widths, int n_widths, double eps, double tau,
-                      int mode, int dist_mode, int cap_mult, int cap_add, int W,
+                      int mode, int dist_mode, int cap_mult, int cap_add, int W, float lambda,
                       uint32_t *out_ids, float *out_d2,
                       int32_t *final_L, int32_t *n_expand, int32_t *n_scored, int32_t *flags,
                       int64_t *phase_active)
@@ -442,6 +456,7 @@ void orc_boa_search_w(const orc_index *ix, const float *queries, int64_t Q,
     int Cmax = 0;
     for (int p = 0; p < n_widths; ++p) if (widths[p] > Cmax) Cmax = widths[p];
     orc_state *st = orc_state_new(ix, Cmax);
+    orc_state_set_lambda(st, lambda);
     for (int p = 0; p < n_widths; ++p) phase_active[p] = 0;
 
     uint8_t *active = (uint8_t *)malloc((size_t)Q + 1);             /* the set A */
@@ -483,6 +498,20 @@ void orc_boa_search_w(const orc_index *ix, const float *queries, int64_t Q,
     free(saved);
     free(active);
     orc_state_free(st);
+}
+
+/* lexicographic order (lambda -> infinity), any expansion width */
+void orc_boa_search_w(const orc_index *ix, const float *queries, int64_t Q,
+                      const int32_t *lo, const int32_t *hi, int k,
+                      const int32_t *widths, int n_widths, double eps, double tau,
+                      int mode, int dist_mode, int cap_mult, int cap_add, int W,
+                      uint32_t *out_ids, float *out_d2,
+                      int32_t *final_L, int32_t *n_expand, int32_t *n_scored, int32_t *flags,
+                      int64_t *phase_active)
+{
+    orc_boa_search_wl(ix, queries, Q, lo, hi, k, widths, n_widths, eps, tau, mode, dist_mode,
+                      cap_mult, cap_add, W, INFINITY, out_ids, out_d2, final_L, n_expand, n_scored,
+                      flags, phase_active);
 }
 
 /* the paper's setting: expansion width 1 */

@@ -37,6 +37,7 @@ def lib():
         L.orc_state_new.restype = vp
         L.orc_state_new.argtypes = [vp, i32]
         L.orc_state_free.argtypes = [vp]
+        L.orc_state_set_lambda.argtypes = [vp, C.c_float]
         L.orc_beam_init.argtypes = [vp, i32, vp, vp, vp, i32]
         L.orc_beam_run.argtypes = [vp, i32, vp, vp, vp, i32, i64]
         L.orc_beam_run_w.argtypes = [vp, i32, vp, vp, vp, i32, i64, i32]
@@ -57,6 +58,8 @@ def lib():
                                      i32, i32, vp, vp, vp, vp, vp, vp, vp]
         L.orc_boa_search_w.argtypes = [vp, vp, i64, vp, vp, i32, vp, i32, dbl, dbl, i32, i32,
                                        i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.orc_boa_search_wl.argtypes = [vp, vp, i64, vp, vp, i32, vp, i32, dbl, dbl, i32, i32,
+                                        i32, i32, i32, C.c_float, vp, vp, vp, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -130,13 +133,14 @@ class OracleIndex:
         return ids, d2, nvalid
 
     # --- one beam search, step-wise ------------------------------------------
-    def beam(self, q, lo, hi, L, C=None, dist_mode=0, max_expand=1 << 40, expand_w=1):
+    def beam(self, q, lo, hi, L, C=None, dist_mode=0, max_expand=1 << 40, expand_w=1,
+             lam=float("inf")):
         return OracleBeam(self, q, lo, hi, L, C if C is not None else L, dist_mode, max_expand,
-                          expand_w)
+                          expand_w, lam)
 
     # --- the multi-phase batch driver ----------------------------------------
     def search(self, queries, lo, hi, k, widths, eps=0.05, tau=0.0, mode="restart",
-               dist_mode=0, cap=DEFAULT_CAP, expand_w=1):
+               dist_mode=0, cap=DEFAULT_CAP, expand_w=1, lam=float("inf")):
         queries = np.ascontiguousarray(queries, dtype=np.float32)
         lo = np.ascontiguousarray(lo, dtype=np.int32)
         hi = np.ascontiguousarray(hi, dtype=np.int32)
@@ -149,9 +153,9 @@ class OracleIndex:
         n_scored = np.empty(Q, dtype=np.int32)
         flags = np.empty(Q, dtype=np.int32)
         phase_active = np.zeros(len(w), dtype=np.int64)
-        lib().orc_boa_search_w(self.h, _p(queries), Q, _p(lo), _p(hi), k, _p(w), len(w),
+        lib().orc_boa_search_wl(self.h, _p(queries), Q, _p(lo), _p(hi), k, _p(w), len(w),
                                float(eps), float(tau), 1 if mode == "resume" else 0, int(dist_mode),
-                               int(cap[0]), int(cap[1]), int(expand_w), _p(ids), _p(d2), _p(final_L),
+                               int(cap[0]), int(cap[1]), int(expand_w), float(lam), _p(ids), _p(d2), _p(final_L),
                                _p(n_expand), _p(n_scored), _p(flags), _p(phase_active))
         return dict(ids=ids, d2=d2, final_L=final_L, n_expand=n_expand, n_scored=n_scored,
                     flags=flags, phase_active=phase_active)
@@ -160,7 +164,7 @@ class OracleIndex:
 class OracleBeam:
     """One query's Algorithm-2 state, for tests that look inside a search."""
 
-    def __init__(self, index, q, lo, hi, L, C, dist_mode, max_expand, expand_w=1):
+    def __init__(self, index, q, lo, hi, L, C, dist_mode, max_expand, expand_w=1, lam=float("inf")):
         self.ix = index
         self.expand_w = int(expand_w)
         self.q = np.ascontiguousarray(q, dtype=np.float32)
@@ -168,6 +172,7 @@ class OracleBeam:
         self.hi = np.ascontiguousarray(hi, dtype=np.int32)
         self.dist_mode = dist_mode
         self.st = lib().orc_state_new(index.h, int(C))
+        lib().orc_state_set_lambda(self.st, float(lam))
         lib().orc_beam_init(self.st, int(C), _p(self.q), _p(self.lo), _p(self.hi), dist_mode)
         self.run(L, max_expand)
 

@@ -228,6 +228,64 @@ def test_ring_walk_passes_through_invalid_nodes():
 
 
 # ----------------------------------------------------------------------------
+# finite lambda: the score dist + lambda*phi as the paper states it
+# ----------------------------------------------------------------------------
+def test_ring_hand_traces_with_finite_lambda():
+    gold = {r[0]: [int(v) for v in r[1:]] for r in _read_golden("ring_trace_finite_lambda.txt")}
+    ix = _ring()
+    q = np.array([5.2], dtype=np.float32)
+    one = np.array([1], dtype=np.int32)
+    for lam, tag in ((2.0, "l2"), (0.5, "l05")):
+        b = ix.beam(q, one, one, L=3, C=3, lam=lam)
+        assert b.n_expand == len(gold[tag + "_expansions"])
+        assert b.n_scored == len(gold[tag + "_scored"])
+        ids, d2, phi, ex = b.pool()
+        assert [int(i) for i in ids] == gold[tag + "_final_pool"]
+        rid, rd2, n = b.result(2)
+        assert [int(i) for i in rid[:n]] == gold[tag + "_result_ids"]
+        assert (rid[n:] == SENTINEL).all()
+    # the lexicographic order expands node 1, lambda = 2 does not
+    assert ix.beam(q, one, one, L=3, C=3).n_expand == 5
+
+
+def test_lambda_zero_walks_like_an_unfiltered_search(small):
+    """With lambda = 0 the predicates cannot steer the walk: the pool is that of a search
+    whose ranges admit everything, and the answer is its filter-valid part."""
+    w, d, ix = small
+    everything_lo = np.full(w.m, np.iinfo(np.int32).min, dtype=np.int32)
+    everything_hi = np.full(w.m, np.iinfo(np.int32).max, dtype=np.int32)
+    for i in range(8):
+        a = ix.beam(d["queries"][i], d["lo"][i], d["hi"][i], L=32, lam=0.0)
+        b = ix.beam(d["queries"][i], everything_lo, everything_hi, L=32)
+        assert (a.pool()[0] == b.pool()[0]).all() and a.n_scored == b.n_scored
+        ok = _valid_mask(d, i)
+        want = [int(v) for v in b.pool()[0] if ok[int(v)]][:w.k]
+        got = a.result(w.k)
+        assert [int(v) for v in got[0][:got[2]]] == want
+
+
+def test_large_exact_lambda_equals_the_lexicographic_order():
+    """Integer data with every d2 < 1024 and lambda = 1024: the score d2 + 1024*phi is exact
+    in fp32 and orders like (phi, d2), so the two searches are the same search."""
+    rng = np.random.default_rng(5)
+    N, D, R, k = 400, 4, 6, 5
+    x = rng.integers(0, 16, size=(N, D)).astype(np.float32)          # d2 <= 4*15^2 = 900
+    attrs = rng.integers(0, 10, size=(N, 3)).astype(np.int32)
+    g = rng.integers(0, N, size=(N, R)).astype(np.uint32)
+    g[:, 0] = (np.arange(N) + 1) % N
+    ix = OracleIndex(x, attrs, np.zeros(3, np.int32), g)
+    q = rng.integers(0, 16, size=(12, D)).astype(np.float32)
+    lo = rng.integers(0, 5, size=(12, 3)).astype(np.int32)
+    hi = (lo + rng.integers(0, 5, size=(12, 3))).astype(np.int32)
+    a = ix.search(q, lo, hi, k, [6, 24], mode="resume", lam=1024.0)
+    b = ix.search(q, lo, hi, k, [6, 24], mode="resume")
+    for key in ("ids", "d2", "final_L", "n_expand", "n_scored"):
+        assert (a[key] == b[key]).all(), key
+    c = ix.search(q, lo, hi, k, [6, 24], mode="resume", lam=8.0)      # a small lambda does differ
+    assert (c["n_scored"] != b["n_scored"]).any()
+
+
+# ----------------------------------------------------------------------------
 # expansion width W > 1 (an extension of Algorithm 2): a second hand trace
 # ----------------------------------------------------------------------------
 def _stride_line():
