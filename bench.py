@@ -54,6 +54,8 @@ def parse_args():
     ap.add_argument("--plus-k", type=int, default=0)
     ap.add_argument("--expand-w", type=int, default=1, choices=[1, 2],
                     help="nodes expanded per iteration: 1 = Algorithm 2 as printed, 2 = extension")
+    ap.add_argument("--lam", type=float, default=float("inf"),
+                    help="weight of the filter penalty; default infinity = lexicographic keys")
     ap.add_argument("--table-kb", type=int, default=0)
     ap.add_argument("--table-tags", type=int, default=0, choices=[0, 16])
     ap.add_argument("--max-warps", type=int, default=0)
@@ -194,12 +196,12 @@ def run_oracle_sample(w, d, widths, args, seconds, dist_mode=1):
     probe = min(8, w.Q)
     t0 = time.perf_counter()
     orc.search(d["queries"][:probe], d["lo"][:probe], d["hi"][:probe], w.k, widths, eps=args.eps,
-               mode=args.mode, dist_mode=dist_mode, expand_w=args.expand_w)
+               mode=args.mode, dist_mode=dist_mode, expand_w=args.expand_w, lam=args.lam)
     per = max((time.perf_counter() - t0) / probe, 1e-6)
     n = int(max(8, min(w.Q, seconds / per)))
     t0 = time.perf_counter()
     o = orc.search(d["queries"][:n], d["lo"][:n], d["hi"][:n], w.k, widths, eps=args.eps,
-                   mode=args.mode, dist_mode=dist_mode, expand_w=args.expand_w)
+                   mode=args.mode, dist_mode=dist_mode, expand_w=args.expand_w, lam=args.lam)
     dt = time.perf_counter() - t0
     return orc, o, n, dt
 
@@ -219,7 +221,7 @@ def reference_arm(args):
     probe = min(8, w.Q)
     t0 = time.perf_counter()
     orc.search(d["queries"][:probe], d["lo"][:probe], d["hi"][:probe], w.k, widths, eps=args.eps,
-               mode=args.mode, dist_mode=1, expand_w=args.expand_w)
+               mode=args.mode, dist_mode=1, expand_w=args.expand_w, lam=args.lam)
     per = max((time.perf_counter() - t0) / probe, 1e-6)
     n = int(max(4, min(w.Q, per_step / per)))
     times = []
@@ -227,7 +229,7 @@ def reference_arm(args):
         a = (s * n) % max(1, w.Q - n + 1)
         t0 = time.perf_counter()
         orc.search(d["queries"][a:a + n], d["lo"][a:a + n], d["hi"][a:a + n], w.k, widths,
-                   eps=args.eps, mode=args.mode, dist_mode=1, expand_w=args.expand_w)
+                   eps=args.eps, mode=args.mode, dist_mode=1, expand_w=args.expand_w, lam=args.lam)
         if s >= args.warmup:
             times.append(time.perf_counter() - t0)
     ms = 1e3 * float(np.mean(times))
@@ -247,7 +249,7 @@ def config_dict(w, widths, args):
     return {"workload": f"{w.name}: N={w.N} D={w.D} {w.vec_dtype} m={w.m} R={w.R} Q={w.Q} k={w.k} "
                         f"L0={w.L0} Lmax={w.Lmax}",
             "schedule": widths, "eps": args.eps, "mode": args.mode, "plus_k": args.plus_k,
-            "expand_w": args.expand_w,
+            "expand_w": args.expand_w, "lambda": "inf" if np.isinf(args.lam) else args.lam,
             "selectivity": f"{w.sel_kind} {w.sel_lo}-{w.sel_hi}", "seed": args.seed,
             "l2": "inputs larger than L2: records + graph are read by random access from a "
                   "working set far above 126 MB; no flush between steps"}
@@ -283,6 +285,7 @@ def main():
     ix.set_param("eps", args.eps)
     ix.set_param("plus_k", args.plus_k)
     ix.set_param("expand_w", args.expand_w)
+    ix.set_param("lam", args.lam)
     ix.set_param("table_kb", args.table_kb)
     ix.set_param("table_tags", args.table_tags)
     ix.set_param("max_warps_per_sm", args.max_warps)

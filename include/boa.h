@@ -65,6 +65,15 @@ enum {
                                points with the default 4 KB), else 16-bit tags, four to an
                                8-byte bucket; 16 = always the latter.  Never changes
                                results.                                                      */
+    BOA_PARAM_LAMBDA = 11,  /* weight lambda of the filter penalty in the score the search
+                               orders by, dist + lambda*phi ("Graph construction" paragraph;
+                               phi = number of violated predicates).  Default +infinity: any
+                               violated predicate outweighs any distance, keys order by
+                               (phi, d^2, id).  A finite value >= 0 orders by the score
+                               d^2 + lambda*phi (squared distance, one fp32 fused
+                               multiply-add), ties by id.  Answers are filter-valid either
+                               way; a finite lambda lets invalid nodes push valid ones out
+                               of the pool.                                                  */
     BOA_PARAM_EXPAND_W = 9  /* nodes expanded per iteration of Algorithm 2.  1 (default) is
                                the algorithm as printed ("each iteration expands one
                                node").  2 is an extension: the first two unexpanded beam

@@ -160,6 +160,7 @@ struct boa_index {
     // parameters
     double eps = 0.05, growth = 4.0, tau = 0.0;
     int mode = 0, plus_k = 0, cap_mult = 8, cap_add = 64, table_kb = 0, max_ctas = 0, expand_w = 1, table_tags = 0;
+    double lambda = INFINITY;          // weight of the filter penalty; infinity = lexicographic keys
     int n_sched = 0;
     int sched[BOA_MAX_PHASES] = {0};
     // scratch
@@ -600,6 +601,9 @@ int boa_set_param(boa_index* ix, int key, double v)
         case BOA_PARAM_TABLE_TAGS:
             if (v != 0.0 && v != 16.0) return BOA_EINVAL;
             ix->table_tags = (int)v; return BOA_OK;
+        case BOA_PARAM_LAMBDA:
+            if (!(v >= 0.0)) return BOA_EINVAL;
+            ix->lambda = v; return BOA_OK;
         case BOA_PARAM_EXPAND_W:
             if (v != 1.0 && v != 2.0) return BOA_EINVAL;
             ix->expand_w = (int)v; return BOA_OK;
@@ -663,6 +667,8 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
     b.hi = reinterpret_cast<const int32_t*>(hi);
     b.out_ids = out_ids; b.out_d2 = out_dists; b.Q = Q; b.k = k;
     b.tau_q = ix->tau * (double)Q;
+    b.fin = isinf(ix->lambda) ? 0 : 1;
+    b.lambda = b.fin ? (float)ix->lambda : 0.0f;
     if (ix->eps < 0.0) b.eps_mode = -1;
     else if (ix->eps >= 1.0) b.eps_mode = 1;
     else { b.eps_mode = 0; b.c_eps = (float)((1.0 - ix->eps) * (1.0 - ix->eps)); }

@@ -7,13 +7,14 @@
 // shared memory.  A pool entry is one 64-bit key
 //     [63:60] phi (violated predicates)  [59:29] fp32 bits of d^2  [28:1] id  [0] expanded
 // so that integer order of keys is the lexicographic order (phi, d^2, id): the
-// lambda -> infinity reading of the paper's score dist + lambda*phi.
+// lambda -> infinity reading of the paper's score dist + lambda*phi.  With a finite
+// lambda the key carries the score itself (layout at pack_key).
 //
 // Neighbour records (vector + attribute cells, one contiguous 32-byte-aligned row
 // each) are read with 16-byte read-only loads straight into registers: eight
 // rows per pass, 8 lanes per row, every lane issues all its loads of the pass (two
 // rows, up to four chunks each) before the first use, so a warp keeps 4 KB in flight
-// and an SM with 16 resident warps about 64 KB.  Two staged variants were measured
+// and an SM with 20 resident warps about 80 KB.  Two staged variants were measured
 // first and dropped: one cp.async.bulk (TMA) copy per row into shared memory needs a
 // uniform-datapath instruction sequence per row, and 16-byte cp.async copies spend
 // as long issuing as waiting; both were 40 % slower than register loads on the 1M x
@@ -105,6 +106,8 @@ struct SearchParams {
     float c_eps;              // (1-eps)^2 rounded once to fp32
     int eps_mode;             // 0: use c_eps; -1: never confident; 1: confident iff > k valid
     double tau_q;             // tau * Q: a phase runs only while |A| > tau*Q
+    int fin;                  // 1: keys order by the score d^2 + lambda*phi (finite lambda)
+    float lambda;
     // work list of this launch: positions [begin, end) of in_list (identity when null)
     const uint32_t* in_list;
     const uint32_t* in_begin_ptr;  // device values read at kernel start (null: use constants)
@@ -127,17 +130,30 @@ struct SearchParams {
 };
 
 // ---------------------------------------------------------------- helpers
-__device__ __forceinline__ uint64_t pack_key(uint32_t phi, float d2, uint32_t id)
+// Two key layouts.  Lexicographic (lambda -> infinity): phi on top, then the distance bits.
+// Finite lambda: the score bits on top, then the id; phi rides below the id, where it
+// cannot change the order of two different nodes.
+//     fin == false: [63:60] phi  [59:29] fp32 bits of d^2    [28:1] id            [0] expanded
+//     fin == true : [63:33] fp32 bits of d^2 + lambda*phi    [32:5] id  [4:1] phi [0] expanded
+__device__ __forceinline__ uint64_t pack_key(bool fin, uint32_t phi, float key, uint32_t id)
 {
-    return ((uint64_t)phi << 60) | ((uint64_t)(__float_as_uint(d2) & 0x7FFFFFFFu) << 29) |
-           ((uint64_t)id << 1);
+    const uint64_t bits = __float_as_uint(key) & 0x7FFFFFFFu;
+    return fin ? ((bits << 33) | ((uint64_t)id << 5) | ((uint64_t)phi << 1))
+               : (((uint64_t)phi << 60) | (bits << 29) | ((uint64_t)id << 1));
 }
-__device__ __forceinline__ uint32_t key_id(uint64_t k) { return (uint32_t)(k >> 1) & 0x0FFFFFFFu; }
-__device__ __forceinline__ float key_d2(uint64_t k)
+__device__ __forceinline__ uint32_t key_id(bool fin, uint64_t k)
 {
-    return __uint_as_float((uint32_t)(k >> 29) & 0x7FFFFFFFu);
+    return (uint32_t)(k >> (fin ? 5 : 1)) & 0x0FFFFFFFu;
 }
-__device__ __forceinline__ uint32_t key_phi(uint64_t k) { return (uint32_t)(k >> 60); }
+// d^2 in the lexicographic layout; the score in the other (equal to d^2 where phi == 0)
+__device__ __forceinline__ float key_d2(bool fin, uint64_t k)
+{
+    return __uint_as_float((uint32_t)(k >> (fin ? 33 : 29)) & 0x7FFFFFFFu);
+}
+__device__ __forceinline__ uint32_t key_phi(bool fin, uint64_t k)
+{
+    return fin ? ((uint32_t)(k >> 1) & 0xFu) : (uint32_t)(k >> 60);
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p)
 {
@@ -318,6 +334,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
     uint16_t* hash = reinterpret_cast<uint16_t*>(smem_raw + lay.hash_off);
     float4* qs = reinterpret_cast<float4*>(smem_raw + lay.q_off);
 
+    const bool fin = p.fin != 0;
     const uint32_t id_mask = (p.id_bits >= 32) ? 0xFFFFFFFFu : ((1u << p.id_bits) - 1u);
     const uint32_t low_mask = (1u << p.low_bits) - 1u;
 
@@ -394,7 +411,12 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             const unsigned bal = hi4 ? bal1 : bal0;
             const int jj = hi4 ? j1 : j0;
             if ((g & 3) == 0 && jj < cnt)
-                nk[jj] = pack_key(__popc((bal >> (8 * gi)) & 0xFFu), v, hi4 ? id1 : id0);
+            {
+                const uint32_t phi = __popc((bal >> (8 * gi)) & 0xFFu);
+                // finite lambda: one fused multiply-add gives the score the pool orders by
+                if (fin) nk[jj] = pack_key(true, phi, __fmaf_rn(p.lambda, (float)phi, v), hi4 ? id1 : id0);
+                else nk[jj] = pack_key(false, phi, v, hi4 ? id1 : id0);
+            }
         };
 
         // Scores cand[0..cnt) straight from global memory: eight rows per pass, every lane
@@ -576,7 +598,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             for (int i = lane; i < n; i += 32) {
                 const uint64_t e = src[i];
                 pool[i] = e;
-                hash_test_and_set(key_id(e));
+                hash_test_and_set(key_id(fin, e));
             }
             __syncwarp();
         } else {
@@ -601,10 +623,10 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             if (pos < 0) break;                                   // converged
             if (n_exp >= p.max_expand) { capped = true; break; }
             if (!have_row) {
-                load_row_ids(key_id(pool[pos]), nb, 0);
+                load_row_ids(key_id(fin, pool[pos]), nb, 0);
                 if (W > 1) {
                     pos2 = (n_exp + 1 < p.max_expand) ? first_unexpanded(pos + 1, n < p.L ? n : p.L) : -1;
-                    load_row_ids(pos2 >= 0 ? key_id(pool[pos2]) : kNoId, nb, RN);
+                    load_row_ids(pos2 >= 0 ? key_id(fin, pool[pos2]) : kNoId, nb, RN);
                 }
             }
             __syncwarp();
@@ -784,10 +806,10 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                     uint32_t next_id;
                     if (pos_old_new < 0 || rmin < pos_old_new) {
                         next_pos = rmin;                         // the smallest new key comes first
-                        next_id = key_id(first_new);
+                        next_id = key_id(fin, first_new);
                     } else {
                         next_pos = pos_old_new;
-                        next_id = key_id(pool[pos_old]);
+                        next_id = key_id(fin, pool[pos_old]);
                     }
                     if (next_pos >= lim_new) next_pos = -1;
                     pos = next_pos;
@@ -800,7 +822,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                     // two unexpanded old entries and the first two kept new keys
                     constexpr int kNone = 0x7fffffff;
                     const int a0 = pos_old_new >= 0 ? pos_old_new : kNone;
-                    const uint32_t a0id = pos_old >= 0 ? key_id(pool[pos_old]) : kNoId;
+                    const uint32_t a0id = pos_old >= 0 ? key_id(fin, pool[pos_old]) : kNoId;
                     int a1 = kNone;
                     uint32_t a1id = kNoId;
                     if (pos_old >= 0) {
@@ -811,11 +833,11 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                             for (int s = 0; s < RS; ++s)
                                 sh += __popc(__ballot_sync(0xffffffffu, keep[s] && rank_s[s] <= o2));
                             a1 = o2 + sh;
-                            a1id = key_id(pool[o2]);
+                            a1id = key_id(fin, pool[o2]);
                         }
                     }
                     const int b0 = rmin;
-                    const uint32_t b0id = key_id(first_new);
+                    const uint32_t b0id = key_id(fin, first_new);
                     int b1 = kNone;
                     uint32_t b1id = kNoId;
                     {
@@ -827,7 +849,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                             if (b1 == kNone && mk) {
                                 const int src = __ffs(mk) - 1;
                                 b1 = __shfl_sync(0xffffffffu, pos_new[s], src);
-                                b1id = key_id(__shfl_sync(0xffffffffu, x[s], src));
+                                b1id = key_id(fin, __shfl_sync(0xffffffffu, x[s], src));
                             }
                         }
                     }
@@ -906,23 +928,58 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             }
             BOA_T_MARK(9);
         }
-        // ---- result: the k nearest filter-valid entries (valid ones sort first)
+        // ---- result: the k nearest filter-valid entries; V = the valid ones among the first L
         const int lim = n < p.L ? n : p.L;
-        int nv_beam = 0;            // filter-valid entries among the first L
-        for (int b0 = 0; b0 < lim; b0 += 32) {
-            const int i = b0 + lane;
-            const bool ok = (i < lim) && (key_phi(pool[i]) == 0u);
-            nv_beam += __popc(__ballot_sync(0xffffffffu, ok));
-        }
-        for (int i = lane; i < p.k; i += 32) {
-            uint32_t id = kNoId;
-            float d2 = __int_as_float(0x7f800000);
-            if (i < n) {
-                const uint64_t e = pool[i];
-                if (key_phi(e) == 0u) { id = key_id(e); d2 = key_d2(e); }
+        int nv_beam = 0;            // |V|
+        float d2k = 0.0f, d2max = 0.0f;     // k-th and last distance of V
+        if (!fin) {
+            // valid entries sort first
+            for (int b0 = 0; b0 < lim; b0 += 32) {
+                const int i = b0 + lane;
+                const bool ok = (i < lim) && (key_phi(false, pool[i]) == 0u);
+                nv_beam += __popc(__ballot_sync(0xffffffffu, ok));
             }
-            p.out_ids[(size_t)qi * p.k + i] = id;
-            p.out_d2[(size_t)qi * p.k + i] = d2;
+            for (int i = lane; i < p.k; i += 32) {
+                uint32_t id = kNoId;
+                float d2 = __int_as_float(0x7f800000);
+                if (i < n) {
+                    const uint64_t e = pool[i];
+                    if (key_phi(false, e) == 0u) { id = key_id(false, e); d2 = key_d2(false, e); }
+                }
+                p.out_ids[(size_t)qi * p.k + i] = id;
+                p.out_d2[(size_t)qi * p.k + i] = d2;
+            }
+            if (nv_beam > p.k) {
+                d2k = key_d2(false, pool[p.k - 1]);
+                d2max = key_d2(false, pool[nv_beam - 1]);
+            }
+        } else {
+            // valid entries lie among invalid ones: one pass over the pool
+            int have = 0;           // valid entries met so far
+            for (int b0 = 0; b0 < n; b0 += 32) {
+                const int i = b0 + lane;
+                const uint64_t e = (i < n) ? pool[i] : 0ull;
+                const bool ok = (i < n) && (key_phi(true, e) == 0u);
+                const float d2 = key_d2(true, e);           // phi == 0: the score is d^2
+                const unsigned bal = __ballot_sync(0xffffffffu, ok);
+                const int r = have + __popc(bal & lt_mask);
+                if (ok && r < p.k) {
+                    p.out_ids[(size_t)qi * p.k + r] = key_id(true, e);
+                    p.out_d2[(size_t)qi * p.k + r] = d2;
+                }
+                const unsigned balb = __ballot_sync(0xffffffffu, ok && i < lim);
+                const int rb = nv_beam + __popc(balb & lt_mask);
+                const unsigned kth = __ballot_sync(0xffffffffu, ok && i < lim && rb == p.k - 1);
+                if (kth) d2k = __shfl_sync(0xffffffffu, d2, __ffs(kth) - 1);
+                if (balb) d2max = __shfl_sync(0xffffffffu, d2, 31 - __clz(balb));
+                nv_beam += __popc(balb);
+                have += __popc(bal);
+            }
+            for (int i = lane; i < p.k; i += 32)
+                if (i >= have) {
+                    p.out_ids[(size_t)qi * p.k + i] = kNoId;
+                    p.out_d2[(size_t)qi * p.k + i] = __int_as_float(0x7f800000);
+                }
         }
 
         // ---- confidence test (Eq. 3) and compaction of the uncertain
@@ -930,11 +987,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
         if (nv_beam > p.k) {
             if (p.eps_mode < 0) uncertain = true;
             else if (p.eps_mode > 0) uncertain = false;
-            else {
-                const float d2k = key_d2(pool[p.k - 1]);
-                const float d2max = key_d2(pool[nv_beam - 1]);
-                uncertain = !(d2k >= p.c_eps * d2max);
-            }
+            else uncertain = !(d2k >= p.c_eps * d2max);
         }
         if (lane == 0) {
             p.final_L[qi] = p.L;

@@ -95,6 +95,54 @@ def test_stride_line_hand_trace_width_2_on_gpu():
     gpu.close()
 
 
+@pytest.mark.parametrize("name,lam", [("c2", 2000.0), ("c2", 0.0), ("c3", 0.05), ("c4", 30000.0),
+                                      ("c5", 0.3)])
+@pytest.mark.parametrize("mode", ["restart", "resume"])
+def test_finite_lambda_matches_oracle_bit_for_bit(name, lam, mode):
+    """Keys ordered by the score d2 + lambda*phi (the paper's stated form): same score bits
+    (one fp32 fused multiply-add on both sides), same trajectories, same answers."""
+    w, d, orc, gpu, g = _get(name)
+    widths = default_widths(w.L0, min(w.Lmax, 256))
+    eps = {"c4": 0.2}.get(name, 0.05)
+    o = orc.search(d["queries"], d["lo"], d["hi"], w.k, widths, eps=eps, mode=mode, dist_mode=1, lam=lam)
+    r = gpu_search(gpu, g, w.k, widths, eps=eps, mode=mode, lam=lam)
+    assert_bit_parity(o, r, f"{name}/{mode}/lambda={lam}")
+    o_inf = orc.search(d["queries"], d["lo"], d["hi"], w.k, widths, eps=eps, mode=mode, dist_mode=1)
+    assert (o_inf["n_scored"] != o["n_scored"]).any()        # the order does change the search
+    # answers stay filter-valid and sorted
+    for i in range(0, len(r["ids"]), 17):
+        ids = r["ids"][i]
+        n = int((ids != SENTINEL).sum())
+        assert (ids[n:] == SENTINEL).all() and (np.diff(r["d2"][i][:n]) >= 0).all()
+        a = d["attrs"][ids[:n].astype(np.int64)]
+        for j, t in enumerate(d["attr_types"]):
+            col = a[:, j].view(np.float32) if t == 1 else a[:, j]
+            l = d["lo"][i, j:j + 1].view(np.float32)[0] if t == 1 else d["lo"][i, j]
+            h = d["hi"][i, j:j + 1].view(np.float32)[0] if t == 1 else d["hi"][i, j]
+            assert ((col >= l) & (col <= h)).all()
+
+
+def test_finite_lambda_ring_hand_traces_width_2_and_boa_plus():
+    x = np.zeros((8, 4), dtype=np.float32)
+    x[:, 0] = np.arange(8)
+    d = dict(vectors=x, attrs=(np.arange(8) % 2).astype(np.int32)[:, None],
+             attr_types=np.zeros(1, np.int32),
+             graph=np.stack([(np.arange(8) - 1) % 8, (np.arange(8) + 1) % 8], 1).astype(np.uint32),
+             queries=np.array([[5.2, 0, 0, 0]], dtype=np.float32),
+             lo=np.array([[1]], np.int32), hi=np.array([[1]], np.int32))
+    orc, gpu, g = make_pair(d, entry=0)
+    r = gpu_search(gpu, g, 2, [3], lam=2.0)              # tests/golden/ring_trace_finite_lambda.txt
+    assert r["ids"][0].tolist() == [5, 7] and r["n_expand"][0] == 4 and r["n_scored"][0] == 5
+    r = gpu_search(gpu, g, 2, [3], lam=0.5)
+    assert r["ids"][0].tolist() == [5, SENTINEL] and r["n_expand"][0] == 5 and r["n_scored"][0] == 6
+    gpu.close()
+    w, d, orc, gpu, g = _get("c2")
+    o = orc.search(d["queries"], d["lo"], d["hi"], w.k, [16, 128], mode="resume", dist_mode=1, lam=500.0,
+                   expand_w=2)
+    r = gpu_search(gpu, g, w.k, [16, 128], mode="resume", plus_k=3, lam=500.0, expand_w=2)
+    assert_bit_parity(o, r, "BOA+/W=2/lambda=500")
+
+
 @pytest.mark.parametrize("name", ["c2", "c4"])
 def test_integer_data_matches_double_accumulation_too(name):
     """Every partial sum of integer-valued rows is below 2^24, so the fp32 order cannot

@@ -62,6 +62,10 @@ def test_shape_variants_match_oracle(case):
         o = orc.search(d["queries"], d["lo"], d["hi"], k, widths, mode=mode, dist_mode=1, expand_w=2)
         r = gpu_search(gpu, g, k, widths, mode=mode, expand_w=2)
         assert_bit_parity(o, r, f"{name}/{mode}/W=2")
+        lam = 40.0 if dtype == "f32" else 30000.0
+        o = orc.search(d["queries"], d["lo"], d["hi"], k, widths, mode=mode, dist_mode=1, lam=lam)
+        r = gpu_search(gpu, g, k, widths, mode=mode, lam=lam)
+        assert_bit_parity(o, r, f"{name}/{mode}/lambda={lam}")
     assert (r["ids"] != SENTINEL).any()
     gpu.close()
 
