@@ -28,7 +28,9 @@ thread_local int g_last_cuda = 0;
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // ------------------------------------------------------------------ index build kernels
-// Record i = [vector bytes | m attribute cells | zero padding], rec_stride bytes.
+// Record i = [vector bytes | zero padding], rec_stride bytes.  The attribute cells live in
+// an array of their own ([N][m], a few MB that stay in L2), so a scored row costs whole
+// 64-byte DRAM bursts of vector data only.
 __global__ void build_records_kernel(const uint8_t* __restrict__ vec, const int32_t* __restrict__ attrs,
                                      uint8_t* __restrict__ rec, int64_t N, int vec_bytes, int m,
                                      int stride)
@@ -151,7 +153,8 @@ __global__ void copy_word_kernel(uint32_t* dst, const uint32_t* src) { *dst = *s
 struct boa_index {
     int64_t N = 0;
     int D = 0, m = 0, R = 0, vec_dtype = 0;
-    int rec_stride = 0, nchunks = 0, attr_off = 0;
+    int rec_stride = 0, nchunks = 0;
+    uint32_t* attr_cells = nullptr;    // [N][m] attribute cells
     uint32_t attr_float_mask = 0;
     int64_t entry = 0;
     uint8_t* rec = nullptr;
@@ -478,14 +481,16 @@ int boa_index_create(boa_index** out, const void* vectors, int vec_dtype, int64_
     ix->N = N; ix->D = D; ix->m = m; ix->R = R; ix->vec_dtype = vec_dtype;
     const int vec_bytes = vec_dtype == BOA_U8 ? D : 4 * D;
     ix->nchunks = vec_bytes / 16;
-    ix->attr_off = vec_bytes;
-    ix->rec_stride = (vec_bytes + 4 * m + 31) & ~31;
+    ix->rec_stride = (vec_bytes + 31) & ~31;
     for (int j = 0; j < m; ++j)
         if (attr_types[j] == BOA_ATTR_F32) ix->attr_float_mask |= 1u << j;
     BOA_TRY(cudaGetDevice(&ix->device));
     BOA_TRY(cudaDeviceGetAttribute(&ix->num_sms, cudaDevAttrMultiProcessorCount, ix->device));
     BOA_TRY(cudaMalloc(&ix->rec, (size_t)N * ix->rec_stride));
     BOA_TRY(cudaMalloc(&ix->graph, (size_t)N * R * sizeof(uint32_t)));
+    BOA_TRY(cudaMalloc(&ix->attr_cells, (size_t)N * m * sizeof(uint32_t)));
+    BOA_TRY(cudaMemcpyAsync(ix->attr_cells, attrs, (size_t)N * m * sizeof(uint32_t),
+                            cudaMemcpyDeviceToDevice, st));
     BOA_TRY(cudaStreamCreateWithFlags(&ix->side, cudaStreamNonBlocking));
     BOA_TRY(cudaEventCreateWithFlags(&ix->ev_fork, cudaEventDisableTiming));
     BOA_TRY(cudaEventCreateWithFlags(&ix->ev_join, cudaEventDisableTiming));
@@ -493,7 +498,7 @@ int boa_index_create(boa_index** out, const void* vectors, int vec_dtype, int64_
     const int blocks = ix->num_sms * 8;
     build_records_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const uint8_t*>(vectors),
                                                  reinterpret_cast<const int32_t*>(attrs), ix->rec, N,
-                                                 vec_bytes, m, ix->rec_stride);
+                                                 vec_bytes, 0, ix->rec_stride);
     BOA_TRY(cudaGetLastError());
     int* d_bad = nullptr;
     BOA_TRY(cudaMalloc(&d_bad, sizeof(int)));
@@ -557,7 +562,7 @@ int boa_index_create(boa_index** out, const void* vectors, int vec_dtype, int64_
 int boa_index_destroy(boa_index* ix)
 {
     if (!ix) return BOA_OK;
-    cudaFree(ix->rec); cudaFree(ix->graph); cudaFree(ix->lists); cudaFree(ix->counters);
+    cudaFree(ix->rec); cudaFree(ix->attr_cells); cudaFree(ix->graph); cudaFree(ix->lists); cudaFree(ix->counters);
     cudaFree(ix->stats); cudaFree(ix->spill); cudaFree(ix->spill_size);
     if (ix->side) cudaStreamDestroy(ix->side);
     if (ix->ev_fork) cudaEventDestroy(ix->ev_fork);
@@ -659,7 +664,7 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
     memset(&b, 0, sizeof(b));
     b.rec = ix->rec; b.graph = ix->graph; b.N = ix->N; b.D = ix->D; b.m = ix->m; b.R = ix->R;
     b.rec_stride = ix->rec_stride; b.nchunks = ix->nchunks;
-    b.attr_off = ix->attr_off; b.status = ix->counters + kCntStatus;
+    b.attrs = ix->attr_cells; b.status = ix->counters + kCntStatus;
     b.timers = reinterpret_cast<unsigned long long*>(ix->counters + kCntWords);
     b.attr_float_mask = ix->attr_float_mask; b.entry = (uint32_t)ix->entry;
     b.queries = queries;

@@ -10,8 +10,8 @@
 // lambda -> infinity reading of the paper's score dist + lambda*phi.  With a finite
 // lambda the key carries the score itself (layout at pack_key).
 //
-// Neighbour records (vector + attribute cells, one contiguous 32-byte-aligned row
-// each) are read with 16-byte read-only loads straight into registers: eight
+// Neighbour records (the vector, one 32-byte-aligned row each; the attribute cells sit in a
+// compact array of their own that stays in L2) are read with 16-byte read-only loads straight into registers: eight
 // rows per pass, 8 lanes per row, every lane issues all its loads of the pass (two
 // rows, up to four chunks each) before the first use, so a warp keeps 4 KB in flight
 // and an SM with 20 resident warps about 80 KB.  Two staged variants were measured
@@ -73,13 +73,13 @@ enum : uint32_t { kStatusCopyTimeout = 1u };   // reserved: no wait in the kerne
 
 struct SearchParams {
     // index
-    const uint8_t* rec;       // [N] records: vector, then m attribute cells, padded to rec_stride
+    const uint8_t* rec;       // [N] records: the vector, padded to rec_stride
+    const uint32_t* attrs;    // [N][m] attribute cells
     const uint32_t* graph;    // [N][R]
     int64_t N;
     int D, m, R;
     int rec_stride;           // bytes, multiple of 32
     int nchunks;              // 16-byte chunks of one vector
-    int attr_off;             // byte offset of the attribute cells inside a record
     uint32_t attr_float_mask; // bit j set: column j is float
     uint32_t entry;
     // batch
@@ -450,8 +450,8 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                             x1[i] = ldg_stream128(row1 + 16 * c, act1 && c < p.nchunks);
                         }
                     }
-                    av0 = ldg_stream32(row0 + p.attr_off + 4 * ga, act0 && g < p.m);
-                    av1 = ldg_stream32(row1 + p.attr_off + 4 * ga, act1 && g < p.m);
+                    av0 = ldg_stream32(p.attrs + (size_t)id0 * p.m + ga, act0 && g < p.m);
+                    av1 = ldg_stream32(p.attrs + (size_t)id1 * p.m + ga, act1 && g < p.m);
                 };
                 issue_pass(0);
 #pragma unroll 1
@@ -494,8 +494,8 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                     const uint8_t* row0 = p.rec + (size_t)id0 * p.rec_stride;
                     const uint8_t* row1 = p.rec + (size_t)id1 * p.rec_stride;
                     float a0 = 0.0f, a1 = 0.0f;
-                    const uint32_t av0 = ldg_stream32(row0 + p.attr_off + 4 * ga, act0 && g < p.m);
-                    const uint32_t av1 = ldg_stream32(row1 + p.attr_off + 4 * ga, act1 && g < p.m);
+                    const uint32_t av0 = ldg_stream32(p.attrs + (size_t)id0 * p.m + ga, act0 && g < p.m);
+                    const uint32_t av1 = ldg_stream32(p.attrs + (size_t)id1 * p.m + ga, act1 && g < p.m);
                     // long rows: four chunks of each row in flight per lane at a time
                     for (int c0 = g; c0 < p.nchunks; c0 += 32) {
                         uint4 x0[4], x1[4];

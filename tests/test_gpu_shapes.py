@@ -91,7 +91,8 @@ def test_degenerate_sizes():
 
 def test_many_random_small_cases():
     """Thirty seeded random shapes (dimension, element type, attribute count and types,
-    degree, k, widths, ε, mode, BOA+), each against the oracle bit for bit."""
+    degree, k, widths, ε, mode, BOA+, expansion width, λ, table format), each against the oracle
+    bit for bit."""
     rng = np.random.default_rng(2024)
     for case in range(30):
         dtype = "u8" if rng.random() < 0.4 else "f32"
@@ -112,9 +113,10 @@ def test_many_random_small_cases():
         for ew in (1, 2):
             if ew == 2:
                 gpu.set_param("table_kb", int(rng.choice([0, 1])))   # a 1 KB table forgets at once
+            lam = float(rng.choice([np.inf, np.inf, 0.0, 3.0, 20000.0]))
             o = orc.search(d["queries"], d["lo"], d["hi"], k, widths, eps=eps, mode=mode, dist_mode=1,
-                           expand_w=ew)
-            r = gpu_search(gpu, g, k, widths, mode=mode, eps=eps, plus_k=plus_k, expand_w=ew)
+                           expand_w=ew, lam=lam)
+            r = gpu_search(gpu, g, k, widths, mode=mode, eps=eps, plus_k=plus_k, expand_w=ew, lam=lam)
             assert_bit_parity(o, r, f"case {case}: {dtype} D={D} m={m} R={R} N={N} k={k} {widths} "
-                                    f"{mode} W={ew}")
+                                    f"{mode} W={ew} lambda={lam}")
         gpu.close()
