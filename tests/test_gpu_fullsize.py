@@ -78,3 +78,40 @@ def test_full_size_boa_plus_and_restart_agree_with_their_definitions(full):
     o = orc.search(d["queries"][sample], d["lo"][sample], d["hi"][sample], w.k, [16, 64, 256], eps=0.05,
                    mode="restart", dist_mode=1)
     assert (o["ids"] == r["ids"]).all() and (o["n_expand"] == r["n_expand"]).all()
+
+
+def test_full_size_float_workload_c3():
+    """The 1M x 96-d unit-norm float workload at full size: sampled queries bit for bit
+    against the oracle's fixed-order fp32 distances, within the stated tolerance of its
+    double-precision distances, and the recall bar."""
+    from boa_synth import C3
+    w = C3
+    d = make_workload(w, seed=0)
+    orc, gpu, g = make_pair(d)
+    widths, eps = [16, 512], 0.03
+    r = gpu_search(gpu, g, w.k, widths, mode="resume", eps=eps)
+    assert gpu.device_status() == 0
+    sample = np.random.default_rng(6).choice(w.Q, size=96, replace=False)
+    o = orc.search(d["queries"][sample], d["lo"][sample], d["hi"][sample], w.k, widths, eps=eps,
+                   mode="resume", dist_mode=1)
+    assert (o["ids"] == r["ids"][sample]).all()
+    assert (o["d2"].view(np.uint32) == r["d2"][sample].view(np.uint32)).all()
+    assert (o["final_L"] == r["final_L"][sample]).all() and (o["n_expand"] == r["n_expand"][sample]).all()
+    # double accumulation: same ids except at near-ties below 1e-5 relative, distances within 1e-5
+    o64 = orc.search(d["queries"][sample], d["lo"][sample], d["hi"][sample], w.k, widths, eps=eps,
+                     mode="resume", dist_mode=0)
+    same_path = (o64["final_L"] == r["final_L"][sample]) & (o64["n_expand"] == r["n_expand"][sample])
+    assert same_path.mean() > 0.9
+    for t in np.nonzero(same_path)[0]:
+        gi, oi = r["ids"][sample[t]], o64["ids"][t]
+        gd, od = r["d2"][sample[t]], o64["d2"][t]
+        fin = np.isfinite(od)
+        assert (np.isfinite(gd) == fin).all()
+        np.testing.assert_allclose(gd[fin], od[fin], rtol=1e-5)
+        for c in np.nonzero(gi != oi)[0]:                      # a swap is allowed only at a near-tie
+            assert abs(float(gd[c]) - float(od[c])) <= 1e-5 * max(float(od[c]), 1e-30)
+    gt_ids, gt_d2, gt_nv = filtered_topk(g["vectors"], g["attrs"], d["attr_types"], g["queries"],
+                                         g["lo"], g["hi"], w.k)
+    rec = recall_against(r["ids"], r["d2"], gt_d2.cpu().numpy(), gt_nv.cpu().numpy(), w.k)
+    assert np.nanmean(rec) >= 0.95
+    gpu.close()
