@@ -49,6 +49,13 @@ namespace boa {
 #ifndef BOA_MIN_CTAS
 #define BOA_MIN_CTAS 20
 #endif
+// Rows per 8-lane group and scoring pass for rows of one / two 16-byte chunks per lane.
+#ifndef BOA_SHORT_RPG1
+#define BOA_SHORT_RPG1 4
+#endif
+#ifndef BOA_SHORT_RPG2
+#define BOA_SHORT_RPG2 4
+#endif
 
 constexpr uint32_t kNoId = 0xFFFFFFFFu;
 constexpr int kThreads = 32;           // one warp per CTA
@@ -427,7 +434,70 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
         auto score = [&](int cnt) {
             BOA_T_MARK(3);
             const int ga = (g < p.m) ? g : 0;
-            if (CPL > 0) {
+            if (CPL == 1 || CPL == 2) {
+                // short rows: RPG rows per 8-lane group and pass (16 or 32 rows a pass), so that
+                // a row list of 40 costs two or three dependent round trips instead of six
+                constexpr int NC = (CPL > 0 ? CPL : 1);
+                constexpr int RPG = (CPL == 1) ? BOA_SHORT_RPG1 : BOA_SHORT_RPG2;
+                constexpr int RPP = 4 * RPG;
+                uint4 x[RPG][NC];
+                uint32_t av[RPG], id[RPG];
+                auto issue_pass = [&](int r0) {
+#pragma unroll
+                    for (int t = 0; t < RPG; ++t) {
+                        const int j = r0 + gi + 4 * t;
+                        const bool act = j < cnt;
+                        id[t] = cand[act ? j : 0];
+                        const uint8_t* row = p.rec + (size_t)id[t] * p.rec_stride;
+                        if (EXACT) {
+                            ldg_chunks<NC>(x[t], row + 16 * g, act);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < NC; ++i) {
+                                const int c = g + 8 * i;
+                                x[t][i] = ldg_stream128(row + 16 * c, act && c < p.nchunks);
+                            }
+                        }
+                        av[t] = ldg_stream32(p.attrs + (size_t)id[t] * p.m + ga, act && g < p.m);
+                    }
+                };
+                issue_pass(0);
+#pragma unroll 1
+                for (int r0 = 0; r0 < cnt; r0 += RPP) {
+                    BOA_T_MARK(4);
+                    BOA_SCHED_FENCE();        // every load of the pass is issued before its first use
+                    float a[RPG];
+                    uint32_t c_av[RPG], c_id[RPG];
+#pragma unroll
+                    for (int t = 0; t < RPG; ++t) {
+                        a[t] = 0.0f;
+#pragma unroll
+                        for (int i = 0; i < NC; ++i) {
+                            if (!EXACT && g + 8 * i >= p.nchunks) continue;
+                            if (VT == 0) {
+                                a[t] = sq_acc4u(a[t], x[t][i], qreg[i]);
+                            } else {
+                                a[t] = sq_acc_bytes(a[t], x[t][i].x, qreg[4 * i + 0]);
+                                a[t] = sq_acc_bytes(a[t], x[t][i].y, qreg[4 * i + 1]);
+                                a[t] = sq_acc_bytes(a[t], x[t][i].z, qreg[4 * i + 2]);
+                                a[t] = sq_acc_bytes(a[t], x[t][i].w, qreg[4 * i + 3]);
+                            }
+                        }
+                        c_av[t] = av[t];
+                        c_id[t] = id[t];
+                    }
+                    BOA_SCHED_FENCE();
+                    if (r0 + RPP < cnt) issue_pass(r0 + RPP);
+                    BOA_SCHED_FENCE();
+#pragma unroll
+                    for (int u = 0; u < RPG; u += 2) {
+                        const int ja = r0 + gi + 4 * u, jb = r0 + gi + 4 * (u + 1);
+                        finish_pass(cnt, a[u], a[u + 1], c_av[u], c_av[u + 1], c_id[u], c_id[u + 1], ja, jb,
+                                    ja < cnt, jb < cnt);
+                    }
+                    BOA_T_MARK(6);
+                }
+            } else if (CPL > 0) {
                 uint4 x0[CPL > 0 ? CPL : 1], x1[CPL > 0 ? CPL : 1];
                 uint32_t av0, av1, id0, id1;
                 bool act0, act1;
