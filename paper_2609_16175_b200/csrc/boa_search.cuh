@@ -248,13 +248,17 @@ __device__ __forceinline__ float sq_acc4u(float acc, uint4 x, float4 q)
     return sq_acc4(acc, make_float4(__uint_as_float(x.x), __uint_as_float(x.y), __uint_as_float(x.z),
                                     __uint_as_float(x.w)), q);
 }
+// Four bytes of a uint8 row against four query values.  A byte b becomes the float b exactly
+// by a byte permute into the mantissa of 2^23 and one subtraction: full-rate instructions
+// instead of an integer-to-float conversion per element.
 __device__ __forceinline__ float sq_acc_bytes(float acc, uint32_t w, float4 q)
 {
+    const float magic = 8388608.0f;                     // 2^23 = 0x4B000000
     float d;
-    d = (float)(w & 0xFFu) - q.x;         acc = fmaf(d, d, acc);
-    d = (float)((w >> 8) & 0xFFu) - q.y;  acc = fmaf(d, d, acc);
-    d = (float)((w >> 16) & 0xFFu) - q.z; acc = fmaf(d, d, acc);
-    d = (float)(w >> 24) - q.w;           acc = fmaf(d, d, acc);
+    d = (__uint_as_float(__byte_perm(w, 0x4B000000u, 0x7440)) - magic) - q.x; acc = fmaf(d, d, acc);
+    d = (__uint_as_float(__byte_perm(w, 0x4B000000u, 0x7441)) - magic) - q.y; acc = fmaf(d, d, acc);
+    d = (__uint_as_float(__byte_perm(w, 0x4B000000u, 0x7442)) - magic) - q.z; acc = fmaf(d, d, acc);
+    d = (__uint_as_float(__byte_perm(w, 0x4B000000u, 0x7443)) - magic) - q.w; acc = fmaf(d, d, acc);
     return acc;
 }
 
