@@ -747,18 +747,34 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             }
             if (live > 0) {
                 // sort the survivors: by counting for a handful, bitonic otherwise
-                if (RS == 1 && live <= 8) {
-                    const unsigned m0 = __ballot_sync(0xffffffffu, x[0] != kKeyMax);
-                    int r = 0;
-                    for (unsigned mm = m0; mm; mm &= mm - 1) {
-                        const uint64_t y = __shfl_sync(0xffffffffu, x[0], __ffs(mm) - 1);
-                        r += (y < x[0]) ? 1 : 0;
+                if (live <= 8) {
+                    // every live key counts the live keys before it (equal keys, which two rows
+                    // of one iteration can produce, order by where they sit), then moves there
+                    int r[RS];
+#pragma unroll
+                    for (int s = 0; s < RS; ++s) r[s] = 0;
+#pragma unroll
+                    for (int s2 = 0; s2 < RS; ++s2) {
+                        const unsigned m2 = __ballot_sync(0xffffffffu, x[s2] != kKeyMax);
+                        for (unsigned mm = m2; mm; mm &= mm - 1) {
+                            const int src = __ffs(mm) - 1;
+                            const uint64_t y = __shfl_sync(0xffffffffu, x[s2], src);
+#pragma unroll
+                            for (int s = 0; s < RS; ++s) {
+                                const bool before = (RS == 1) ? (y < x[s])
+                                    : (y < x[s] || (y == x[s] && src + 32 * s2 < lane + 32 * s));
+                                r[s] += before ? 1 : 0;
+                            }
+                        }
                     }
                     __syncwarp();
-                    if (x[0] != kKeyMax) nk[r] = x[0];
+#pragma unroll
+                    for (int s = 0; s < RS; ++s)
+                        if (x[s] != kKeyMax) nk[r[s]] = x[s];
                     __syncwarp();
-                    x[0] = (lane < live) ? nk[lane] : kKeyMax;
-                } else {   // also for a single key: it has to end up in lane 0
+#pragma unroll
+                    for (int s = 0; s < RS; ++s) x[s] = (s == 0 && lane < live) ? nk[lane] : kKeyMax;
+                } else {
                     sort_keys<RS>(x, lane);
                 }
                 BOA_T_MARK(7);
