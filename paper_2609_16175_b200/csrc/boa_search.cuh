@@ -711,6 +711,18 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             cur = ((W > 1 && pos2 >= 0) ? pos2 : pos) + 1;
             n_exp += (W > 1 && pos2 >= 0) ? 2 : 1;
             have_row = false;
+            // The probable next node is the next unexpanded entry of the pool as it is now (it
+            // is, unless a key scored in this iteration ranks before it): its adjacency row is
+            // requested here, a whole scoring pass ahead of its use.  Only for one node per
+            // iteration and R <= 32: with longer rows the requests wasted on wrong guesses
+            // cost more than the hidden latency saves.
+            constexpr bool PRED = (W == 1 && RN == 1);
+            int pred_pos = -1;
+            uint32_t nbp[RS];
+            if (PRED) {
+                pred_pos = first_unexpanded(cur, n < p.L ? n : p.L);
+                load_row_ids(pred_pos >= 0 ? key_id(fin, pool[pred_pos]) : kNoId, nbp, 0);
+            }
             BOA_T_MARK(1);
 
             // drop ids scored before, compact the rest
@@ -861,7 +873,14 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             }
             if (kept == 0) {
                 // pool unchanged: the next node is simply the next unexpanded entry
-                pos = first_unexpanded(cur, n < p.L ? n : p.L);
+                if (PRED) {
+                    pos = pred_pos;
+#pragma unroll
+                    for (int s = 0; s < RS; ++s) nb[s] = nbp[s];
+                    have_row = pos >= 0;
+                } else {
+                    pos = first_unexpanded(cur, n < p.L ? n : p.L);
+                }
                 continue;
             }
             // smallest rank among the kept keys = rank of the first kept key; and that key
@@ -880,7 +899,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             // position, and start loading that node's adjacency row before the merge.
             {
                 const int lim_old = n < p.L ? n : p.L;
-                const int pos_old = first_unexpanded(cur, lim_old);
+                const int pos_old = PRED ? pred_pos : first_unexpanded(cur, lim_old);
                 int pos_old_new = -1;
                 if (pos_old >= 0) {
                     int sh = 0;                       // kept keys ranked at or before it
@@ -893,18 +912,18 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                 const int lim_new = n_new < p.L ? n_new : p.L;
                 if (W == 1) {
                     int next_pos;
-                    uint32_t next_id;
-                    if (pos_old_new < 0 || rmin < pos_old_new) {
-                        next_pos = rmin;                         // the smallest new key comes first
-                        next_id = key_id(fin, first_new);
-                    } else {
-                        next_pos = pos_old_new;
-                        next_id = key_id(fin, pool[pos_old]);
-                    }
+                    const bool new_first = pos_old_new < 0 || rmin < pos_old_new;
+                    if (new_first) next_pos = rmin;              // the smallest new key comes first
+                    else next_pos = pos_old_new;
                     if (next_pos >= lim_new) next_pos = -1;
                     pos = next_pos;
                     if (pos >= 0 && n_exp < p.max_expand) {
-                        load_row_ids(next_id, nb, 0);
+                        if (new_first || !PRED) {
+                            load_row_ids(key_id(fin, new_first ? first_new : pool[pos_old]), nb, 0);
+                        } else {
+#pragma unroll
+                            for (int s = 0; s < RS; ++s) nb[s] = nbp[s];     // requested a pass ago
+                        }
                         have_row = true;
                     }
                 } else {
