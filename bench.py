@@ -34,9 +34,9 @@ UNIT = "queries/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the search kernel per scored neighbour
 # record, from the full-size ncu capture summarised in
-# profiles/boa_search_kernel_c2_dram_traffic.md (38.22 GB for 91.20 M records).  It holds
+# profiles/boa_search_kernel_c2_dram_traffic.md (38.24 GB for 91.20 M records).  It holds
 # for the default workload and table size only.
-NCU_DRAM_BYTES_PER_SCORED = {"c2": 419.1}
+NCU_DRAM_BYTES_PER_SCORED = {"c2": 419.3}
 
 
 def parse_args():
