@@ -14,7 +14,7 @@
  *   orc_beam_*         filter-aware beam search at one beamwidth (Algorithm 2),
  *                      with exact L2 distances instead of PQ look-ups
  *   orc_uncertain      confidence test gamma(D_i) <= eps (Eq. 3)
- *   orc_boa_search     multi-phase driver (Algorithm 1)
+ *   orc_boa_search_wl  multi-phase driver (Algorithm 1)
  *
  * Readings of points the paper leaves open (each is listed in the design notes):
  *   - the score dist + lambda*phi is taken in its lambda -> infinity limit by default:
@@ -345,13 +345,6 @@ void orc_beam_run_w(orc_state *st, int L, const float *q, const int32_t *lo, con
     }
 }
 
-/* Algorithm 2 as printed: one node per iteration */
-void orc_beam_run(orc_state *st, int L, const float *q, const int32_t *lo, const int32_t *hi,
-                  int dist_mode, int64_t max_expand)
-{
-    orc_beam_run_w(st, L, q, lo, hi, dist_mode, max_expand, 1);
-}
-
 /* K_i <- the k nearest filter-valid pool entries; returns how many there are */
 int orc_beam_result(const orc_state *st, int k, uint32_t *out_ids, float *out_d2)
 {
@@ -498,32 +491,4 @@ void orc_boa_search_wl(const orc_index *ix, const float *queries, int64_t Q,
     free(saved);
     free(active);
     orc_state_free(st);
-}
-
-/* lexicographic order (lambda -> infinity), any expansion width */
-void orc_boa_search_w(const orc_index *ix, const float *queries, int64_t Q,
-                      const int32_t *lo, const int32_t *hi, int k,
-                      const int32_t *widths, int n_widths, double eps, double tau,
-                      int mode, int dist_mode, int cap_mult, int cap_add, int W,
-                      uint32_t *out_ids, float *out_d2,
-                      int32_t *final_L, int32_t *n_expand, int32_t *n_scored, int32_t *flags,
-                      int64_t *phase_active)
-{
-    orc_boa_search_wl(ix, queries, Q, lo, hi, k, widths, n_widths, eps, tau, mode, dist_mode,
-                      cap_mult, cap_add, W, INFINITY, out_ids, out_d2, final_L, n_expand, n_scored,
-                      flags, phase_active);
-}
-
-/* the paper's setting: expansion width 1 */
-void orc_boa_search(const orc_index *ix, const float *queries, int64_t Q,
-                    const int32_t *lo, const int32_t *hi, int k,
-                    const int32_t *widths, int n_widths, double eps, double tau,
-                    int mode, int dist_mode, int cap_mult, int cap_add,
-                    uint32_t *out_ids, float *out_d2,
-                    int32_t *final_L, int32_t *n_expand, int32_t *n_scored, int32_t *flags,
-                    int64_t *phase_active)
-{
-    orc_boa_search_w(ix, queries, Q, lo, hi, k, widths, n_widths, eps, tau, mode, dist_mode,
-                     cap_mult, cap_add, 1, out_ids, out_d2, final_L, n_expand, n_scored, flags,
-                     phase_active);
 }

@@ -39,7 +39,6 @@ def lib():
         L.orc_state_free.argtypes = [vp]
         L.orc_state_set_lambda.argtypes = [vp, C.c_float]
         L.orc_beam_init.argtypes = [vp, i32, vp, vp, vp, i32]
-        L.orc_beam_run.argtypes = [vp, i32, vp, vp, vp, i32, i64]
         L.orc_beam_run_w.argtypes = [vp, i32, vp, vp, vp, i32, i64, i32]
         L.orc_beam_result.restype = i32
         L.orc_beam_result.argtypes = [vp, i32, vp, vp]
@@ -54,10 +53,6 @@ def lib():
         L.orc_state_pool.argtypes = [vp, vp, vp, vp, vp]
         L.orc_uncertain.restype = i32
         L.orc_uncertain.argtypes = [vp, i32, i32, dbl]
-        L.orc_boa_search.argtypes = [vp, vp, i64, vp, vp, i32, vp, i32, dbl, dbl, i32, i32,
-                                     i32, i32, vp, vp, vp, vp, vp, vp, vp]
-        L.orc_boa_search_w.argtypes = [vp, vp, i64, vp, vp, i32, vp, i32, dbl, dbl, i32, i32,
-                                       i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         L.orc_boa_search_wl.argtypes = [vp, vp, i64, vp, vp, i32, vp, i32, dbl, dbl, i32, i32,
                                         i32, i32, i32, C.c_float, vp, vp, vp, vp, vp, vp, vp]
         _lib = L

@@ -423,6 +423,44 @@ def test_resume_kth_distance_never_grows(small):
         prev = kth
 
 
+def test_resume_continues_the_same_search(small):
+    """What resume mode carries from phase to phase is the whole search: one beam that is
+    never saved or put back, run at 16, then on at 64, then on at 128 with the pool capacity
+    of the last width, must give the driver's resume-mode results, and the same cumulative
+    expansion and scoring counts (a restore that lost the expanded flags would expand nodes
+    again; one that lost part of the seen set would score nodes again)."""
+    w, d, ix = small
+    widths = [16, 64, 128]
+    r = ix.search(d["queries"], d["lo"], d["hi"], 10, widths, eps=-1.0, mode="resume")
+    assert (r["final_L"] == 128).all()
+    grew = 0
+    for i in range(w.Q):
+        b = ix.beam(d["queries"][i], d["lo"][i], d["hi"][i], L=16, C=128, max_expand=8 * 16 + 64)
+        e0 = b.n_expand
+        b.run(64, 8 * 64 + 64)
+        e1 = b.n_expand
+        b.run(128, 8 * 128 + 64)
+        ids, d2, _ = b.result(10)
+        assert (ids == r["ids"][i]).all() and (d2 == r["d2"][i]).all()
+        assert b.n_expand == r["n_expand"][i]
+        assert b.n_scored == r["n_scored"][i]
+        _, _, _, ex = b.pool()
+        assert ex[:128].all()
+        # later phases do continue, and do not start over: they expand more nodes, fewer
+        # than a fresh search at that width would
+        grew += int(e1 > e0)
+        fresh = ix.beam(d["queries"][i], d["lo"][i], d["hi"][i], L=128, C=128)
+        assert b.n_expand - e1 <= fresh.n_expand
+    assert grew > w.Q // 2
+    # two phases: the same relation with one hand-over
+    r2 = ix.search(d["queries"], d["lo"], d["hi"], 10, [16, 64], eps=-1.0, mode="resume")
+    for i in range(0, w.Q, 3):
+        b = ix.beam(d["queries"][i], d["lo"][i], d["hi"][i], L=16, C=64, max_expand=8 * 16 + 64)
+        b.run(64, 8 * 64 + 64)
+        assert (b.result(10)[0] == r2["ids"][i]).all()
+        assert b.n_expand == r2["n_expand"][i] and b.n_scored == r2["n_scored"][i]
+
+
 def test_single_width_schedule_is_plain_fixed_L(small):
     w, d, ix = small
     a = ix.search(d["queries"], d["lo"], d["hi"], 10, [64], mode="restart")
@@ -502,6 +540,28 @@ def test_tau_stops_the_loop(small):
     tau = (act[1] + 0.5) / w.Q          # |A| after phase 0 is not > tau*Q: phase 1 must not run
     r1 = ix.search(d["queries"], d["lo"], d["hi"], 10, widths, tau=tau)
     assert r1["phase_active"][1] == 0 and (r1["final_L"] == 16).all()
+
+
+def test_tau_boundary_is_strict(small):
+    """Algorithm 1 loops while |A| > tau * rho: with tau * rho equal to |A| exactly the next
+    phase must not run, with one query fewer it must.  The batch has a power-of-two size so
+    that tau = |A| / rho is exact in floating point."""
+    w, d, ix = small
+    Q = 32
+    q, lo, hi = d["queries"][:Q], d["lo"][:Q], d["hi"][:Q]
+    widths = default_widths(16, 128)
+    seen = set()
+    for eps in (0.05, 0.1):
+        act = ix.search(q, lo, hi, 10, widths, eps=eps, tau=0.0)["phase_active"]
+        a1 = int(act[1])
+        assert 1 < a1 < Q
+        assert (a1 / Q) * Q == a1
+        stop = ix.search(q, lo, hi, 10, widths, eps=eps, tau=a1 / Q)
+        assert stop["phase_active"][1] == 0 and (stop["final_L"] == 16).all()
+        go = ix.search(q, lo, hi, 10, widths, eps=eps, tau=(a1 - 1) / Q)
+        assert go["phase_active"][1] == a1 and (go["final_L"] > 16).sum() == a1
+        seen.add(a1)
+    assert len(seen) == 2
 
 
 # ----------------------------------------------------------------------------
