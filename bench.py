@@ -2,8 +2,9 @@
 """Benchmark of the batched adaptive filtered beam search (BOA / BOA+) on B200.
 
 One step = one boa_search over one batch of synthetic queries: every phase of
-Algorithm 1, all kernels of the hot path.  The workload is the 1M-point, 128-d,
-two-attribute configuration with a 10,000-query batch.  Prints ONE JSON line.
+Algorithm 1, all kernels of the hot path.  The headline workload is the 1M-point, 128-d,
+two-attribute configuration with a 10,000-query batch; on one GPU the other
+configurations are measured too and reported under "per_config".  Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W]        this library (CUDA)
   python bench.py --impl reference ...                        the CPU oracle, timed
@@ -33,10 +34,31 @@ METRIC = "queries/sec at recall@10>=0.95 (10k-query batch)"
 UNIT = "queries/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the search kernel per scored neighbour
-# record, from the full-size ncu capture summarised in
-# profiles/boa_search_kernel_c2_dram_traffic.md (38.24 GB for 91.20 M records).  It holds
-# for the default workload and table size only.
-NCU_DRAM_BYTES_PER_SCORED = {"c2": 419.3}
+# record, from the ncu captures summarised under profiles/ (file named beside each figure),
+# together with the digest of the kernel source the capture was taken with.  A figure is
+# used only while the kernel source still has that digest; after any change to the kernel
+# the line reports "traffic": null until the capture is repeated.
+NCU_DRAM_BYTES_PER_SCORED = {
+    # workload: (bytes per scored record, sha256[:12] of csrc/boa_search.cuh, summary file)
+}
+
+# Operating point of each workload: explicit phase widths and eps, chosen from the sweeps in
+# the design notes as the fastest setting of the adaptive method with recall@10 >= 0.95
+# (c5: the configuration's own 16 -> 512, recall below the bar, reported beside fixed 500).
+OPERATING = {
+    "c1": dict(schedule=[16, 64, 128], eps=0.05, steps=20),    # literal, disconnected graph: parity only
+    "c1b": dict(schedule=[16, 128], eps=0.02, steps=20),
+    "c2": dict(schedule=[16, 512], eps=0.03, steps=20),
+    "c3": dict(schedule=[16, 512], eps=0.03, steps=10),
+    "c4": dict(schedule=[32, 512], eps=0.05, steps=10),
+    "c5": dict(schedule=[16, 512], eps=0.03, steps=4),
+}
+
+
+def kernel_source_digest() -> str:
+    import hashlib
+    with open(os.path.join(ROOT, "paper_2609_16175_b200", "csrc", "boa_search.cuh"), "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()[:12]
 
 
 def parse_args():
@@ -48,9 +70,11 @@ def parse_args():
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--scale-n", type=int, default=0, help="debug: shrink the data set")
     ap.add_argument("--queries", type=int, default=0, help="debug: shrink the batch")
-    ap.add_argument("--eps", type=float, default=0.03)
+    ap.add_argument("--eps", type=float, default=None, help="default: the workload's operating point")
     ap.add_argument("--mode", default="resume", choices=["restart", "resume"])
-    ap.add_argument("--schedule", default="16,512")
+    ap.add_argument("--schedule", default="", help="phase widths; default: the workload's operating point")
+    ap.add_argument("--no-per-config", action="store_true",
+                    help="measure the headline workload only (always so with more than one GPU)")
     ap.add_argument("--plus-k", type=int, default=0)
     ap.add_argument("--expand-w", type=int, default=1, choices=[1, 2],
                     help="nodes expanded per iteration: 1 = Algorithm 2 as printed, 2 = extension")
@@ -87,10 +111,20 @@ def get_workload(args):
 def schedule_of(args, w):
     if getattr(args, "fixed_L", 0):
         return [int(args.fixed_L)]
+    if not args.schedule:
+        op = OPERATING.get(args.workload)
+        return list(op["schedule"]) if op and not args.scale_n else [w.L0, w.Lmax]
     s = [int(x) for x in args.schedule.split(",") if x]
-    if s[0] != w.L0 or s[-1] != w.Lmax:
-        s = [w.L0] + [x for x in s[1:-1] if w.L0 < x < w.Lmax] + [w.Lmax]
+    if s[0] != w.L0:
+        s = [w.L0] + [x for x in s[1:] if x > w.L0]
     return s
+
+
+def eps_of(args):
+    if args.eps is not None:
+        return args.eps
+    op = OPERATING.get(args.workload)
+    return op["eps"] if op else 0.05
 
 
 class ClockSampler:
@@ -255,8 +289,114 @@ def config_dict(w, widths, args):
                   "working set far above 126 MB; no flush between steps"}
 
 
+def to_device(d, dev):
+    import torch
+    return {k: torch.from_numpy(v.view(np.int32) if v.dtype == np.uint32 else v).to(dev)
+            for k, v in d.items() if k in ("vectors", "attrs", "graph", "queries", "lo", "hi")}
+
+
+def configure(ix, args, widths):
+    ix.set_param("mode", 1 if args.mode == "resume" else 0)
+    ix.set_param("eps", args.eps)
+    ix.set_param("plus_k", args.plus_k)
+    ix.set_param("expand_w", args.expand_w)
+    ix.set_param("lam", args.lam)
+    ix.set_param("table_kb", args.table_kb)
+    ix.set_param("table_tags", args.table_tags)
+    ix.set_param("max_warps_per_sm", args.max_warps)
+    ix.set_schedule(widths)
+
+
+def timed_steps(ix, t, k, widths, out_ids, out_d2, steps, warmup, barrier):
+    """W untimed steps, then exactly `steps` timed ones: CUDA events on the launching stream
+    around every step.  Returns (total ms, per-step ms list)."""
+    import torch
+    for _ in range(max(3, warmup)):
+        ix.search(t["queries"], t["lo"], t["hi"], k, widths[0], widths[-1], out_ids, out_d2)
+    barrier()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    barrier()
+    ev[0].record()
+    for s in range(steps):
+        ix.search(t["queries"], t["lo"], t["hi"], k, widths[0], widths[-1], out_ids, out_d2)
+        ev[s + 1].record()
+    torch.cuda.synchronize()
+    barrier()
+    return ev[0].elapsed_time(ev[-1]), [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+
+
+def quality(w, d, t, ix, args, widths, ids_np, d2_np, st, gt_queries, cpu_seconds):
+    """Recall against exact filtered top-k (on the first gt_queries queries), the oracle on a
+    bounded sample (parity, exact scored counts, CPU timing) and the algorithmic bytes."""
+    from boa_synth.groundtruth import filtered_topk, recall_against
+    n_gt = min(gt_queries, ids_np.shape[0])
+    gt_ids, gt_d2, gt_nv = filtered_topk(t["vectors"], t["attrs"], d["attr_types"], t["queries"][:n_gt],
+                                         t["lo"][:n_gt], t["hi"][:n_gt], w.k)
+    rec = recall_against(ids_np[:n_gt], d2_np[:n_gt], gt_d2.cpu().numpy(), gt_nv.cpu().numpy(), w.k)
+    del gt_ids, gt_d2, gt_nv
+    orc, o, n_s, dt_s = run_oracle_sample(w, d, widths, args, cpu_seconds)
+    parity_ok = bool((o["ids"] == ids_np[:n_s]).all() and (o["final_L"] == st["final_L"][:n_s]).all()
+                     and (o["n_expand"] == st["n_expand"][:n_s]).all()
+                     and (o["d2"].view(np.uint32) == d2_np[:n_s].view(np.uint32)).all())
+    ratio = float(o["n_scored"].sum()) / max(1.0, float(st["n_scored"][:n_s].sum()))
+    del orc
+    return dict(recall=float(np.nanmean(rec)), recall_queries=n_gt, parity=parity_ok, unique_ratio=ratio,
+                cpu_qps=n_s / dt_s, cpu_n=n_s, cpu_dt=dt_s)
+
+
+def measure_config(name, args, dev, steps, cpu_seconds, fixed_widths=(), gt_queries=10_000):
+    """One workload at its operating point, then at each fixed beamwidth asked for, on one
+    build of its inputs: the entries of per_config (keys name, name_fixed<L>)."""
+    import copy
+    import torch
+    from boa_synth import ALL, make_workload
+    from paper_2609_16175_b200 import BoaIndex
+    w = ALL[name]
+    t0 = time.perf_counter()
+    d = make_workload(w, seed=args.seed, device=str(dev))
+    t_build = time.perf_counter() - t0
+    t = to_device(d, dev)
+    ix = BoaIndex(t["vectors"], t["attrs"], d["attr_types"].tolist(), t["graph"])
+    out_ids = torch.empty((w.Q, w.k), dtype=torch.int32, device=dev)
+    out_d2 = torch.empty((w.Q, w.k), dtype=torch.float32, device=dev)
+    peak, peak_kind = measured_peak_gbs()
+    res = {}
+    for fixed_L in (0,) + tuple(fixed_widths):
+        a = copy.copy(args)
+        a.workload, a.scale_n, a.queries, a.schedule, a.fixed_L = name, 0, 0, "", fixed_L
+        a.eps = OPERATING[name]["eps"]
+        a.plus_k, a.expand_w, a.lam, a.table_kb, a.table_tags, a.max_warps = 0, 1, float("inf"), 0, 0, 0
+        widths = schedule_of(a, w)
+        configure(ix, a, widths)
+        n_steps = steps if not fixed_L else max(3, steps // 2)
+        total_ms, step_ms = timed_steps(ix, t, w.k, widths, out_ids, out_d2, n_steps, 3, torch.cuda.synchronize)
+        st = {kk: v.cpu().numpy() for kk, v in ix.stats().items()}
+        counts = ix.phase_counts()
+        ids_np, d2_np = out_ids.cpu().numpy().view(np.uint32), out_d2.cpu().numpy()
+        ql = quality(w, d, t, ix, a, widths, ids_np, d2_np, st, gt_queries, cpu_seconds)
+        alg = algorithmic_bytes(w, st, ql["unique_ratio"], a.mode, widths)
+        ms = total_ms / n_steps
+        res[name if not fixed_L else f"{name}_fixed{fixed_L}"] = {
+            "workload": config_dict(w, widths, a)["workload"], "schedule": widths, "eps": a.eps, "mode": a.mode,
+            "steps": n_steps, "ms_per_step": ms, "queries_per_s": w.Q / (ms / 1e3),
+            "recall_at_10": ql["recall"], "recall_queries": ql["recall_queries"],
+            "avg_beamwidth": float(st["final_L"].mean()), "phase_active": counts,
+            "mean_expansions": float(st["n_expand"].mean()), "mean_scored": float(st["n_scored"].mean()),
+            "rescored_fraction": 1.0 - ql["unique_ratio"], "capped_fraction": float((st["flags"] & 1).mean()),
+            "algorithmic_bytes_per_step": alg, "achieved_gbs": alg / (ms / 1e3) / 1e9,
+            "frac": alg / (ms / 1e3) / 1e9 / peak, "peak_kind": peak_kind,
+            "parity_with_oracle_on_sample": ql["parity"], "oracle_sample_queries": ql["cpu_n"],
+            "cpu_oracle_queries_per_s": ql["cpu_qps"], "gpu_launches_per_step": ix.last_launch_count,
+            "device_status": ix.device_status(), "fixture_build_s": round(t_build, 1)}
+    ix.close()
+    del t, d, ix, out_ids, out_d2
+    torch.cuda.empty_cache()
+    return res
+
+
 def main():
     args = parse_args()
+    args.eps = eps_of(args)
     if args.impl == "reference":
         reference_arm(args)
         return
@@ -264,7 +404,6 @@ def main():
     import torch
     import torch.distributed as dist
     from boa_synth import make_workload
-    from boa_synth.groundtruth import filtered_topk, recall_against
     from paper_2609_16175_b200 import BoaIndex
 
     rank, world, local = dist_env()
@@ -278,24 +417,12 @@ def main():
     w = get_workload(args)
     widths = schedule_of(args, w)
     d = make_workload(w, seed=args.seed, device=str(dev))
-    t = {k: torch.from_numpy(v.view(np.int32) if v.dtype == np.uint32 else v).to(dev)
-         for k, v in d.items() if k in ("vectors", "attrs", "graph", "queries", "lo", "hi")}
+    t = to_device(d, dev)
     ix = BoaIndex(t["vectors"], t["attrs"], d["attr_types"].tolist(), t["graph"])
-    ix.set_param("mode", 1 if args.mode == "resume" else 0)
-    ix.set_param("eps", args.eps)
-    ix.set_param("plus_k", args.plus_k)
-    ix.set_param("expand_w", args.expand_w)
-    ix.set_param("lam", args.lam)
-    ix.set_param("table_kb", args.table_kb)
-    ix.set_param("table_tags", args.table_tags)
-    ix.set_param("max_warps_per_sm", args.max_warps)
-    ix.set_schedule(widths)
+    configure(ix, args, widths)
     Q, k = w.Q, w.k
     out_ids = torch.empty((Q, k), dtype=torch.int32, device=dev)
     out_d2 = torch.empty((Q, k), dtype=torch.float32, device=dev)
-
-    def step():
-        ix.search(t["queries"], t["lo"], t["hi"], k, widths[0], widths[-1], out_ids, out_d2)
 
     def barrier():
         if world > 1:
@@ -303,23 +430,11 @@ def main():
         torch.cuda.synchronize()
 
     # ---- device-resident timing: W warm-up steps, then exactly K timed steps
-    for _ in range(max(3, args.warmup)):
-        step()
-    barrier()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    barrier()
-    ev[0].record()
-    for s in range(args.steps):
-        step()
-        ev[s + 1].record()
-    torch.cuda.synchronize()
-    barrier()
-    total_ms = ev[0].elapsed_time(ev[-1])
-    step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    total_ms, step_ms = timed_steps(ix, t, k, widths, out_ids, out_d2, args.steps, args.warmup, barrier)
     launches = ix.last_launch_count * args.steps
     ms_per_step = max_over_ranks(total_ms, dev, world) / args.steps
     value = whole_job_value(Q, world, ms_per_step)
@@ -377,28 +492,42 @@ def main():
             dist.destroy_process_group()
         return
 
-    # ---- recall against exact filtered top-k (torch brute force: harness, not search path)
-    gt_ids, gt_d2, gt_nv = filtered_topk(t["vectors"], t["attrs"], d["attr_types"], t["queries"],
-                                         t["lo"], t["hi"], k)
-    rec = recall_against(ids_np, d2_np, gt_d2.cpu().numpy(), gt_nv.cpu().numpy(), k)
-    recall = float(np.nanmean(rec))
-
-    # ---- CPU baseline: the oracle on a bounded sample; also gives the exact scored counts
-    orc, o, n_s, dt_s = run_oracle_sample(w, d, widths, args, args.cpu_seconds)
-    parity_ok = bool((o["ids"] == ids_np[:n_s]).all() and (o["final_L"] == st["final_L"][:n_s]).all()
-                     and (o["n_expand"] == st["n_expand"][:n_s]).all())
-    ratio = float(o["n_scored"].sum()) / max(1.0, float(st["n_scored"][:n_s].sum()))
-    cpu_qps = n_s / dt_s
+    # ---- recall, oracle sample (parity, CPU baseline, exact scored counts)
+    ql = quality(w, d, t, ix, args, widths, ids_np, d2_np, st, 10_000, args.cpu_seconds)
+    recall = ql["recall"]
 
     # ---- roofline of the search kernel (HBM-bound random gather)
     peak, peak_kind = measured_peak_gbs()
-    alg_bytes = algorithmic_bytes(w, st, ratio, args.mode, widths)
+    alg_bytes = algorithmic_bytes(w, st, ql["unique_ratio"], args.mode, widths)
     kernel_ms = float(np.mean(step_ms))
     achieved = alg_bytes / (kernel_ms / 1e3) / 1e9
-    traffic = None
-    if (args.workload in NCU_DRAM_BYTES_PER_SCORED and not args.scale_n and not args.table_kb and not args.table_tags
-            and args.expand_w == 1):
-        traffic = NCU_DRAM_BYTES_PER_SCORED[args.workload] * float(st["n_scored"].sum())
+    traffic, traffic_note = None, "no ncu capture on file for this workload and kernel source"
+    cap = NCU_DRAM_BYTES_PER_SCORED.get(args.workload)
+    plain = not (args.scale_n or args.table_kb or args.table_tags or args.expand_w != 1 or args.fixed_L)
+    if cap and plain and cap[1] == kernel_source_digest() and widths == OPERATING[args.workload]["schedule"]:
+        traffic = cap[0] * float(st["n_scored"].sum())
+        traffic_note = f"{cap[0]} DRAM bytes per scored record ({cap[2]}) x records scored in this run"
+
+    # ---- the fastest fixed beamwidth that reaches the same recall bar, for comparison
+    fixed_same = None
+    if plain and not args.scale_n and world == 1:
+        from boa_synth.groundtruth import filtered_topk, recall_against
+        gt_ids, gt_d2, gt_nv = filtered_topk(t["vectors"], t["attrs"], d["attr_types"], t["queries"],
+                                             t["lo"], t["hi"], k)
+        gt_d2, gt_nv = gt_d2.cpu().numpy(), gt_nv.cpu().numpy()
+        ix.set_param("mode", 0)
+        for L in (48, 56, 64, 72, 80, 96, 128, 192, 256, 512):
+            if L < w.L0:
+                continue
+            ix.set_schedule([L])
+            tot, _ = timed_steps(ix, t, k, [L], out_ids, out_d2, 5, 3, torch.cuda.synchronize)
+            r = float(np.nanmean(recall_against(out_ids.cpu().numpy().view(np.uint32), out_d2.cpu().numpy(),
+                                                gt_d2, gt_nv, k)))
+            if r >= 0.95:
+                fixed_same = {"L": L, "recall_at_10": r, "ms_per_step": tot / 5, "queries_per_s": Q / (tot / 5 / 1e3)}
+                break
+        configure(ix, args, widths)
+        del gt_ids, gt_d2, gt_nv
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -409,18 +538,34 @@ def main():
         "avg_beamwidth": float(st["final_L"].mean()),
         "phase_active": phase_counts,
         "mean_expansions": float(st["n_expand"].mean()), "mean_scored": float(st["n_scored"].mean()),
-        "rescored_fraction": 1.0 - ratio, "capped_fraction": float((st["flags"] & 1).mean()),
-        "parity_with_oracle_on_sample": parity_ok,
+        "rescored_fraction": 1.0 - ql["unique_ratio"], "capped_fraction": float((st["flags"] & 1).mean()),
+        "parity_with_oracle_on_sample": ql["parity"],
+        "fixed_L_at_same_recall": fixed_same,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": traffic, "peak_kind": peak_kind,
+                     "frac": achieved / peak, "traffic": traffic, "traffic_note": traffic_note,
+                     "peak_kind": peak_kind,
                      "kernel": "boa_search_kernel, all phase launches of one step",
                      "kernel_ms_per_step": kernel_ms, "algorithmic_bytes_per_step": alg_bytes},
-        "cpu_baseline": {"value": cpu_qps, "unit": UNIT, "cores": 1, "kind": "oracle",
-                         "sample": f"first {n_s} queries of the batch, full index, {dt_s:.1f} s"},
+        "cpu_baseline": {"value": ql["cpu_qps"], "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": f"first {ql['cpu_n']} queries of the batch, full index, {ql['cpu_dt']:.1f} s"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches,
         "clocks": clocks,
     }
+    ix.close()
+    del t, d, ix, dq, dlo, dhi
+    torch.cuda.empty_cache()
+
+    # ---- the other configurations, one GPU only
+    if world == 1 and plain and not args.no_per_config and args.workload == "c2":
+        per = {}
+        for name in ("c1", "c1b", "c3", "c4", "c5"):
+            try:
+                per.update(measure_config(name, args, dev, OPERATING[name]["steps"], 3.0,
+                                          fixed_widths=(500,) if name == "c5" else ()))
+            except Exception as e:           # one workload failing must not lose the line
+                per[name] = {"error": f"{type(e).__name__}: {e}"}
+        line["per_config"] = per
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -15,7 +15,10 @@ the int32 matrix; `attr_types[j]` says how to read column j (0 = int32,
 """
 from __future__ import annotations
 
+import hashlib
 import math
+import os
+import tempfile
 from typing import Dict
 
 import numpy as np
@@ -273,7 +276,8 @@ def mixed_graph(w: Workload, vectors: np.ndarray, attrs: np.ndarray, types: np.n
     crank = np.argsort(cdist, axis=1, kind="stable")        # crank[c][0] == c
     t_near = min(w.t_near, nc)
     fracs = [f for f in w.attr_fracs if f > 0] if r_attr > 0 else []
-    ranks = torch.from_numpy(_rank_columns(attrs, types)[order]).to(dev) if fracs else None
+    ranks01 = _rank_columns(attrs, types)
+    ranks = torch.from_numpy(ranks01[order]).to(dev) if fracs else None
 
     graph = np.full((n, R), SENTINEL, dtype=np.uint32)
     xs = torch.from_numpy(np.ascontiguousarray(vectors[order].astype(np.float32))).to(dev)
@@ -326,18 +330,20 @@ def mixed_graph(w: Workload, vectors: np.ndarray, attrs: np.ndarray, types: np.n
                     col0 += cnt
     # reverse edges: v gets up to r_rev of the nodes that point at it, in a seeded random order
     if r_rev > 0:
-        src = np.repeat(np.arange(n, dtype=np.int64), r_knn)
-        dst = graph[:, :r_knn].reshape(-1).astype(np.int64)
+        gk = torch.from_numpy(graph[:, :r_knn].astype(np.int64)).to(dev)
+        src = torch.arange(n, dtype=torch.int64, device=dev).repeat_interleave(r_knn)
+        dst = gk.reshape(-1)
         ok = dst != int(SENTINEL)
         src, dst = src[ok], dst[ok]
-        shuffle = rng.permutation(src.shape[0])
+        shuffle = torch.from_numpy(rng.permutation(int(src.shape[0]))).to(dev)
         src, dst = src[shuffle], dst[shuffle]
-        o = np.argsort(dst, kind="stable")
+        o = torch.argsort(dst, stable=True)
         src, dst = src[o], dst[o]
-        first = np.searchsorted(dst, np.arange(n))
-        pos = np.arange(dst.shape[0]) - first[dst]
+        first = torch.searchsorted(dst, torch.arange(n, dtype=torch.int64, device=dev))
+        pos = torch.arange(dst.shape[0], dtype=torch.int64, device=dev) - first[dst]
         keep = pos < r_rev
-        graph[dst[keep], r_knn + pos[keep]] = src[keep].astype(np.uint32)
+        graph[dst[keep].cpu().numpy(), (r_knn + pos[keep]).cpu().numpy()] = src[keep].cpu().numpy().astype(np.uint32)
+        del gk, src, dst, ok, shuffle, o, first, pos, keep
     # long edges: cell rank drawn log-uniformly in [1, nc); inside that cell the point whose
     # attributes are nearest to the node's own along a Z-order curve over the attribute
     # ranks (plus a small random offset), so that long hops tend to stay inside a range
@@ -348,12 +354,14 @@ def mixed_graph(w: Workload, vectors: np.ndarray, attrs: np.ndarray, types: np.n
         tgt_cell = crank[cell[:, None], rank]
         size = (starts[1:] - starts[:-1])[tgt_cell]
         if w.long_attr_aware:
-            zc = _zorder(_rank_columns(attrs, types))
-            key = cell.astype(np.int64) * (1 << 32) + zc
-            korder = np.argsort(key, kind="stable")         # grouped by cell, Z-ordered inside
-            ksorted = key[korder]
-            want = tgt_cell.astype(np.int64) * (1 << 32) + zc[:, None]
-            pos = np.searchsorted(ksorted, want.reshape(-1)).reshape(n, r_long)
+            zc = _zorder(ranks01)
+            key = torch.from_numpy(cell.astype(np.int64) * (1 << 32) + zc).to(dev)
+            korder_t = torch.argsort(key, stable=True)      # grouped by cell, Z-ordered inside
+            ksorted = key[korder_t]
+            want = torch.from_numpy(tgt_cell.astype(np.int64) * (1 << 32) + zc[:, None]).to(dev)
+            pos = torch.searchsorted(ksorted, want.reshape(-1)).reshape(n, r_long).cpu().numpy()
+            korder = korder_t.cpu().numpy()
+            del key, korder_t, ksorted, want
             pos = pos + rng.integers(-2, 3, size=(n, r_long))
             pos = np.clip(pos, starts[tgt_cell], np.maximum(starts[tgt_cell + 1] - 1, starts[tgt_cell]))
             tgt = korder[np.minimum(pos, n - 1)].astype(np.uint32)
@@ -362,26 +370,82 @@ def mixed_graph(w: Workload, vectors: np.ndarray, attrs: np.ndarray, types: np.n
             tgt = order[np.minimum(starts[tgt_cell] + off, n - 1)].astype(np.uint32)
         tgt = np.where(size > 0, tgt, SENTINEL)
         graph[:, R - r_long:] = tgt
-    return clean_rows(graph)
+    return clean_rows(graph, str(dev))
 
 
-def clean_rows(graph: np.ndarray) -> np.ndarray:
+def clean_rows(graph: np.ndarray, device: str = "cpu") -> np.ndarray:
     """Replace self references and repeated ids inside a row by the sentinel."""
     n, R = graph.shape
-    g = graph.copy()
-    g[g == np.arange(n, dtype=np.uint32)[:, None]] = SENTINEL
+    dev = torch.device(device)
+    g = torch.from_numpy(np.ascontiguousarray(graph).view(np.int32).copy()).to(dev)   # sentinel == -1
+    g[g == torch.arange(n, dtype=torch.int32, device=dev)[:, None]] = -1
     for j in range(1, R):
-        dup = (g[:, :j] == g[:, j:j + 1]).any(axis=1)
-        g[dup, j] = SENTINEL
-    return g
+        dup = (g[:, :j] == g[:, j:j + 1]).any(dim=1)
+        g[dup, j] = -1
+    return g.cpu().numpy().view(np.uint32)
 
 
 # ----------------------------------------------------------------------------
 # entry point
 # ----------------------------------------------------------------------------
+_CACHED = ("vectors", "queries", "attrs", "attr_types", "lo", "hi", "target_sel", "cluster", "graph")
+
+
+def _cache_dir(w: Workload, seed: int, dev: torch.device, with_graph: bool) -> str | None:
+    """Where the arrays of a large workload are kept between processes on one machine, or
+    None.  Building the 10M-point graph takes minutes; a test run and a benchmark run on the
+    same machine then build it once.  The key covers the whole description, the seed, the
+    kind of device that found the neighbours and the source of this package, so a change of
+    recipe never meets old arrays.  BOA_SYNTH_CACHE=0 switches it off, another value moves it."""
+    where = os.environ.get("BOA_SYNTH_CACHE", "")
+    if where == "0" or w.N < 500_000 or not with_graph:
+        return None
+    h = hashlib.sha256()
+    h.update(repr(w).encode())
+    h.update(f"|{seed}|{dev.type}|".encode())
+    here = os.path.dirname(os.path.abspath(__file__))
+    for name in ("generate.py", "configs.py"):
+        with open(os.path.join(here, name), "rb") as f:
+            h.update(f.read())
+    root = where or os.path.join(tempfile.gettempdir(), "boa_synth_cache")
+    return os.path.join(root, f"{w.name}_{h.hexdigest()[:16]}")
+
+
+def _cache_load(path: str):
+    try:
+        if not os.path.exists(os.path.join(path, "done")):
+            return None
+        return {k: np.load(os.path.join(path, k + ".npy")) for k in _CACHED}
+    except Exception:
+        return None
+
+
+def _cache_store(path: str, out: Dict[str, np.ndarray]) -> None:
+    try:
+        os.makedirs(path, exist_ok=True)
+        for k in _CACHED:
+            np.save(os.path.join(path, k + ".npy"), out[k])
+        with open(os.path.join(path, "done"), "w") as f:
+            f.write("ok")
+    except Exception:
+        pass                      # a full or read-only disk only costs the next build
+
+
 def make_workload(w: Workload, seed: int = 0, device: str | None = None,
                   with_graph: bool = True) -> Dict[str, np.ndarray]:
     """Build every input array of workload `w` for `seed`."""
+    cache = _cache_dir(w, seed, _prep_device(device), with_graph)
+    if cache:
+        hit = _cache_load(cache)
+        if hit is not None:
+            return hit
+    out = _build_workload(w, seed, device, with_graph)
+    if cache:
+        _cache_store(cache, out)
+    return out
+
+
+def _build_workload(w: Workload, seed: int, device: str | None, with_graph: bool) -> Dict[str, np.ndarray]:
     ss = np.random.SeedSequence(seed).spawn(5)
     vectors, queries, cl, centres = _make_vectors(w, ss[0], ss[3])
     rng_a = np.random.default_rng(ss[1])

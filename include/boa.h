@@ -75,8 +75,9 @@ enum {
                                way; a finite lambda lets invalid nodes push valid ones out
                                of the pool.                                                  */
     BOA_PARAM_EXPAND_W = 9  /* nodes expanded per iteration of Algorithm 2.  1 (default) is
-                               the algorithm as printed ("each iteration expands one
-                               node").  2 is an extension: the first two unexpanded beam
+                               the algorithm as printed (one node per iteration, Section
+                               "How Filtered Search Works").  2 is an extension: the first
+                               two unexpanded beam
                                entries are marked and their rows scored together (first
                                node's row first), at most as many as the expansion cap
                                leaves.  Changes which nodes get expanded, hence results.  */
@@ -92,7 +93,7 @@ enum {
  *   attr_types  HOST array [m]
  *   graph       [N][R] node ids, BOA_NO_ID pads short rows; self references and
  *               repeated ids inside a row are tolerated (ignored by the search)
- *   entry       start node s of every search (Algorithm 2, "entry medoid s"); -1 = the
+ *   entry       start node s of every search (the entry medoid of Algorithm 2); -1 = the
  *               point nearest to the coordinate-wise mean, lower id on ties
  *
  * The index copies and re-lays-out everything into device memory it owns, so the
@@ -159,7 +160,8 @@ int boa_search(boa_index* index, const float* queries, int64_t Q, const void* lo
  *     previous call's contents (what must start at zero is cleared on `stream` at the
  *     start of each call), and two calls whose GPU work overlaps in time race on it --
  *     run them one after the other, on one stream or ordered by events;
- *   - boa_get_stats and boa_get_phase_counts do not cover this call.
+ *   - boa_get_stats and boa_get_phase_counts do not cover this call: they keep
+ *     describing the last boa_search on the index.
  */
 #define BOA_NOALLOC_MAX_Q 1024
 #define BOA_NOALLOC_MAX_WIDTH 512

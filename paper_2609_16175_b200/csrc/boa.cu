@@ -8,6 +8,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
 #include <new>
 
 #include "boa_search.cuh"
@@ -26,6 +27,14 @@ thread_local int g_last_cuda = 0;
     } while (0)
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// The index's buffers live on the device that was current when it was built: a search
+// launched with another device current would hand its kernels foreign pointers.
+inline bool on_device(int device)
+{
+    int cur = -1;
+    return cudaGetDevice(&cur) == cudaSuccess && cur == device;
+}
 
 // ------------------------------------------------------------------ index build kernels
 // Record i = [vector bytes | zero padding], rec_stride bytes.  The attribute cells live in
@@ -192,6 +201,11 @@ constexpr int kCntStatus = 47;                        // device status bits
 constexpr int kCntTicket = 48;                        // one per launch
 constexpr int kMaxLaunches = 128;
 constexpr int kCntWords = kCntTicket + kMaxLaunches;   // 176: the 64-bit words after it stay aligned
+#ifdef BOA_SECTION_TIMERS
+constexpr size_t kTimerBytes = 12 * sizeof(unsigned long long);   // debug builds: cycle counters
+#else
+constexpr size_t kTimerBytes = 0;
+#endif
 
 // ---- scratch of boa_search_noalloc: lives in the library image, never allocated
 constexpr int64_t kNoAllocMaxQ = BOA_NOALLOC_MAX_Q;
@@ -202,7 +216,7 @@ constexpr size_t kNaStats = kNaLists + (size_t)2 * BOA_MAX_PHASES * kNoAllocMaxQ
 constexpr size_t kNaSpillSize = kNaStats + (size_t)4 * kNoAllocMaxQ * 4;
 constexpr size_t kNaSpill = kNaSpillSize + (size_t)kNoAllocMaxQ * 4;
 constexpr size_t kNaBytes = kNaSpill + (size_t)kNoAllocMaxQ * kNoAllocMaxWidth * 8;
-static_assert(kCntWords * 4 + 12 * 8 <= 1024, "counter block must fit its slot");
+static_assert(kCntWords * 4 + kTimerBytes <= 1024, "counter block must fit its slot");
 static_assert(kNaSpill % 256 == 0 && kNaStats % 256 == 0, "sub-buffers stay aligned");
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaBytes];
@@ -210,19 +224,22 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaBytes];
 // In host code `g_noalloc_scratch` is only a handle for the runtime, not an address a
 // kernel can use: the device address is asked for once per device and kept here.
 constexpr int kMaxDevices = 64;
-unsigned char* g_noalloc_ptr[kMaxDevices] = {nullptr};
+std::atomic<unsigned char*> g_noalloc_ptr[kMaxDevices];
 
 int noalloc_scratch(unsigned char** out)
 {
     int dev = 0;
     BOA_CUDA(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return BOA_EINVAL;
-    if (!g_noalloc_ptr[dev]) {
+    unsigned char* cached = g_noalloc_ptr[dev].load(std::memory_order_acquire);
+    if (!cached) {
+        // two threads may both ask; they get the same address
         void* ptr = nullptr;
         BOA_CUDA(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
-        g_noalloc_ptr[dev] = static_cast<unsigned char*>(ptr);
+        cached = static_cast<unsigned char*>(ptr);
+        g_noalloc_ptr[dev].store(cached, std::memory_order_release);
     }
-    *out = g_noalloc_ptr[dev];
+    *out = cached;
     return BOA_OK;
 }
 
@@ -342,9 +359,8 @@ int ensure_workspace(boa_index* ix, int64_t Q, int Lmax)
 {
     const int need_spill = ix->mode == 1 ? ((Lmax + 1) & ~1) : 0;
     if (ix->counters == nullptr) {
-        // 12 trailing 64-bit words: section timers of debug builds
-        BOA_CUDA(cudaMalloc(&ix->counters, kCntWords * sizeof(uint32_t) + 12 * sizeof(unsigned long long)));
-        BOA_CUDA(cudaMemset(ix->counters, 0, kCntWords * sizeof(uint32_t) + 12 * sizeof(unsigned long long)));
+        BOA_CUDA(cudaMalloc(&ix->counters, kCntWords * sizeof(uint32_t) + kTimerBytes));
+        BOA_CUDA(cudaMemset(ix->counters, 0, kCntWords * sizeof(uint32_t) + kTimerBytes));
     }
     if (Q > ix->ws_Q || need_spill > ix->ws_spill) {
         const int64_t nq = Q > ix->ws_Q ? Q : ix->ws_Q;
@@ -607,7 +623,9 @@ int boa_set_param(boa_index* ix, int key, double v)
             if (v != 0.0 && v != 16.0) return BOA_EINVAL;
             ix->table_tags = (int)v; return BOA_OK;
         case BOA_PARAM_LAMBDA:
-            if (!(v >= 0.0)) return BOA_EINVAL;
+            // finite values must stay finite as fp32: an overflow to +inf would turn the
+            // score of every filter-valid node into inf * 0
+            if (!(v >= 0.0) || (!isinf(v) && v > 3.4028234663852886e38)) return BOA_EINVAL;
             ix->lambda = v; return BOA_OK;
         case BOA_PARAM_EXPAND_W:
             if (v != 1.0 && v != 2.0) return BOA_EINVAL;
@@ -647,6 +665,7 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
     if (ix->n_sched > 0 && (L0 != ix->sched[0] || Lmax != ix->sched[ix->n_sched - 1])) return BOA_EINVAL;
     if (Q == 0) { ix->last_Q = 0; ix->last_phases = 0; ix->last_launches = 0; return BOA_OK; }
     if (!queries || !lo || !hi || !out_ids || !out_dists) return BOA_EINVAL;
+    if (!on_device(ix->device)) return BOA_EINVAL;
     if (!aligned16(queries) || !aligned16(lo) || !aligned16(hi) || !aligned16(out_ids) ||
         !aligned16(out_dists))
         return BOA_EINVAL;
@@ -665,7 +684,9 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
     b.rec = ix->rec; b.graph = ix->graph; b.N = ix->N; b.D = ix->D; b.m = ix->m; b.R = ix->R;
     b.rec_stride = ix->rec_stride; b.nchunks = ix->nchunks;
     b.attrs = ix->attr_cells; b.status = ix->counters + kCntStatus;
+#ifdef BOA_SECTION_TIMERS
     b.timers = reinterpret_cast<unsigned long long*>(ix->counters + kCntWords);
+#endif
     b.attr_float_mask = ix->attr_float_mask; b.entry = (uint32_t)ix->entry;
     b.queries = queries;
     b.lo = reinterpret_cast<const int32_t*>(lo);
@@ -798,6 +819,7 @@ int boa_search_noalloc(boa_index* ix, const float* queries, int64_t Q, const voi
 {
     if (!ix) return BOA_EINVAL;
     if (Q > kNoAllocMaxQ || Lmax > kNoAllocMaxWidth) return BOA_ETOOBIG;
+    if (!on_device(ix->device)) return BOA_EINVAL;
     unsigned char* base = nullptr;
     const int rc0 = noalloc_scratch(&base);
     if (rc0 != BOA_OK) return rc0;
@@ -807,7 +829,10 @@ int boa_search_noalloc(boa_index* ix, const float* queries, int64_t Q, const voi
     struct Saved {
         uint32_t *lists, *counters; int32_t *stats, *spill_size; uint64_t* spill;
         int64_t ws_Q; int ws_spill;
-    } sv = {ix->lists, ix->counters, ix->stats, ix->spill_size, ix->spill, ix->ws_Q, ix->ws_spill};
+        int64_t last_Q; int last_phases, last_launches; int last_widths[BOA_MAX_PHASES];
+    } sv = {ix->lists, ix->counters, ix->stats, ix->spill_size, ix->spill, ix->ws_Q, ix->ws_spill,
+            ix->last_Q, ix->last_phases, ix->last_launches, {0}};
+    memcpy(sv.last_widths, ix->last_widths, sizeof(sv.last_widths));
     ix->counters = reinterpret_cast<uint32_t*>(base + kNaCounters);
     ix->lists = reinterpret_cast<uint32_t*>(base + kNaLists);
     ix->stats = reinterpret_cast<int32_t*>(base + kNaStats);
@@ -818,8 +843,10 @@ int boa_search_noalloc(boa_index* ix, const float* queries, int64_t Q, const voi
     const int rc = boa_search(ix, queries, Q, lo, hi, k, L0, Lmax, out_ids, out_dists, stream);
     ix->lists = sv.lists; ix->counters = sv.counters; ix->stats = sv.stats;
     ix->spill_size = sv.spill_size; ix->spill = sv.spill; ix->ws_Q = sv.ws_Q; ix->ws_spill = sv.ws_spill;
-    ix->last_Q = 0;            // the per-query statistics of this call are not kept
-    ix->last_phases = 0;
+    // boa_get_stats / boa_get_phase_counts keep describing the last boa_search: this call's
+    // statistics sit in the shared array, which the next call overwrites
+    ix->last_Q = sv.last_Q; ix->last_phases = sv.last_phases; ix->last_launches = sv.last_launches;
+    memcpy(ix->last_widths, sv.last_widths, sizeof(sv.last_widths));
     return rc;
 }
 

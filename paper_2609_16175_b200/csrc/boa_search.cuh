@@ -1,5 +1,5 @@
 // Warp-per-query filter-aware beam search (Algorithm 2) with the confidence test
-// (Eq. 3) and survivor compaction (Algorithm 1, "compact active queries") fused
+// (Eq. 3) and survivor compaction (the gather step of Algorithm 1) fused
 // into its epilogue.  sm_100a only.
 //
 // One warp (one CTA of 32 threads) owns one query from start to convergence.  Its
@@ -55,6 +55,16 @@ namespace boa {
 #endif
 #ifndef BOA_SHORT_RPG2
 #define BOA_SHORT_RPG2 4
+#endif
+
+// L2 prefetch of the rows about to be scored (all of an expansion's rows are requested as
+// soon as they are known, so only the first scoring pass waits for DRAM) and of the
+// adjacency row of the probable next node.
+#ifndef BOA_PREFETCH_ROWS
+#define BOA_PREFETCH_ROWS 1
+#endif
+#ifndef BOA_PREFETCH_ADJ
+#define BOA_PREFETCH_ADJ 1
 #endif
 
 constexpr uint32_t kNoId = 0xFFFFFFFFu;
@@ -125,7 +135,9 @@ struct SearchParams {
     uint32_t* out_list;            // survivors of this phase
     uint32_t* out_count;
     uint32_t* status;              // device status word (kStatus* bits)
-    unsigned long long* timers;    // section cycle counters (only with BOA_SECTION_TIMERS)
+#ifdef BOA_SECTION_TIMERS
+    unsigned long long* timers;    // section cycle counters of debug builds
+#endif
     // per-query state
     int32_t* final_L;
     int32_t* n_expand;
@@ -232,6 +244,11 @@ __device__ __forceinline__ uint32_t ldg_stream32(const void* ptr, bool pred)
         : "l"(ptr), "r"((uint32_t)pred));
     return v;
 }
+// Ask for the 128-byte line holding `ptr` to be brought into L2; nothing waits for it.
+__device__ __forceinline__ void prefetch_l2(const void* ptr)
+{
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr));
+}
 __device__ __forceinline__ float sq_acc4u(float acc, uint4 x, float4 q);
 
 __device__ __forceinline__ float sq_acc4(float acc, float4 x, float4 q)
@@ -259,6 +276,16 @@ __device__ __forceinline__ float sq_acc_bytes(float acc, uint32_t w, float4 q)
     d = (__uint_as_float(__byte_perm(w, 0x4B000000u, 0x7441)) - magic) - q.y; acc = fmaf(d, d, acc);
     d = (__uint_as_float(__byte_perm(w, 0x4B000000u, 0x7442)) - magic) - q.z; acc = fmaf(d, d, acc);
     d = (__uint_as_float(__byte_perm(w, 0x4B000000u, 0x7443)) - magic) - q.w; acc = fmaf(d, d, acc);
+    return acc;
+}
+
+// acc + sum over the 16 byte pairs of two 16-byte chunks of a[i]*b[i]
+__device__ __forceinline__ uint32_t dot4_bytes(uint4 a, uint4 b, uint32_t acc)
+{
+    acc = __dp4a(a.x, b.x, acc);
+    acc = __dp4a(a.y, b.y, acc);
+    acc = __dp4a(a.z, b.z, acc);
+    acc = __dp4a(a.w, b.w, acc);
     return acc;
 }
 
@@ -353,7 +380,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
     const uint32_t w_begin = p.in_begin_ptr ? *p.in_begin_ptr : p.in_begin;
     const uint32_t w_end = p.in_end_ptr ? *p.in_end_ptr : p.in_end;
     if (p.active_count) {
-        // Algorithm 1: "while |A| > tau * rho"
+        // loop condition of Algorithm 1: a phase runs only while |A| exceeds tau * rho
         if (!((double)(*p.active_count) > p.tau_q)) return;
     }
     const uint32_t n_work = w_end > w_begin ? w_end - w_begin : 0u;
@@ -393,6 +420,39 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
 #pragma unroll
                 for (int f = 0; f < QF4; ++f)
                     qreg[i * QF4 + f] = (c < p.nchunks) ? __ldg(qsrc + c * QF4 + f) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+        // Byte rows against a query whose elements are themselves whole numbers 0..255 (the
+        // usual case when data and queries come from one byte-valued source): every term
+        // (x-q)^2 and every partial sum of at most 256 of them is an integer below 2^24, so
+        // fp32 accumulation in any order is exact and equals the integer sum.  The distance
+        // is then computed with 4-way byte dot products, sum x*x - 2 sum x*q + sum q*q, two
+        // instructions per four elements instead of sixteen.  The query bytes take the place
+        // of the first float slices in qreg; qq_lane is this lane's sum q*q.
+        bool q_bytes = false;
+        int qq_lane = 0;
+        if (VT == 1 && (CPL == 1 || CPL == 2)) {
+            bool ok = true;
+#pragma unroll
+            for (int j = 0; j < NQ; ++j) {
+                const float4 v = qreg[j];
+                ok = ok && v.x >= 0.f && v.x <= 255.f && v.x == truncf(v.x) && v.y >= 0.f && v.y <= 255.f &&
+                     v.y == truncf(v.y) && v.z >= 0.f && v.z <= 255.f && v.z == truncf(v.z) && v.w >= 0.f &&
+                     v.w <= 255.f && v.w == truncf(v.w);
+            }
+            q_bytes = __all_sync(0xffffffffu, ok);
+            if (q_bytes) {
+                uint32_t wq[NQ];
+#pragma unroll
+                for (int j = 0; j < NQ; ++j) {
+                    const float4 v = qreg[j];
+                    wq[j] = (uint32_t)v.x | ((uint32_t)v.y << 8) | ((uint32_t)v.z << 16) | ((uint32_t)v.w << 24);
+                    qq_lane = (int)__dp4a(wq[j], wq[j], (uint32_t)qq_lane);
+                }
+#pragma unroll
+                for (int i = 0; i < (CPL > 0 ? CPL : 1); ++i)
+                    qreg[i] = make_float4(__uint_as_float(wq[4 * i + 0]), __uint_as_float(wq[4 * i + 1]),
+                                          __uint_as_float(wq[4 * i + 2]), __uint_as_float(wq[4 * i + 3]));
             }
         }
 
@@ -475,16 +535,29 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
 #pragma unroll
                     for (int t = 0; t < RPG; ++t) {
                         a[t] = 0.0f;
+                        if (VT == 1 && q_bytes) {
+                            uint32_t xx = 0u, xq = 0u;
 #pragma unroll
-                        for (int i = 0; i < NC; ++i) {
-                            if (!EXACT && g + 8 * i >= p.nchunks) continue;
-                            if (VT == 0) {
-                                a[t] = sq_acc4u(a[t], x[t][i], qreg[i]);
-                            } else {
-                                a[t] = sq_acc_bytes(a[t], x[t][i].x, qreg[4 * i + 0]);
-                                a[t] = sq_acc_bytes(a[t], x[t][i].y, qreg[4 * i + 1]);
-                                a[t] = sq_acc_bytes(a[t], x[t][i].z, qreg[4 * i + 2]);
-                                a[t] = sq_acc_bytes(a[t], x[t][i].w, qreg[4 * i + 3]);
+                            for (int i = 0; i < NC; ++i) {
+                                if (!EXACT && g + 8 * i >= p.nchunks) continue;
+                                xx = dot4_bytes(x[t][i], x[t][i], xx);
+                                xq = dot4_bytes(x[t][i], make_uint4(__float_as_uint(qreg[i].x), __float_as_uint(qreg[i].y),
+                                                                    __float_as_uint(qreg[i].z), __float_as_uint(qreg[i].w)), xq);
+                            }
+                            // this lane's sum of (x-q)^2: a whole number in [0, 2^24)
+                            a[t] = (float)((int)xx - 2 * (int)xq + qq_lane);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < NC; ++i) {
+                                if (!EXACT && g + 8 * i >= p.nchunks) continue;
+                                if (VT == 0) {
+                                    a[t] = sq_acc4u(a[t], x[t][i], qreg[i]);
+                                } else {
+                                    a[t] = sq_acc_bytes(a[t], x[t][i].x, qreg[4 * i + 0]);
+                                    a[t] = sq_acc_bytes(a[t], x[t][i].y, qreg[4 * i + 1]);
+                                    a[t] = sq_acc_bytes(a[t], x[t][i].z, qreg[4 * i + 2]);
+                                    a[t] = sq_acc_bytes(a[t], x[t][i].w, qreg[4 * i + 3]);
+                                }
                             }
                         }
                         c_av[t] = av[t];
@@ -722,6 +795,11 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             if (PRED) {
                 pred_pos = first_unexpanded(cur, n < p.L ? n : p.L);
                 load_row_ids(pred_pos >= 0 ? key_id(fin, pool[pred_pos]) : kNoId, nbp, 0);
+            } else if (BOA_PREFETCH_ADJ) {
+                // no early load here, but the line(s) of that row can be on their way to L2
+                const int guess = first_unexpanded(cur, n < p.L ? n : p.L);
+                if (guess >= 0 && lane * 32 < p.R)
+                    prefetch_l2(p.graph + (size_t)key_id(fin, pool[guess]) * p.R + lane * 32);
             }
             BOA_T_MARK(1);
 
@@ -732,10 +810,27 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                 if (W > 1 && s == RN) __syncwarp();   // the second row sees what the first recorded
                 const bool fresh = (nb[s] != kNoId) && hash_test_and_set(nb[s]);
                 const unsigned bal = __ballot_sync(0xffffffffu, fresh);
-                if (fresh) cand[cnt + __popc(bal & lt_mask)] = nb[s];
+                if (fresh) {
+                    cand[cnt + __popc(bal & lt_mask)] = nb[s];
+                    if (BOA_PREFETCH_ROWS && p.rec_stride <= 512) {
+                        const uint8_t* row = p.rec + (size_t)nb[s] * p.rec_stride;
+                        for (int off = 0; off < p.rec_stride; off += 128) prefetch_l2(row + off);
+                        prefetch_l2(p.attrs + (size_t)nb[s] * p.m);
+                    }
+                }
                 cnt += __popc(bal);
             }
             __syncwarp();
+            if (BOA_PREFETCH_ROWS && p.rec_stride > 512) {
+                // long rows: the lanes share the lines of one row at a time
+                const int lines = (p.rec_stride + 127) >> 7;
+                for (int j = 0; j < cnt; ++j) {
+                    const uint8_t* row = p.rec + (size_t)cand[j] * p.rec_stride;
+                    for (int l = lane; l < lines; l += 32) prefetch_l2(row + 128 * l);
+                }
+                if (lane < cnt) prefetch_l2(p.attrs + (size_t)cand[lane] * p.m);
+                if (lane + 32 < cnt) prefetch_l2(p.attrs + (size_t)cand[lane + 32] * p.m);
+            }
             BOA_T_MARK(2);
             int kept = 0, live = 0;
             uint64_t x[RS];

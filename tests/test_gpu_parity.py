@@ -204,6 +204,16 @@ def test_eps_and_tau_special_cases():
         o = orc.search(d["queries"], d["lo"], d["hi"], w.k, widths, tau=tau, dist_mode=1)
         r = gpu_search(gpu, g, w.k, widths, tau=tau)
         assert_bit_parity(o, r, f"tau={tau}")
+    # the boundary itself: tau * rho == |A| stops (strict > of Algorithm 1); 256 queries make
+    # tau exact in floating point
+    sl = slice(0, 256)
+    a1 = int(orc.search(d["queries"][sl], d["lo"][sl], d["hi"][sl], w.k, widths, dist_mode=1)["phase_active"][1])
+    assert 1 < a1 < 256
+    for tau in (a1 / 256, (a1 - 1) / 256):
+        o = orc.search(d["queries"][sl], d["lo"][sl], d["hi"][sl], w.k, widths, tau=tau, dist_mode=1)
+        r = gpu_search(gpu, g, w.k, widths, tau=tau, sel=sl)
+        assert_bit_parity(o, r, f"tau boundary {tau}")
+    assert o["phase_active"][1] == a1
 
 
 def test_expansion_cap():
@@ -291,6 +301,12 @@ def test_empty_batch_and_argument_errors():
     for k, L0, Lmax in ((0, 16, 64), (17, 16, 64), (10, 64, 16), (10, 16, 4096)):
         with pytest.raises(BoaError):
             gpu.search(g["queries"], g["lo"], g["hi"], k, L0, Lmax)
+    # a finite lambda must stay finite in fp32; infinity (the default) is accepted
+    with pytest.raises(BoaError) as e:
+        gpu.set_param("lam", 1e39)
+    assert e.value.status == -1
+    gpu.set_param("lam", 3.0e38)
+    gpu.set_param("lam", float("inf"))
     bad = g["graph"].clone()
     bad[5, 2] = w.N + 3
     from paper_2609_16175_b200 import BoaIndex

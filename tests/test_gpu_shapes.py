@@ -70,6 +70,46 @@ def test_shape_variants_match_oracle(case):
     gpu.close()
 
 
+@pytest.mark.parametrize("D", [128, 48, 256, 192, 272])
+def test_byte_rows_with_queries_of_every_kind(D):
+    """uint8 rows take an integer dot-product path when the query is itself byte-valued and
+    the fp32 path otherwise; both must equal the oracle's fixed-order fp32 distance bit for
+    bit.  The batch mixes whole-number queries, fractional ones, values outside 0..255, one
+    fractional element at the very end, and the two extreme rows (all 0 against all 255: the
+    largest distance, D * 255^2, still below 2^24 at D = 256)."""
+    N, Q, m, R = 3000, 64, 2, 24
+    d = _random_case(77 + D, N, D, "u8", m, R, Q)
+    rng = np.random.default_rng(D)
+    d["vectors"][0] = 0
+    d["vectors"][1] = 255
+    q = d["queries"]
+    q[0] = 255.0
+    q[1] = 0.0
+    q[8:24] += rng.random((16, D)).astype(np.float32)           # fractional everywhere
+    q[24, -1] += 0.25                                             # one fractional element, last lane
+    q[25, 0] = 256.0                                              # just outside the byte range
+    q[26, D // 2] = -1.0
+    q[27] = -q[27]                                                # all negative (and -0.0)
+    q[28, 3] = np.float32(1e-30)                                  # tiny, not a whole number
+    q[29] = q[29] * 4.0                                           # whole numbers up to 1020
+    d["lo"][:, :] = np.iinfo(np.int32).min                        # every point valid: distances decide
+    d["hi"][:, :] = np.iinfo(np.int32).max
+    d["hi"][32:, 0] = 500                                         # and a filtered half
+    orc, gpu, g = make_pair(d, entry=0)
+    for mode, widths in (("restart", [16, 64]), ("resume", [12, 300])):
+        o = orc.search(q, d["lo"], d["hi"], 10, widths, eps=0.1, mode=mode, dist_mode=1)
+        r = gpu_search(gpu, g, 10, widths, mode=mode, eps=0.1)
+        assert_bit_parity(o, r, f"u8 D={D} {mode}")
+    # the entry point alone (no expansion allowed): the all-zero row against the all-255
+    # query is the largest distance there is, and must come out exactly
+    r = gpu_search(gpu, g, 1, [1], cap=(0, 0), sel=slice(0, 2))
+    o = orc.search(q[:2], d["lo"][:2], d["hi"][:2], 1, [1], cap=(0, 0), dist_mode=1)
+    assert_bit_parity(o, r, f"u8 D={D} entry only")
+    assert r["ids"][:, 0].tolist() == [0, 0]
+    assert r["d2"][:, 0].tolist() == [D * 255.0 ** 2, 0.0] and orc.dist2_f64(q[0], 0) == D * 255.0 ** 2
+    gpu.close()
+
+
 def test_degenerate_sizes():
     """One point, two points, one query, every neighbour slot empty."""
     for N in (1, 2, 5):
