@@ -57,14 +57,15 @@ namespace boa {
 #define BOA_SHORT_RPG2 4
 #endif
 
-// L2 prefetch of the rows about to be scored (all of an expansion's rows are requested as
-// soon as they are known, so only the first scoring pass waits for DRAM) and of the
-// adjacency row of the probable next node.
+// L2 prefetch of the rows about to be scored: all of an expansion's rows are requested as
+// soon as they are known, so only the first scoring pass waits for DRAM.  Measured on B200:
+// +2 to +5 % for rows of 384 and 512 bytes (three scoring passes of eight rows); nothing
+// or a loss for 128-byte rows (16 to a pass already) and for rows of several KB (the
+// requests cost more issue slots than the latency they hide), so only rows of 129..512
+// bytes use it.  Requesting the adjacency row of the probable next node the same way
+// measured as no gain and is not done.
 #ifndef BOA_PREFETCH_ROWS
 #define BOA_PREFETCH_ROWS 1
-#endif
-#ifndef BOA_PREFETCH_ADJ
-#define BOA_PREFETCH_ADJ 1
 #endif
 
 constexpr uint32_t kNoId = 0xFFFFFFFFu;
@@ -795,11 +796,6 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             if (PRED) {
                 pred_pos = first_unexpanded(cur, n < p.L ? n : p.L);
                 load_row_ids(pred_pos >= 0 ? key_id(fin, pool[pred_pos]) : kNoId, nbp, 0);
-            } else if (BOA_PREFETCH_ADJ) {
-                // no early load here, but the line(s) of that row can be on their way to L2
-                const int guess = first_unexpanded(cur, n < p.L ? n : p.L);
-                if (guess >= 0 && lane * 32 < p.R)
-                    prefetch_l2(p.graph + (size_t)key_id(fin, pool[guess]) * p.R + lane * 32);
             }
             BOA_T_MARK(1);
 
@@ -812,7 +808,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                 const unsigned bal = __ballot_sync(0xffffffffu, fresh);
                 if (fresh) {
                     cand[cnt + __popc(bal & lt_mask)] = nb[s];
-                    if (BOA_PREFETCH_ROWS && p.rec_stride <= 512) {
+                    if (BOA_PREFETCH_ROWS && p.rec_stride > 128 && p.rec_stride <= 512) {
                         const uint8_t* row = p.rec + (size_t)nb[s] * p.rec_stride;
                         for (int off = 0; off < p.rec_stride; off += 128) prefetch_l2(row + off);
                         prefetch_l2(p.attrs + (size_t)nb[s] * p.m);
@@ -821,16 +817,6 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                 cnt += __popc(bal);
             }
             __syncwarp();
-            if (BOA_PREFETCH_ROWS && p.rec_stride > 512) {
-                // long rows: the lanes share the lines of one row at a time
-                const int lines = (p.rec_stride + 127) >> 7;
-                for (int j = 0; j < cnt; ++j) {
-                    const uint8_t* row = p.rec + (size_t)cand[j] * p.rec_stride;
-                    for (int l = lane; l < lines; l += 32) prefetch_l2(row + 128 * l);
-                }
-                if (lane < cnt) prefetch_l2(p.attrs + (size_t)cand[lane] * p.m);
-                if (lane + 32 < cnt) prefetch_l2(p.attrs + (size_t)cand[lane + 32] * p.m);
-            }
             BOA_T_MARK(2);
             int kept = 0, live = 0;
             uint64_t x[RS];
