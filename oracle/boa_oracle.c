@@ -14,6 +14,10 @@
  *   orc_beam_*         filter-aware beam search at one beamwidth (Algorithm 2),
  *                      with exact L2 distances instead of PQ look-ups
  *   orc_uncertain      confidence test gamma(D_i) <= eps (Eq. 3)
+ *   orc_pq_*           product-quantised traversal (Algorithm 2's PQDist line; Section "BOA
+ *                      Implementation on a GPU System": the per-query distance table, the
+ *                      asymmetric PQ distance as a sum of table look-ups, and the final
+ *                      ranking of the candidates by exact distance with invalid ones excluded)
  *   orc_boa_search_wl  multi-phase driver (Algorithm 1)
  *
  * Readings of points the paper leaves open (each is listed in the design notes):
@@ -33,12 +37,20 @@
  *   - a phase stops after cap_mult*L + cap_add expansions at the latest
  *   - expansion width W (nodes expanded per iteration) is 1 as in the paper unless a
  *     caller asks for more; see orc_beam_run_w
+ *   - with PQ traversal the keys of the search are PQ distances; when a phase has converged
+ *     the filter-valid entries of the beam (the first L pool entries, the worklist of
+ *     Algorithm 2) are ranked by exact distance, the k nearest are the result, and the
+ *     confidence test reads those exact distances
  *
  * parity pins: tests/test_oracle_pins.py (brute force vs. an independent sort,
  * g == 1 vs. a library k-NN, the ring-graph hand trace, full-graph search ==
  * brute force, restart/resume relations, eps special cases, L_avg vs. the
  * paper's Table III).  Unpinned by the paper itself: the exact trajectories on
  * large inputs, the constants alpha, tau, lambda.
+ * PQ pins: tests/test_oracle_pq_pins.py (hand-worked table and look-up sums, numpy, a
+ * lossless codebook == the exact search, a full-width beam == brute force, properties of
+ * the final ranking).  Unpinned by the paper: which candidates the final ranking covers
+ * (taken: the filter-valid entries of the beam).
  */
 #include <math.h>
 #include <stdint.h>
@@ -60,6 +72,10 @@ typedef struct {
     const int32_t *attr_types; /* [m]                          */
     const uint32_t *graph;    /* [N][R], ORC_SENTINEL = no edge */
     int64_t entry;
+    /* product quantisation (optional): D = pq_M * dsub */
+    int pq_M, pq_K;
+    const float *pq_pivots;   /* [M][K][dsub] centroids of every subspace */
+    const uint8_t *pq_codes;  /* [N][M] centroid index of every point in every subspace */
 } orc_index;
 
 /* ------------------------------------------------------------------ */
@@ -139,6 +155,62 @@ int orc_phi(const orc_index *ix, const int32_t *lo, const int32_t *hi, int64_t p
         }
     }
     return v;
+}
+
+/* ------------------------------------------------------------------ */
+/* product quantisation                                                */
+/* ------------------------------------------------------------------ */
+/* The vector space is cut into M subspaces of dsub = D/M consecutive dimensions; every
+   subspace has K centroids ("pivots"); a point is stored as the M indices of its nearest
+   centroids.  The codebook is an input (trained by whoever built the index). */
+void orc_pq_attach(orc_index *ix, const float *pivots, const uint8_t *codes, int M, int K)
+{
+    ix->pq_M = M; ix->pq_K = K; ix->pq_pivots = pivots; ix->pq_codes = codes;
+}
+
+/* The distance table of one query: table[m][c] = squared L2 distance between the m-th
+   subvector of q and centroid c of subspace m.  dist_mode 1: fp32, one
+   acc = fmaf(q - piv, q - piv, acc) per dimension in ascending order; dist_mode 0: the same
+   sum in double, rounded once to float. */
+void orc_pq_table(const orc_index *ix, const float *q, int dist_mode, float *table)
+{
+    const int M = ix->pq_M, K = ix->pq_K, dsub = ix->D / M;
+    for (int m = 0; m < M; ++m)
+        for (int c = 0; c < K; ++c) {
+            const float *piv = ix->pq_pivots + ((size_t)m * K + c) * dsub;
+            if (dist_mode == 1) {
+                float acc = 0.0f;
+                for (int i = 0; i < dsub; ++i) {
+                    float diff = q[m * dsub + i] - piv[i];
+                    acc = fmaf(diff, diff, acc);
+                }
+                table[m * K + c] = acc;
+            } else {
+                double acc = 0.0;
+                for (int i = 0; i < dsub; ++i) {
+                    double diff = (double)q[m * dsub + i] - (double)piv[i];
+                    acc += diff * diff;
+                }
+                table[m * K + c] = (float)acc;
+            }
+        }
+}
+
+/* Asymmetric PQ distance of point p: the sum over the subspaces of the table entry its
+   code selects, added in ascending subspace order (fp32 in mode 1, double rounded once in
+   mode 0). */
+float orc_pq_dist(const orc_index *ix, const float *table, int dist_mode, int64_t p)
+{
+    const int M = ix->pq_M, K = ix->pq_K;
+    const uint8_t *code = ix->pq_codes + (size_t)p * M;
+    if (dist_mode == 1) {
+        float acc = 0.0f;
+        for (int m = 0; m < M; ++m) acc = acc + table[m * K + code[m]];
+        return acc;
+    }
+    double acc = 0.0;
+    for (int m = 0; m < M; ++m) acc += (double)table[m * K + code[m]];
+    return (float)acc;
 }
 
 /* ------------------------------------------------------------------ */
@@ -228,6 +300,7 @@ typedef struct {
     int64_t ntouched, touched_cap;
     int64_t n_expand, n_scored;
     int hit_cap;
+    float *pq_table;     /* [M][K] of the current query when the search runs on PQ distances, else NULL */
 } orc_state;
 
 /* The order the search works by.  The paper's score is dist + lambda*phi with one lambda
@@ -259,7 +332,25 @@ orc_state *orc_state_new(const orc_index *ix, int C)
 void orc_state_set_lambda(orc_state *st, float lambda) { st->lambda = lambda; }
 void orc_state_free(orc_state *st)
 {
-    free(st->pool); free(st->seen); free(st->touched); free(st);
+    free(st->pool); free(st->seen); free(st->touched); free(st->pq_table); free(st);
+}
+
+/* Switch the state to PQ traversal for query q (on != 0: the distance table is built here),
+   or back to exact distances.  Call before orc_beam_init, and again before a resumed run
+   of another query. */
+void orc_state_use_pq(orc_state *st, int on, const float *q, int dist_mode)
+{
+    if (!on) { free(st->pq_table); st->pq_table = NULL; return; }
+    if (!st->pq_table)
+        st->pq_table = (float *)malloc((size_t)st->ix->pq_M * st->ix->pq_K * sizeof(float));
+    orc_pq_table(st->ix, q, dist_mode, st->pq_table);
+}
+
+/* the distance the traversal orders by */
+static float orc_search_dist(const orc_state *st, const float *q, int64_t p, int dist_mode)
+{
+    if (st->pq_table) return orc_pq_dist(st->ix, st->pq_table, dist_mode, p);
+    return orc_dist2(st->ix, q, p, dist_mode);
 }
 
 static void orc_mark_seen(orc_state *st, uint32_t id)
@@ -291,7 +382,7 @@ void orc_beam_init(orc_state *st, int C, const float *q, const int32_t *lo, cons
     orc_entry_t e;
     e.id = (uint32_t)ix->entry; e.expanded = 0;
     e.phi = orc_phi(ix, lo, hi, ix->entry);
-    e.d2 = orc_dist2(ix, q, ix->entry, dist_mode);
+    e.d2 = orc_search_dist(st, q, ix->entry, dist_mode);
     orc_mark_seen(st, e.id);
     orc_pool_insert(st, e);
 }
@@ -337,7 +428,7 @@ void orc_beam_run_w(orc_state *st, int L, const float *q, const int32_t *lo, con
                 orc_entry_t e;
                 e.id = n; e.expanded = 0;
                 e.phi = orc_phi(ix, lo, hi, n);
-                e.d2 = orc_dist2(ix, q, n, dist_mode);
+                e.d2 = orc_search_dist(st, q, n, dist_mode);
                 orc_pool_insert(st, e);
             }
         }
@@ -373,6 +464,16 @@ void orc_state_pool(const orc_state *st, uint32_t *ids, float *d2, int32_t *phi,
  * evaluated without square roots as d2_k >= (1-eps)^2 * d2_max, in fp32, the
  * constant rounded once to float.  Returns 1 when the query must escalate.
  */
+static int orc_gap_uncertain(int nv, int k, float d2k, float d2max, double eps)
+{
+    if (nv <= k) return 1;
+    if (eps < 0.0) return 1;
+    if (eps >= 1.0) return 0;
+    float c = (float)((1.0 - eps) * (1.0 - eps));
+    float rhs = c * d2max;
+    return !(d2k >= rhs);
+}
+
 int orc_uncertain(const orc_state *st, int L, int k, double eps)
 {
     int lim = st->size < L ? st->size : L;
@@ -384,12 +485,48 @@ int orc_uncertain(const orc_state *st, int L, int k, double eps)
         if (nv == k) d2k = st->pool[t].d2;
         d2max = st->pool[t].d2;                           /* entries ascend */
     }
-    if (nv <= k) return 1;
-    if (eps < 0.0) return 1;
-    if (eps >= 1.0) return 0;
-    float c = (float)((1.0 - eps) * (1.0 - eps));
-    float rhs = c * d2max;
-    return !(d2k >= rhs);
+    return orc_gap_uncertain(nv, k, d2k, d2max, eps);
+}
+
+/*
+ * End of a PQ search ("Re-rank exact": on convergence the candidates are ranked by exact
+ * distance, invalid ones excluded).  V = the filter-valid entries among the first L pool
+ * entries.  Every member of V gets its exact squared distance; V is ordered by (d2, id);
+ * the first k are the result (padded as usual).  Returns |V|; *d2k and *d2max receive the
+ * k-th and the largest exact distance of V (what the confidence test reads), 0 when
+ * |V| < k or V is empty.
+ */
+int orc_beam_rerank(const orc_state *st, int L, int k, const float *q, int dist_mode,
+                    uint32_t *out_ids, float *out_d2, float *d2k, float *d2max)
+{
+    int lim = st->size < L ? st->size : L;
+    uint32_t *vid = (uint32_t *)malloc((size_t)(lim + 1) * sizeof(uint32_t));
+    float *vd = (float *)calloc((size_t)lim + 1, sizeof(float));
+    int nv = 0;
+    for (int t = 0; t < lim; ++t) {
+        if (st->pool[t].phi != 0) continue;
+        uint32_t id = st->pool[t].id;
+        float d = orc_dist2(st->ix, q, id, dist_mode);
+        int pos = nv;                                      /* insertion by (d2, id) */
+        while (pos > 0 && (d < vd[pos - 1] || (d == vd[pos - 1] && id < vid[pos - 1]))) {
+            vd[pos] = vd[pos - 1]; vid[pos] = vid[pos - 1]; pos--;
+        }
+        vd[pos] = d; vid[pos] = id; nv++;
+    }
+    for (int t = 0; t < k; ++t) {
+        if (t < nv) { out_ids[t] = vid[t]; out_d2[t] = vd[t]; }
+        else { out_ids[t] = ORC_SENTINEL; out_d2[t] = INFINITY; }
+    }
+    *d2k = nv >= k ? vd[k - 1] : 0.0f;
+    *d2max = nv > 0 ? vd[nv - 1] : 0.0f;
+    free(vid); free(vd);
+    return nv;
+}
+
+/* Eq. 3 on the exact distances a PQ search ends with */
+int orc_uncertain_reranked(int nv, int k, float d2k, float d2max, double eps)
+{
+    return orc_gap_uncertain(nv, k, d2k, d2max, eps);
 }
 
 /* ------------------------------------------------------------------ */
@@ -442,6 +579,7 @@ void orc_boa_search_wl(const orc_index *ix, const float *queries, int64_t Q,
                       const int32_t *lo, const int32_t *hi, int k,
                       const int32_t *widths, int n_widths, double eps, double tau,
                       int mode, int dist_mode, int cap_mult, int cap_add, int W, float lambda,
+                      int use_pq,
                       uint32_t *out_ids, float *out_d2,
                       int32_t *final_L, int32_t *n_expand, int32_t *n_scored, int32_t *flags,
                       int64_t *phase_active)
@@ -468,6 +606,7 @@ void orc_boa_search_wl(const orc_index *ix, const float *queries, int64_t Q,
             if (!active[i]) continue;
             const float *q = queries + i * ix->D;
             const int32_t *l = lo + i * ix->m, *h = hi + i * ix->m;
+            if (use_pq) orc_state_use_pq(st, 1, q, dist_mode);      /* this query's distance table */
             if (mode == 1 && saved[i]) {
                 orc_restore(st, saved[i], Cmax);
                 orc_saved_free(saved[i]); saved[i] = NULL;
@@ -475,12 +614,20 @@ void orc_boa_search_wl(const orc_index *ix, const float *queries, int64_t Q,
                 orc_beam_init(st, mode == 1 ? Cmax : L, q, l, h, dist_mode);
             }
             orc_beam_run_w(st, L, q, l, h, dist_mode, cap, W);
-            orc_beam_result(st, k, out_ids + i * k, out_d2 + i * k);    /* scatter */
+            int unc;
+            if (use_pq) {
+                float d2k, d2max;
+                int nv = orc_beam_rerank(st, L, k, q, dist_mode, out_ids + i * k, out_d2 + i * k, &d2k, &d2max);
+                unc = orc_gap_uncertain(nv, k, d2k, d2max, eps);
+            } else {
+                orc_beam_result(st, k, out_ids + i * k, out_d2 + i * k);    /* scatter */
+                unc = orc_uncertain(st, L, k, eps);
+            }
             final_L[i] = L;
             n_expand[i] += (int32_t)st->n_expand;
             n_scored[i] += (int32_t)st->n_scored;
             if (st->hit_cap) flags[i] |= 1;
-            if (!orc_uncertain(st, L, k, eps)) {                    /* F: confident */
+            if (!unc) {                                             /* F: confident */
                 active[i] = 0; n_active--;
             } else if (mode == 1 && p + 1 < n_widths) {
                 saved[i] = orc_save(st);

@@ -54,7 +54,16 @@ def lib():
         L.orc_uncertain.restype = i32
         L.orc_uncertain.argtypes = [vp, i32, i32, dbl]
         L.orc_boa_search_wl.argtypes = [vp, vp, i64, vp, vp, i32, vp, i32, dbl, dbl, i32, i32,
-                                        i32, i32, i32, C.c_float, vp, vp, vp, vp, vp, vp, vp]
+                                        i32, i32, i32, C.c_float, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.orc_pq_attach.argtypes = [vp, vp, vp, i32, i32]
+        L.orc_pq_table.argtypes = [vp, vp, i32, vp]
+        L.orc_pq_dist.restype = C.c_float
+        L.orc_pq_dist.argtypes = [vp, vp, i32, i64]
+        L.orc_state_use_pq.argtypes = [vp, i32, vp, i32]
+        L.orc_beam_rerank.restype = i32
+        L.orc_beam_rerank.argtypes = [vp, i32, i32, vp, i32, vp, vp, vp, vp]
+        L.orc_uncertain_reranked.restype = i32
+        L.orc_uncertain_reranked.argtypes = [i32, i32, C.c_float, C.c_float, dbl]
         _lib = L
     return _lib
 
@@ -113,6 +122,26 @@ class OracleIndex:
     def medoid(self):
         return int(lib().orc_medoid(self.h))
 
+    # --- product quantisation ------------------------------------------------
+    def attach_pq(self, pivots, codes):
+        """pivots [M][K][D/M] float32, codes [N][M] uint8 (the arrays are kept, not copied)."""
+        self.pq_pivots = np.ascontiguousarray(pivots, dtype=np.float32)
+        self.pq_codes = np.ascontiguousarray(codes, dtype=np.uint8)
+        M, K, dsub = self.pq_pivots.shape
+        assert M * dsub == self.D and self.pq_codes.shape == (self.N, M) and K <= 256
+        self.pq_M, self.pq_K = M, K
+        lib().orc_pq_attach(self.h, _p(self.pq_pivots), _p(self.pq_codes), M, K)
+
+    def pq_table(self, q, dist_mode=0):
+        q = np.ascontiguousarray(q, dtype=np.float32)
+        t = np.empty((self.pq_M, self.pq_K), dtype=np.float32)
+        lib().orc_pq_table(self.h, _p(q), int(dist_mode), _p(t))
+        return t
+
+    def pq_dist(self, table, p, dist_mode=0):
+        table = np.ascontiguousarray(table, dtype=np.float32)
+        return np.float32(lib().orc_pq_dist(self.h, _p(table), int(dist_mode), int(p)))
+
     # --- exact filtered top-k ------------------------------------------------
     def bruteforce(self, queries, lo, hi, k):
         queries = np.ascontiguousarray(queries, dtype=np.float32)
@@ -129,13 +158,13 @@ class OracleIndex:
 
     # --- one beam search, step-wise ------------------------------------------
     def beam(self, q, lo, hi, L, C=None, dist_mode=0, max_expand=1 << 40, expand_w=1,
-             lam=float("inf")):
+             lam=float("inf"), pq=False):
         return OracleBeam(self, q, lo, hi, L, C if C is not None else L, dist_mode, max_expand,
-                          expand_w, lam)
+                          expand_w, lam, pq)
 
     # --- the multi-phase batch driver ----------------------------------------
     def search(self, queries, lo, hi, k, widths, eps=0.05, tau=0.0, mode="restart",
-               dist_mode=0, cap=DEFAULT_CAP, expand_w=1, lam=float("inf")):
+               dist_mode=0, cap=DEFAULT_CAP, expand_w=1, lam=float("inf"), pq=False):
         queries = np.ascontiguousarray(queries, dtype=np.float32)
         lo = np.ascontiguousarray(lo, dtype=np.int32)
         hi = np.ascontiguousarray(hi, dtype=np.int32)
@@ -150,7 +179,8 @@ class OracleIndex:
         phase_active = np.zeros(len(w), dtype=np.int64)
         lib().orc_boa_search_wl(self.h, _p(queries), Q, _p(lo), _p(hi), k, _p(w), len(w),
                                float(eps), float(tau), 1 if mode == "resume" else 0, int(dist_mode),
-                               int(cap[0]), int(cap[1]), int(expand_w), float(lam), _p(ids), _p(d2), _p(final_L),
+                               int(cap[0]), int(cap[1]), int(expand_w), float(lam), 1 if pq else 0,
+                               _p(ids), _p(d2), _p(final_L),
                                _p(n_expand), _p(n_scored), _p(flags), _p(phase_active))
         return dict(ids=ids, d2=d2, final_L=final_L, n_expand=n_expand, n_scored=n_scored,
                     flags=flags, phase_active=phase_active)
@@ -159,8 +189,10 @@ class OracleIndex:
 class OracleBeam:
     """One query's Algorithm-2 state, for tests that look inside a search."""
 
-    def __init__(self, index, q, lo, hi, L, C, dist_mode, max_expand, expand_w=1, lam=float("inf")):
+    def __init__(self, index, q, lo, hi, L, C, dist_mode, max_expand, expand_w=1, lam=float("inf"),
+                 pq=False):
         self.ix = index
+        self.pq = bool(pq)
         self.expand_w = int(expand_w)
         self.q = np.ascontiguousarray(q, dtype=np.float32)
         self.lo = np.ascontiguousarray(lo, dtype=np.int32)
@@ -168,6 +200,8 @@ class OracleBeam:
         self.dist_mode = dist_mode
         self.st = lib().orc_state_new(index.h, int(C))
         lib().orc_state_set_lambda(self.st, float(lam))
+        if self.pq:
+            lib().orc_state_use_pq(self.st, 1, _p(self.q), dist_mode)
         lib().orc_beam_init(self.st, int(C), _p(self.q), _p(self.lo), _p(self.hi), dist_mode)
         self.run(L, max_expand)
 
@@ -182,6 +216,15 @@ class OracleBeam:
         d2 = np.empty(k, dtype=np.float32)
         n = lib().orc_beam_result(self.st, k, _p(ids), _p(d2))
         return ids, d2, n
+
+    def rerank(self, k, L=None):
+        """End of a PQ search: (ids, exact d2, |V|, d2_k, d2_max) over the valid beam entries."""
+        ids = np.empty(k, dtype=np.uint32)
+        d2 = np.empty(k, dtype=np.float32)
+        dk, dm = C.c_float(0), C.c_float(0)
+        nv = lib().orc_beam_rerank(self.st, int(self.L if L is None else L), int(k), _p(self.q),
+                                   self.dist_mode, _p(ids), _p(d2), C.byref(dk), C.byref(dm))
+        return ids, d2, nv, np.float32(dk.value), np.float32(dm.value)
 
     def pool(self):
         n = lib().orc_state_size(self.st)
