@@ -38,6 +38,8 @@ enum {
 #define BOA_MAX_WIDTH 1024 /* largest beamwidth / pool capacity */
 #define BOA_MAX_PHASES 8
 #define BOA_MAX_POINTS ((int64_t)1 << 28)
+#define BOA_PQ_MAX_SUBSPACES 64 /* largest M of a product-quantisation codebook */
+#define BOA_PQ_MAX_K 32         /* largest k of a search that traverses on PQ distances */
 
 /* Keys of boa_set_param. */
 enum {
@@ -74,6 +76,12 @@ enum {
                                multiply-add), ties by id.  Answers are filter-valid either
                                way; a finite lambda lets invalid nodes push valid ones out
                                of the pool.                                                  */
+    BOA_PARAM_PQ = 12,      /* 1 = traverse on product-quantised distances (needs
+                               boa_index_attach_pq) and rank the filter-valid beam entries by
+                               exact distance when a phase has converged: Algorithm 2's PQDist
+                               line and the "Re-rank exact" step of Section "BOA Implementation
+                               on a GPU System".  0 (default) = exact distances throughout.
+                               With 1, k <= BOA_PQ_MAX_K and BOA_PARAM_EXPAND_W must be 1.     */
     BOA_PARAM_EXPAND_W = 9  /* nodes expanded per iteration of Algorithm 2.  1 (default) is
                                the algorithm as printed (one node per iteration, Section
                                "How Filtered Search Works").  2 is an extension: the first
@@ -104,6 +112,25 @@ enum {
 int boa_index_create(boa_index** out, const void* vectors, int vec_dtype, int64_t N, int D,
                      const void* attrs, const int* attr_types, int m, const uint32_t* graph, int R,
                      int64_t entry, void* stream);
+
+/*
+ * Give the index a product-quantisation codebook (Section "BOA Implementation on a GPU
+ * System": PQ codes and quantisation pivots live in GPU memory; a query's distance table
+ * holds the distance from each of its subvectors to every centroid of that subspace, and a
+ * candidate's PQ distance is the sum of the table entries its code selects).
+ *
+ *   pivots  [M][K][D/M] float: centroid c of subspace m; subspace m covers dimensions
+ *           [m*D/M, (m+1)*D/M) of the vectors
+ *   codes   [N][M] uint8_t: index of the centroid that stands for point p in subspace m
+ *
+ * M a multiple of 16 in 16..BOA_PQ_MAX_SUBSPACES that divides D, 1 <= K <= 256.  The
+ * codebook is trained by the caller; both arrays are copied into index-owned memory (the
+ * call synchronises `stream`).  Attaching does not switch PQ traversal on: set BOA_PARAM_PQ.
+ * The distance table costs M*K*4 bytes of shared memory per resident query.
+ * Errors: BOA_EINVAL (nulls, bad M or K, misaligned pointers), BOA_ENOMEM, BOA_ECUDA.
+ */
+int boa_index_attach_pq(boa_index* index, const float* pivots, const uint8_t* codes, int M, int K,
+                        void* stream);
 
 /* Free the index and everything it owns.  NULL is accepted. */
 int boa_index_destroy(boa_index* index);
@@ -188,6 +215,10 @@ int boa_set_schedule(boa_index* index, const int* widths, int n);
  */
 int boa_get_stats(boa_index* index, int32_t* final_L, int32_t* n_expand, int32_t* n_scored,
                   int32_t* flags, void* stream);
+
+/* With PQ traversal: rows fetched per query for the final exact ranking, summed over the
+   phases it ran (DEVICE buffer of Q int32, copied on `stream`); zeros otherwise. */
+int boa_get_rerank_counts(boa_index* index, int32_t* n_rerank, void* stream);
 
 /* Number of queries that entered each phase of the last search: writes up to n values
    into the HOST array `active` and returns the number of phases in *n_phases.

@@ -16,7 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = None
 
 PARAM = dict(eps=0, growth=1, tau=2, mode=3, plus_k=4, cap_mult=5, cap_add=6, table_kb=7,
-             max_warps_per_sm=8, expand_w=9, table_tags=10, lam=11)
+             max_warps_per_sm=8, expand_w=9, table_tags=10, lam=11, pq=12)
 F32, U8 = 0, 1
 NO_ID = 0xFFFFFFFF
 
@@ -67,6 +67,10 @@ def load_library():
     L.boa_get_phase_counts.argtypes = [vp, C.POINTER(i64), i32, C.POINTER(i32), vp]
     L.boa_workspace_bytes.restype = i32
     L.boa_workspace_bytes.argtypes = [vp, i64, i32, C.POINTER(C.c_size_t)]
+    L.boa_index_attach_pq.restype = i32
+    L.boa_index_attach_pq.argtypes = [vp, vp, vp, i32, i32, vp]
+    L.boa_get_rerank_counts.restype = i32
+    L.boa_get_rerank_counts.argtypes = [vp, vp, vp]
     L.boa_last_launch_count.restype = i32
     L.boa_last_launch_count.argtypes = [vp]
     L.boa_device_status.restype = i32
@@ -140,6 +144,25 @@ class BoaIndex:
     @property
     def entry(self) -> int:
         return int(self._lib.boa_index_entry(self._h))
+
+    def attach_pq(self, pivots: torch.Tensor, codes: torch.Tensor,
+                  stream: Optional[torch.cuda.Stream] = None):
+        """boa_index_attach_pq: pivots [M][K][D/M] float32, codes [N][M] uint8 (device tensors)."""
+        pivots = _dev(pivots, "pivots")
+        codes = _dev(codes, "codes")
+        if pivots.dtype != torch.float32 or codes.dtype != torch.uint8 or pivots.dim() != 3:
+            raise ValueError("pivots must be float32 [M][K][D/M], codes uint8 [N][M]")
+        M, K = int(pivots.shape[0]), int(pivots.shape[1])
+        if tuple(codes.shape) != (self.N, M) or int(pivots.shape[2]) * M != self.D:
+            raise ValueError("codebook shape does not match the index")
+        _check(self._lib.boa_index_attach_pq(self._h, pivots.data_ptr(), codes.data_ptr(), M, K,
+                                             _stream_ptr(stream)), "boa_index_attach_pq")
+
+    def rerank_counts(self, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+        out = torch.zeros(getattr(self, "_last_Q", 0), dtype=torch.int32, device=self.device)
+        _check(self._lib.boa_get_rerank_counts(self._h, out.data_ptr(), _stream_ptr(stream)),
+               "boa_get_rerank_counts")
+        return out
 
     def set_param(self, name: str, value: float):
         _check(self._lib.boa_set_param(self._h, PARAM[name], float(value)), f"boa_set_param({name})")

@@ -143,13 +143,14 @@ __global__ void medoid_block_kernel(const void* vec, int dtype, int64_t N, int D
 }
 
 __global__ void fill_outputs_kernel(uint32_t* ids, float* d2, int64_t n, int32_t* final_L,
-                                    int32_t* n_expand, int32_t* n_scored, int32_t* flags, int64_t Q)
+                                    int32_t* n_expand, int32_t* n_scored, int32_t* flags, int32_t* n_rerank,
+                                    int64_t Q)
 {
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n;
          i += (int64_t)gridDim.x * blockDim.x) {
         ids[i] = BOA_NO_ID;
         d2[i] = __int_as_float(0x7f800000);
-        if (i < Q) { final_L[i] = 0; n_expand[i] = 0; n_scored[i] = 0; flags[i] = 0; }
+        if (i < Q) { final_L[i] = 0; n_expand[i] = 0; n_scored[i] = 0; flags[i] = 0; n_rerank[i] = 0; }
     }
 }
 
@@ -169,6 +170,10 @@ struct boa_index {
     uint8_t* rec = nullptr;
     uint32_t* graph = nullptr;
     int device = 0, num_sms = 0;
+    // product quantisation (optional)
+    uint8_t* pq_codes = nullptr;       // [N][pq_M]
+    float* pq_pivots = nullptr;        // [pq_M][pq_K][D / pq_M]
+    int pq_M = 0, pq_K = 0, use_pq = 0;
     // parameters
     double eps = 0.05, growth = 4.0, tau = 0.0;
     int mode = 0, plus_k = 0, cap_mult = 8, cap_add = 64, table_kb = 0, max_ctas = 0, expand_w = 1, table_tags = 0;
@@ -180,7 +185,7 @@ struct boa_index {
     int ws_spill = 0;
     uint32_t* lists = nullptr;     // [2][BOA_MAX_PHASES][ws_Q]: survivor lists (second set: BOA+ pool 2)
     uint32_t* counters = nullptr;  // see enum below
-    int32_t* stats = nullptr;      // [4][ws_Q]
+    int32_t* stats = nullptr;      // [5][ws_Q]
     uint64_t* spill = nullptr;     // [ws_Q][ws_spill]
     int32_t* spill_size = nullptr; // [ws_Q]
     cudaStream_t side = nullptr;
@@ -213,7 +218,7 @@ constexpr int kNoAllocMaxWidth = BOA_NOALLOC_MAX_WIDTH;
 constexpr size_t kNaCounters = 0;                                             // 1 KiB
 constexpr size_t kNaLists = 1024;                                             // [phases][Q] u32
 constexpr size_t kNaStats = kNaLists + (size_t)2 * BOA_MAX_PHASES * kNoAllocMaxQ * 4;
-constexpr size_t kNaSpillSize = kNaStats + (size_t)4 * kNoAllocMaxQ * 4;
+constexpr size_t kNaSpillSize = kNaStats + (size_t)5 * kNoAllocMaxQ * 4;
 constexpr size_t kNaSpill = kNaSpillSize + (size_t)kNoAllocMaxQ * 4;
 constexpr size_t kNaBytes = kNaSpill + (size_t)kNoAllocMaxQ * kNoAllocMaxWidth * 8;
 static_assert(kCntWords * 4 + kTimerBytes <= 1024, "counter block must fit its slot");
@@ -243,6 +248,8 @@ int noalloc_scratch(unsigned char** out)
     return BOA_OK;
 }
 
+static_assert(BOA_PQ_MAX_K == boa::kPqMaxK, "header and kernel agree on the largest k of a PQ search");
+
 typedef void (*SearchKernel)(const boa::SearchParams);
 
 struct KernelChoice {
@@ -251,39 +258,41 @@ struct KernelChoice {
     bool q_in_smem;     // the generic-length kernels keep the query in shared memory
 };
 
-template <int VT, int CPL, int W>
+template <int VT, int CPL, int W, bool PQ>
 KernelChoice pick_rn(int R, bool exact)
 {
     if (R <= 32) {
-        if (exact) return {boa::boa_search_kernel<VT, 1, W, CPL, (CPL > 0)>, W, CPL == 0};
-        return {boa::boa_search_kernel<VT, 1, W, CPL, false>, W, CPL == 0};
+        if (exact) return {boa::boa_search_kernel<VT, 1, W, CPL, (CPL > 0), PQ>, W, CPL == 0};
+        return {boa::boa_search_kernel<VT, 1, W, CPL, false, PQ>, W, CPL == 0};
     }
-    if (exact) return {boa::boa_search_kernel<VT, 2, W, CPL, (CPL > 0)>, 2 * W, CPL == 0};
-    return {boa::boa_search_kernel<VT, 2, W, CPL, false>, 2 * W, CPL == 0};
+    if (exact) return {boa::boa_search_kernel<VT, 2, W, CPL, (CPL > 0), PQ>, 2 * W, CPL == 0};
+    return {boa::boa_search_kernel<VT, 2, W, CPL, false, PQ>, 2 * W, CPL == 0};
 }
 template <int VT, int CPL>
-KernelChoice pick_rs(int R, bool exact, int expand_w)
+KernelChoice pick_rs(int R, bool exact, int expand_w, bool pq)
 {
-    return expand_w == 2 ? pick_rn<VT, CPL, 2>(R, exact) : pick_rn<VT, CPL, 1>(R, exact);
+    if (pq) return pick_rn<VT, CPL, 1, true>(R, exact);
+    return expand_w == 2 ? pick_rn<VT, CPL, 2, false>(R, exact) : pick_rn<VT, CPL, 1, false>(R, exact);
 }
 
 KernelChoice pick_kernel(const boa_index* ix)
 {
     const int cpl = (ix->nchunks + 7) / 8;      // 16-byte chunks per lane of an 8-lane group
     const bool exact = ix->nchunks == 8 * cpl;
+    const bool pq = ix->use_pq != 0;
     if (ix->vec_dtype == BOA_F32) {
         switch (cpl) {
-            case 1: return pick_rs<0, 1>(ix->R, exact, ix->expand_w);
-            case 2: return pick_rs<0, 2>(ix->R, exact, ix->expand_w);
-            case 3: return pick_rs<0, 3>(ix->R, exact, ix->expand_w);
-            case 4: return pick_rs<0, 4>(ix->R, exact, ix->expand_w);
-            default: return pick_rs<0, 0>(ix->R, false, ix->expand_w);
+            case 1: return pick_rs<0, 1>(ix->R, exact, ix->expand_w, pq);
+            case 2: return pick_rs<0, 2>(ix->R, exact, ix->expand_w, pq);
+            case 3: return pick_rs<0, 3>(ix->R, exact, ix->expand_w, pq);
+            case 4: return pick_rs<0, 4>(ix->R, exact, ix->expand_w, pq);
+            default: return pick_rs<0, 0>(ix->R, false, ix->expand_w, pq);
         }
     }
     switch (cpl) {
-        case 1: return pick_rs<1, 1>(ix->R, exact, ix->expand_w);
-        case 2: return pick_rs<1, 2>(ix->R, exact, ix->expand_w);
-        default: return pick_rs<1, 0>(ix->R, false, ix->expand_w);
+        case 1: return pick_rs<1, 1>(ix->R, exact, ix->expand_w, pq);
+        case 2: return pick_rs<1, 2>(ix->R, exact, ix->expand_w, pq);
+        default: return pick_rs<1, 0>(ix->R, false, ix->expand_w, pq);
     }
 }
 
@@ -330,7 +339,8 @@ int default_table_kb(const boa_index* ix, const KernelChoice& kc, int C)
     if (ix->rec_stride < 256) return 6;
     const int sizes[4] = {6, 4, 3, 2};
     for (int i = 0; i < 4; ++i) {
-        const boa::WarpSmem lay = boa::warp_smem_layout(C, sizes[i] * 1024, ix->D, kc.rs, kc.q_in_smem);
+        const boa::WarpSmem lay = boa::warp_smem_layout(C, sizes[i] * 1024, ix->D, kc.rs, kc.q_in_smem,
+                                                        ix->use_pq ? ix->pq_M * ix->pq_K : 0);
         if ((int64_t)BOA_MIN_CTAS * (lay.total + 1024) <= 196 * 1024) return sizes[i];
     }
     return 6;
@@ -369,7 +379,7 @@ int ensure_workspace(boa_index* ix, int64_t Q, int Lmax)
         ix->lists = nullptr; ix->stats = nullptr; ix->spill = nullptr; ix->spill_size = nullptr;
         ix->ws_Q = 0; ix->ws_spill = 0;
         BOA_CUDA(cudaMalloc(&ix->lists, (size_t)2 * BOA_MAX_PHASES * nq * sizeof(uint32_t)));
-        BOA_CUDA(cudaMalloc(&ix->stats, (size_t)4 * nq * sizeof(int32_t)));
+        BOA_CUDA(cudaMalloc(&ix->stats, (size_t)5 * nq * sizeof(int32_t)));
         BOA_CUDA(cudaMalloc(&ix->spill_size, (size_t)nq * sizeof(int32_t)));
         if (ns > 0) BOA_CUDA(cudaMalloc(&ix->spill, (size_t)nq * ns * sizeof(uint64_t)));
         ix->ws_Q = nq;
@@ -423,7 +433,8 @@ int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_p
     sp.out_list = lists_c + (size_t)(p + 1 < BOA_MAX_PHASES ? p + 1 : p) * ix->ws_Q;
     sp.out_count = cnt_c + p + 1;
 
-    const boa::WarpSmem lay = boa::warp_smem_layout(sp.C, sp.table_bytes, ix->D, lp.kc.rs, lp.kc.q_in_smem);
+    const boa::WarpSmem lay = boa::warp_smem_layout(sp.C, sp.table_bytes, ix->D, lp.kc.rs, lp.kc.q_in_smem,
+                                                    ix->use_pq ? ix->pq_M * ix->pq_K : 0);
     const size_t smem = (size_t)lay.total;
     if (smem > 48 * 1024) {
         BOA_CUDA(cudaFuncSetAttribute((const void*)lp.kc.fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -580,6 +591,7 @@ int boa_index_destroy(boa_index* ix)
     if (!ix) return BOA_OK;
     cudaFree(ix->rec); cudaFree(ix->attr_cells); cudaFree(ix->graph); cudaFree(ix->lists); cudaFree(ix->counters);
     cudaFree(ix->stats); cudaFree(ix->spill); cudaFree(ix->spill_size);
+    cudaFree(ix->pq_codes); cudaFree(ix->pq_pivots);
     if (ix->side) cudaStreamDestroy(ix->side);
     if (ix->ev_fork) cudaEventDestroy(ix->ev_fork);
     if (ix->ev_join) cudaEventDestroy(ix->ev_join);
@@ -630,6 +642,9 @@ int boa_set_param(boa_index* ix, int key, double v)
         case BOA_PARAM_EXPAND_W:
             if (v != 1.0 && v != 2.0) return BOA_EINVAL;
             ix->expand_w = (int)v; return BOA_OK;
+        case BOA_PARAM_PQ:
+            if ((v != 0.0 && v != 1.0) || (v == 1.0 && !ix->pq_codes)) return BOA_EINVAL;
+            ix->use_pq = (int)v; return BOA_OK;
         default: return BOA_EINVAL;
     }
 }
@@ -650,7 +665,7 @@ int boa_workspace_bytes(const boa_index* ix, int64_t Q, int Lmax, size_t* bytes)
 {
     if (!ix || !bytes || Q < 0 || Lmax < 1 || Lmax > BOA_MAX_WIDTH) return BOA_EINVAL;
     size_t b = kCntWords * sizeof(uint32_t);
-    b += (size_t)2 * BOA_MAX_PHASES * Q * sizeof(uint32_t) + (size_t)5 * Q * sizeof(int32_t);
+    b += (size_t)2 * BOA_MAX_PHASES * Q * sizeof(uint32_t) + (size_t)6 * Q * sizeof(int32_t);
     if (ix->mode == 1) b += (size_t)Q * ((Lmax + 1) & ~1) * sizeof(uint64_t);
     *bytes = b;
     return BOA_OK;
@@ -663,6 +678,7 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
     if (Q < 0 || Q > (int64_t)0x7FFFFFFF) return BOA_EINVAL;
     if (k < 1 || k > L0 || L0 > Lmax || Lmax > BOA_MAX_WIDTH) return BOA_EINVAL;
     if (ix->n_sched > 0 && (L0 != ix->sched[0] || Lmax != ix->sched[ix->n_sched - 1])) return BOA_EINVAL;
+    if (ix->use_pq && (k > boa::kPqMaxK || ix->expand_w != 1)) return BOA_EINVAL;
     if (Q == 0) { ix->last_Q = 0; ix->last_phases = 0; ix->last_launches = 0; return BOA_OK; }
     if (!queries || !lo || !hi || !out_ids || !out_dists) return BOA_EINVAL;
     if (!on_device(ix->device)) return BOA_EINVAL;
@@ -700,6 +716,9 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
     else { b.eps_mode = 0; b.c_eps = (float)((1.0 - ix->eps) * (1.0 - ix->eps)); }
     b.final_L = ix->stats; b.n_expand = ix->stats + ix->ws_Q; b.n_scored = ix->stats + 2 * ix->ws_Q;
     b.flags = ix->stats + 3 * ix->ws_Q;
+    b.n_rerank = ix->stats + 4 * ix->ws_Q;
+    b.pq_codes = ix->pq_codes; b.pq_pivots = ix->pq_pivots; b.pq_M = ix->pq_M; b.pq_K = ix->pq_K;
+    b.pq_dsub = ix->pq_M ? ix->D / ix->pq_M : 0;
     b.spill = ix->spill; b.spill_size = ix->spill_size; b.spill_stride = ix->ws_spill;
 
     ix->last_Q = Q;
@@ -714,7 +733,7 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
         // Algorithm 1's loop body never runs: every query returns "nothing found"
         const int64_t n = Q * k > Q ? Q * k : Q;
         fill_outputs_kernel<<<ix->num_sms * 4, 256, 0, st>>>(out_ids, out_dists, Q * k, b.final_L,
-                                                            b.n_expand, b.n_scored, b.flags, Q);
+                                                            b.n_expand, b.n_scored, b.flags, b.n_rerank, Q);
         (void)n;
         BOA_CUDA(cudaGetLastError());
         ix->last_launches = 1;
@@ -788,6 +807,34 @@ int boa_get_stats(boa_index* ix, int32_t* final_L, int32_t* n_expand, int32_t* n
         BOA_CUDA(cudaMemcpyAsync(dst[i], ix->stats + (size_t)i * ix->ws_Q,
                                  (size_t)ix->last_Q * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
     }
+    return BOA_OK;
+}
+
+int boa_index_attach_pq(boa_index* ix, const float* pivots, const uint8_t* codes, int M, int K, void* stream)
+{
+    if (!ix || !pivots || !codes) return BOA_EINVAL;
+    if (M < 16 || M > BOA_PQ_MAX_SUBSPACES || M % 16 != 0 || ix->D % M != 0) return BOA_EINVAL;
+    if (K < 1 || K > 256) return BOA_EINVAL;
+    if (!aligned16(pivots) || !aligned16(codes) || !on_device(ix->device)) return BOA_EINVAL;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    cudaFree(ix->pq_codes); cudaFree(ix->pq_pivots);
+    ix->pq_codes = nullptr; ix->pq_pivots = nullptr; ix->pq_M = 0; ix->pq_K = 0; ix->use_pq = 0;
+    const size_t cb = (size_t)ix->N * M, pb = (size_t)M * K * (ix->D / M) * sizeof(float);
+    BOA_CUDA(cudaMalloc(&ix->pq_codes, cb));
+    BOA_CUDA(cudaMalloc(&ix->pq_pivots, pb));
+    BOA_CUDA(cudaMemcpyAsync(ix->pq_codes, codes, cb, cudaMemcpyDeviceToDevice, st));
+    BOA_CUDA(cudaMemcpyAsync(ix->pq_pivots, pivots, pb, cudaMemcpyDeviceToDevice, st));
+    BOA_CUDA(cudaStreamSynchronize(st));
+    ix->pq_M = M; ix->pq_K = K;
+    return BOA_OK;
+}
+
+int boa_get_rerank_counts(boa_index* ix, int32_t* n_rerank, void* stream)
+{
+    if (!ix || !n_rerank) return BOA_EINVAL;
+    if (ix->last_Q == 0) return BOA_OK;
+    BOA_CUDA(cudaMemcpyAsync(n_rerank, ix->stats + (size_t)4 * ix->ws_Q, (size_t)ix->last_Q * sizeof(int32_t),
+                             cudaMemcpyDeviceToDevice, reinterpret_cast<cudaStream_t>(stream)));
     return BOA_OK;
 }
 

@@ -100,6 +100,10 @@ struct SearchParams {
     int nchunks;              // 16-byte chunks of one vector
     uint32_t attr_float_mask; // bit j set: column j is float
     uint32_t entry;
+    // product quantisation (PQ kernels only): D = pq_M * pq_dsub
+    const uint8_t* pq_codes;  // [N][pq_M] centroid index per subspace, rows of pq_M bytes (multiple of 16)
+    const float* pq_pivots;   // [pq_M][pq_K][pq_dsub]
+    int pq_M, pq_K, pq_dsub;
     // batch
     const float* queries;     // [Q][D]
     const int32_t* lo;        // [Q][m]
@@ -144,6 +148,7 @@ struct SearchParams {
     int32_t* n_expand;
     int32_t* n_scored;
     int32_t* flags;
+    int32_t* n_rerank;        // PQ kernels: rows fetched for the final exact ranking
     uint64_t* spill;          // [Q][spill_stride] pools carried between phases (resume)
     int32_t* spill_size;      // [Q]
     int spill_stride;
@@ -329,11 +334,13 @@ __device__ __forceinline__ void sort_keys(uint64_t (&x)[RS], int lane)
 
 // Per-warp shared memory carve-up (bytes), shared by host and device.
 struct WarpSmem {
-    int pool_off, nk_off, cand_off, hash_off, q_off, total;
+    int pool_off, nk_off, cand_off, hash_off, q_off, pq_off, top_off, total;
 };
+constexpr int kPqMaxK = 32;            // largest k of a PQ search: its final ranking keeps k keys per warp
 // q_in_smem: the query vector is kept in shared memory (only when lanes do not hold their
 // slices of it in registers).
-__host__ __device__ inline WarpSmem warp_smem_layout(int C, int table_bytes, int D, int RS, bool q_in_smem)
+__host__ __device__ inline WarpSmem warp_smem_layout(int C, int table_bytes, int D, int RS, bool q_in_smem,
+                                                      int pq_entries = 0)
 {
     WarpSmem s;
     int off = 0;
@@ -342,6 +349,8 @@ __host__ __device__ inline WarpSmem warp_smem_layout(int C, int table_bytes, int
     s.q_off = off;     off += q_in_smem ? ((D * 4 + 15) & ~15) : 0;
     s.hash_off = off;  off += table_bytes;
     s.cand_off = off;  off += 32 * RS * 4;
+    s.pq_off = off;    off += pq_entries * 4;                     // distance table of the query
+    s.top_off = off;   off += pq_entries ? kPqMaxK * 8 : 0;       // best exact keys of the final ranking
     s.total = (off + 127) & ~127;
     return s;
 }
@@ -353,10 +362,15 @@ __host__ __device__ inline WarpSmem warp_smem_layout(int C, int table_bytes, int
 // at most 4 (the lane then keeps its slices of the query in registers and the chunk
 // loop is unrolled); 0 = any length, query slices read from shared memory.  EXACT: the
 // row has exactly 8*CPL chunks, so no lane ever has a chunk missing.
-template <int VT, int RN, int W, int CPL, bool EXACT>
-__global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(const SearchParams p)
+// PQ: the traversal orders by product-quantised distances (a per-query table of
+// subvector-to-centroid distances in shared memory, one look-up per subspace and candidate,
+// a lane per candidate); when a phase has converged the filter-valid beam entries are ranked
+// by exact distance with the same row-scoring code the exact search uses.
+template <int VT, int RN, int W, int CPL, bool EXACT, bool PQ = false>
+__global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_kernel(const SearchParams p)
 {
     static_assert(W == 1 || W == 2, "expansion width 1 or 2");
+    static_assert(!PQ || W == 1, "PQ traversal expands one node per iteration");
     constexpr int RS = RN * W;                      // adjacency slots per lane and iteration
     extern __shared__ __align__(128) uint8_t smem_raw[];
     const int lane = threadIdx.x;
@@ -366,7 +380,9 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
     constexpr int QF4 = (VT == 0) ? 1 : 4;          // float4 slices of the query per chunk
     constexpr int NQ = (CPL > 0) ? CPL * QF4 : 1;
 
-    const WarpSmem lay = warp_smem_layout(p.C, p.table_bytes, p.D, RS, CPL == 0);
+    const WarpSmem lay = warp_smem_layout(p.C, p.table_bytes, p.D, RS, CPL == 0, PQ ? p.pq_M * p.pq_K : 0);
+    float* pq_table = reinterpret_cast<float*>(smem_raw + lay.pq_off);
+    uint64_t* topk = reinterpret_cast<uint64_t*>(smem_raw + lay.top_off);
     uint64_t* pool = reinterpret_cast<uint64_t*>(smem_raw + lay.pool_off);
     uint64_t* nk = reinterpret_cast<uint64_t*>(smem_raw + lay.nk_off);
     uint32_t* cand = reinterpret_cast<uint32_t*>(smem_raw + lay.cand_off);
@@ -455,6 +471,34 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                     qreg[i] = make_float4(__uint_as_float(wq[4 * i + 0]), __uint_as_float(wq[4 * i + 1]),
                                           __uint_as_float(wq[4 * i + 2]), __uint_as_float(wq[4 * i + 3]));
             }
+        }
+
+        if (PQ) {
+            // distance table of this query: entry (m, c) = squared distance between the m-th
+            // subvector of q and centroid c of subspace m, one fused multiply-add per dimension
+            // in ascending order; a lane per entry
+            const int entries = p.pq_M * p.pq_K;
+            const float* qv = p.queries + (size_t)qi * p.D;
+            for (int e = lane; e < entries; e += 32) {
+                const int m = e / p.pq_K;
+                const float* piv = p.pq_pivots + (size_t)e * p.pq_dsub;
+                const float* qm = qv + m * p.pq_dsub;
+                float acc = 0.0f;
+                if ((p.pq_dsub & 3) == 0) {
+                    for (int i = 0; i < p.pq_dsub; i += 4) {
+                        const float4 pv = __ldg(reinterpret_cast<const float4*>(piv + i));
+                        const float4 qq = __ldg(reinterpret_cast<const float4*>(qm + i));
+                        acc = sq_acc4(acc, qq, pv);
+                    }
+                } else {
+                    for (int i = 0; i < p.pq_dsub; ++i) {
+                        const float d = __ldg(qm + i) - __ldg(piv + i);
+                        acc = fmaf(d, d, acc);
+                    }
+                }
+                pq_table[e] = acc;
+            }
+            __syncwarp();
         }
 
         // Scores cand[0..cnt) straight from global memory: eight rows per pass, every lane
@@ -682,6 +726,52 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             __syncwarp();
         };
 
+        // PQ scoring of cand[0..cnt): a lane per candidate.  The lane reads the candidate's
+        // code (pq_M bytes) and attribute cells, counts the violated predicates (the bounds sit
+        // in lanes 0..m-1 and are handed round by shuffles) and adds the pq_M table entries the
+        // code selects, in ascending subspace order -> nk[0..cnt).
+        auto score_pq = [&](int cnt) {
+#pragma unroll
+            for (int s = 0; s < RS; ++s) {
+                const int j = lane + 32 * s;
+                const bool act = j < cnt;
+                const uint32_t id = act ? cand[j] : 0u;
+                uint32_t phi = 0;
+                for (int a = 0; a < p.m; ++a) {
+                    const int32_t l = __shfl_sync(0xffffffffu, my_lo, a);
+                    const int32_t h = __shfl_sync(0xffffffffu, my_hi, a);
+                    const uint32_t cell = ldg_stream32(p.attrs + (size_t)id * p.m + a, act);
+                    bool v;
+                    if ((p.attr_float_mask >> a) & 1u)
+                        v = !(__uint_as_float(cell) >= __int_as_float(l) && __uint_as_float(cell) <= __int_as_float(h));
+                    else
+                        v = (int32_t)cell < l || (int32_t)cell > h;
+                    phi += (act && v) ? 1u : 0u;
+                }
+                float d = 0.0f;
+                const uint8_t* code = p.pq_codes + (size_t)id * p.pq_M;
+                for (int c0 = 0; c0 < p.pq_M; c0 += 16) {
+                    const uint4 cw = ldg_stream128(code + c0, act);
+                    if (act) {
+                        const uint32_t w4[4] = {cw.x, cw.y, cw.z, cw.w};
+#pragma unroll
+                        for (int t = 0; t < 16; ++t) {
+                            const uint32_t c = (w4[t >> 2] >> (8 * (t & 3))) & 0xFFu;
+                            d = d + pq_table[(c0 + t) * p.pq_K + c];
+                        }
+                    }
+                }
+                if (act) nk[j] = fin ? pack_key(true, phi, __fmaf_rn(p.lambda, (float)phi, d), id)
+                                     : pack_key(false, phi, d, id);
+            }
+            __syncwarp();
+        };
+        // the distance the traversal orders by
+        auto score_search = [&](int cnt) {
+            if (PQ) score_pq(cnt);
+            else score(cnt);
+        };
+
         // Returns true when id was not in the table; records it either way.
         auto hash_test_and_set = [&](uint32_t id) -> bool {
             const uint32_t h = (id * 0x9E3779B1u) & id_mask;
@@ -752,7 +842,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
         } else {
             if (lane == 0) cand[0] = p.entry;
             __syncwarp();
-            score(1);
+            score_search(1);
             if (lane == 0) {
                 pool[0] = nk[0];
                 hash_test_and_set(p.entry);
@@ -826,7 +916,7 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
             if (cnt > 0) {
                 n_sc += cnt;
                 // gather + distance + range check (fused)
-                score(cnt);
+                score_search(cnt);
 
                 // new keys that cannot enter a full pool are dropped right away
                 const uint64_t worst = (n == p.C) ? (pool[n - 1] >> 1) : (kKeyMax >> 1);
@@ -1122,7 +1212,57 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
         const int lim = n < p.L ? n : p.L;
         int nv_beam = 0;            // |V|
         float d2k = 0.0f, d2max = 0.0f;     // k-th and last distance of V
-        if (!fin) {
+        int n_rr = 0;               // PQ: rows fetched for the final ranking
+        if (PQ) {
+            // Final ranking by exact distance: the filter-valid beam entries, 32 pool places at a
+            // time, are scored exactly (same code as the exact search) and merged into the 32
+            // best keys found so far, kept sorted in shared memory as (d^2 bits, id).
+            topk[lane] = kKeyMax;
+            uint32_t mx = 0u;                         // largest exact d^2 (its bits) over V
+            __syncwarp();
+            for (int b0 = 0; b0 < lim; b0 += 32) {
+                const int i = b0 + lane;
+                const uint64_t e = (i < lim) ? pool[i] : 0ull;
+                const bool ok = (i < lim) && (key_phi(fin, e) == 0u);
+                const unsigned bal = __ballot_sync(0xffffffffu, ok);
+                const int cntc = __popc(bal);
+                if (cntc == 0) continue;
+                if (ok) cand[__popc(bal & lt_mask)] = key_id(fin, e);
+                __syncwarp();
+                score(cntc);
+                uint64_t x2[2];
+                x2[0] = kKeyMax;
+                if (lane < cntc) {
+                    const uint64_t kx = nk[lane];
+                    const uint32_t bits = __float_as_uint(key_d2(fin, kx));
+                    x2[0] = ((uint64_t)bits << 32) | key_id(fin, kx);
+                    mx = bits > mx ? bits : mx;
+                }
+                x2[1] = topk[lane];
+                __syncwarp();
+                sort_keys<2>(x2, lane);
+                topk[lane] = x2[0];
+                n_rr += cntc;
+                __syncwarp();
+            }
+            mx = __reduce_max_sync(0xffffffffu, mx);
+            nv_beam = n_rr;
+            for (int i = lane; i < p.k; i += 32) {
+                uint32_t id = kNoId;
+                float d2 = __int_as_float(0x7f800000);
+                if (i < n_rr && i < kPqMaxK) {
+                    const uint64_t kx = topk[i];
+                    id = (uint32_t)kx;
+                    d2 = __uint_as_float((uint32_t)(kx >> 32));
+                }
+                p.out_ids[(size_t)qi * p.k + i] = id;
+                p.out_d2[(size_t)qi * p.k + i] = d2;
+            }
+            if (nv_beam > p.k) {
+                d2k = __uint_as_float((uint32_t)(topk[p.k - 1] >> 32));
+                d2max = __uint_as_float(mx);
+            }
+        } else if (!fin) {
             // valid entries sort first
             for (int b0 = 0; b0 < lim; b0 += 32) {
                 const int i = b0 + lane;
@@ -1185,10 +1325,12 @@ __global__ void __launch_bounds__(kThreads, BOA_MIN_CTAS) boa_search_kernel(cons
                 p.n_expand[qi] = n_exp;
                 p.n_scored[qi] = n_sc;
                 p.flags[qi] = capped ? 1 : 0;
+                p.n_rerank[qi] = n_rr;
             } else {
                 p.n_expand[qi] += n_exp;
                 p.n_scored[qi] += n_sc;
                 if (capped) p.flags[qi] |= 1;
+                if (PQ) p.n_rerank[qi] += n_rr;
             }
         }
         if (uncertain && !p.last_phase) {

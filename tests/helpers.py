@@ -30,7 +30,7 @@ def make_pair(d, entry=-1):
 
 
 def gpu_search(gpu, g, k, widths, mode="restart", eps=0.05, tau=0.0, plus_k=0, cap=(8, 64),
-               sel=None, expand_w=1, lam=float("inf")):
+               sel=None, expand_w=1, lam=float("inf"), pq=False):
     gpu.set_param("mode", 1 if mode == "resume" else 0)
     gpu.set_param("eps", eps)
     gpu.set_param("tau", tau)
@@ -39,6 +39,7 @@ def gpu_search(gpu, g, k, widths, mode="restart", eps=0.05, tau=0.0, plus_k=0, c
     gpu.set_param("cap_add", cap[1])
     gpu.set_param("expand_w", expand_w)
     gpu.set_param("lam", lam)
+    gpu.set_param("pq", 1 if pq else 0)
     gpu.set_schedule(list(widths))
     q, lo, hi = g["queries"], g["lo"], g["hi"]
     if sel is not None:
