@@ -40,6 +40,7 @@ UNIT = "queries/s"
 # the line reports "traffic": null until the capture is repeated.
 NCU_DRAM_BYTES_PER_SCORED = {
     # workload: (bytes per scored record, sha256[:12] of csrc/boa_search.cuh, summary file)
+    "c2": (410.4, "b5f9ab893803", "profiles/boa_search_kernel_c2_dram_traffic.md"),
 }
 
 # Operating point of each workload: explicit phase widths and eps, chosen from the sweeps in
@@ -48,10 +49,25 @@ NCU_DRAM_BYTES_PER_SCORED = {
 OPERATING = {
     "c1": dict(schedule=[16, 64, 128], eps=0.05, steps=20),    # literal, disconnected graph: parity only
     "c1b": dict(schedule=[16, 128], eps=0.02, steps=20),
-    "c2": dict(schedule=[16, 512], eps=0.03, steps=20),
-    "c3": dict(schedule=[16, 512], eps=0.03, steps=10),
-    "c4": dict(schedule=[32, 512], eps=0.05, steps=10),
+    "c2": dict(schedule=[16, 80], eps=0.02, steps=20),
+    "c3": dict(schedule=[16, 96], eps=0.03, steps=20),
+    "c4": dict(schedule=[32, 96], eps=0.05, steps=20),
     "c5": dict(schedule=[16, 512], eps=0.03, steps=4),
+}
+# The schedule that runs each configuration's own L0 -> Lmax = 512 (most queries end at 512:
+# the wide-beam regime, where one query expands about 500 nodes).
+WIDE = {"c2": dict(schedule=[16, 512], eps=0.03), "c3": dict(schedule=[16, 512], eps=0.03),
+        "c4": dict(schedule=[32, 512], eps=0.05)}
+
+
+# What per_config measures beside each workload's operating point: the wide schedule for
+# c2-c4, the configuration's own fixed beamwidth of 500 for c5, and for c5 the same two runs
+# with PQ traversal (48 subspaces of 20 dimensions, 64 centroids each; exact final ranking).
+PER_CONFIG_VARIANTS = {
+    "c2": (dict(WIDE["c2"], tag="wide"),),
+    "c3": ({}, dict(WIDE["c3"], tag="wide")),
+    "c4": ({}, dict(WIDE["c4"], tag="wide")),
+    "c5": ({}, {"fixed_L": 500}, {"pq": "48,64"}, {"pq": "48,64", "fixed_L": 500}),
 }
 
 
@@ -85,6 +101,8 @@ def parse_args():
     ap.add_argument("--max-warps", type=int, default=0)
     ap.add_argument("--fixed-L", type=int, default=0,
                     help="the paper's Fixed-L baseline: one phase at this beamwidth for every query")
+    ap.add_argument("--pq", default="", help="M[,K]: traverse on product-quantised distances with a codebook "
+                    "of M subspaces and K centroids (default 256) trained on the fixture; exact final ranking")
     ap.add_argument("--no-extras", action="store_true", help="debug: skip recall/e2e/cpu legs")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--seed", type=int, default=0)
@@ -205,14 +223,17 @@ def measured_peak_gbs():
     return 6650.0, "fallback"
 
 
-def algorithmic_bytes(w, st, scored_unique_ratio, mode, widths):
+def algorithmic_bytes(w, st, scored_unique_ratio, mode, widths, pq_M=0, n_rerank=None):
     """Bytes the method must move for one batch: query + bounds, one adjacency row per
     expansion, one record (vector + attribute cells) per neighbour scored for the first
-    time, the outputs, and in resume mode the pool spill and reload of escalated queries."""
+    time, the outputs, and in resume mode the pool spill and reload of escalated queries.
+    With PQ traversal a scored neighbour costs its code (pq_M bytes) and attribute cells, and
+    every row of the final exact ranking one vector; the codebook itself (K*D*4 bytes, read by
+    every query) stays in L2 and is not counted against HBM."""
     sv = 1 if w.vec_dtype == "u8" else 4
     Q = st["n_expand"].shape[0]
     per_query = w.D * 4 + 8 * w.m + 8 * w.k
-    rec = w.D * sv + 4 * w.m
+    rec = (pq_M if pq_M else w.D * sv) + 4 * w.m
     total = Q * per_query
     total += float(st["n_expand"].sum()) * 4 * w.R
     total += float(st["n_scored"].sum()) * scored_unique_ratio * rec
@@ -220,22 +241,44 @@ def algorithmic_bytes(w, st, scored_unique_ratio, mode, widths):
         esc = st["final_L"] > widths[0]
         pool = np.minimum(widths[-1], st["n_scored"][esc] + 1)
         total += float(pool.sum()) * 8 * 2
+    if pq_M and n_rerank is not None:
+        total += float(n_rerank.sum()) * w.D * sv
     return total
+
+
+def parse_pq(args):
+    if not getattr(args, "pq", ""):
+        return 0, 0
+    f = [int(x) for x in str(args.pq).split(",")]
+    return f[0], (f[1] if len(f) > 1 else 256)
+
+
+def codebook(d, args, dev=None):
+    """The fixture's PQ codebook for this run (trained once per process and workload)."""
+    M, K = parse_pq(args)
+    key = ("pq", M, K)
+    if key not in d:
+        from boa_synth.pq import train_pq
+        d[key] = train_pq(d["vectors"], M=M, K=K, iters=6, seed=args.seed, device=dev)
+    return d[key]
 
 
 def run_oracle_sample(w, d, widths, args, seconds, dist_mode=1):
     """The CPU oracle, as it stands, on a leading slice of the batch sized for `seconds`."""
     from oracle.boa_oracle import OracleIndex
     orc = OracleIndex(d["vectors"], d["attrs"], d["attr_types"], d["graph"])
+    if parse_pq(args)[0]:
+        orc.attach_pq(*codebook(d, args))
     probe = min(8, w.Q)
     t0 = time.perf_counter()
+    pq = bool(parse_pq(args)[0])
     orc.search(d["queries"][:probe], d["lo"][:probe], d["hi"][:probe], w.k, widths, eps=args.eps,
-               mode=args.mode, dist_mode=dist_mode, expand_w=args.expand_w, lam=args.lam)
+               mode=args.mode, dist_mode=dist_mode, expand_w=args.expand_w, lam=args.lam, pq=pq)
     per = max((time.perf_counter() - t0) / probe, 1e-6)
     n = int(max(8, min(w.Q, seconds / per)))
     t0 = time.perf_counter()
     o = orc.search(d["queries"][:n], d["lo"][:n], d["hi"][:n], w.k, widths, eps=args.eps,
-                   mode=args.mode, dist_mode=dist_mode, expand_w=args.expand_w, lam=args.lam)
+                   mode=args.mode, dist_mode=dist_mode, expand_w=args.expand_w, lam=args.lam, pq=pq)
     dt = time.perf_counter() - t0
     return orc, o, n, dt
 
@@ -252,10 +295,13 @@ def reference_arm(args):
     per_step = max(2.0, min(10.0, 150.0 / max(1, args.steps + args.warmup)))
     from oracle.boa_oracle import OracleIndex
     orc = OracleIndex(d["vectors"], d["attrs"], d["attr_types"], d["graph"])
+    pq = bool(parse_pq(args)[0])
+    if pq:
+        orc.attach_pq(*codebook(d, args, "cpu"))
     probe = min(8, w.Q)
     t0 = time.perf_counter()
     orc.search(d["queries"][:probe], d["lo"][:probe], d["hi"][:probe], w.k, widths, eps=args.eps,
-               mode=args.mode, dist_mode=1, expand_w=args.expand_w, lam=args.lam)
+               mode=args.mode, dist_mode=1, expand_w=args.expand_w, lam=args.lam, pq=pq)
     per = max((time.perf_counter() - t0) / probe, 1e-6)
     n = int(max(4, min(w.Q, per_step / per)))
     times = []
@@ -263,7 +309,7 @@ def reference_arm(args):
         a = (s * n) % max(1, w.Q - n + 1)
         t0 = time.perf_counter()
         orc.search(d["queries"][a:a + n], d["lo"][a:a + n], d["hi"][a:a + n], w.k, widths,
-                   eps=args.eps, mode=args.mode, dist_mode=1, expand_w=args.expand_w, lam=args.lam)
+                   eps=args.eps, mode=args.mode, dist_mode=1, expand_w=args.expand_w, lam=args.lam, pq=pq)
         if s >= args.warmup:
             times.append(time.perf_counter() - t0)
     ms = 1e3 * float(np.mean(times))
@@ -284,6 +330,7 @@ def config_dict(w, widths, args):
                         f"L0={w.L0} Lmax={w.Lmax}",
             "schedule": widths, "eps": args.eps, "mode": args.mode, "plus_k": args.plus_k,
             "expand_w": args.expand_w, "lambda": "inf" if np.isinf(args.lam) else args.lam,
+            "pq": (dict(zip(("M", "K"), parse_pq(args))) if parse_pq(args)[0] else None),
             "selectivity": f"{w.sel_kind} {w.sel_lo}-{w.sel_hi}", "seed": args.seed,
             "l2": "inputs larger than L2: records + graph are read by random access from a "
                   "working set far above 126 MB; no flush between steps"}
@@ -295,7 +342,14 @@ def to_device(d, dev):
             for k, v in d.items() if k in ("vectors", "attrs", "graph", "queries", "lo", "hi")}
 
 
-def configure(ix, args, widths):
+def configure(ix, args, widths, d=None):
+    if parse_pq(args)[0] and d is not None:
+        import torch
+        if ("attached",) + parse_pq(args) not in d:
+            piv, codes = codebook(d, args, str(ix.device))
+            ix.attach_pq(torch.from_numpy(piv).to(ix.device), torch.from_numpy(codes).to(ix.device))
+            d[("attached",) + parse_pq(args)] = True
+    ix.set_param("pq", 1 if parse_pq(args)[0] else 0)
     ix.set_param("mode", 1 if args.mode == "resume" else 0)
     ix.set_param("eps", args.eps)
     ix.set_param("plus_k", args.plus_k)
@@ -344,9 +398,10 @@ def quality(w, d, t, ix, args, widths, ids_np, d2_np, st, gt_queries, cpu_second
                 cpu_qps=n_s / dt_s, cpu_n=n_s, cpu_dt=dt_s)
 
 
-def measure_config(name, args, dev, steps, cpu_seconds, fixed_widths=(), gt_queries=10_000):
-    """One workload at its operating point, then at each fixed beamwidth asked for, on one
-    build of its inputs: the entries of per_config (keys name, name_fixed<L>)."""
+def measure_config(name, args, dev, steps, cpu_seconds, variants=({},), gt_queries=10_000):
+    """One workload at its operating point and in every variant asked for (fixed beamwidth,
+    PQ traversal), on one build of its inputs: the entries of per_config (keys name,
+    name_fixed<L>, name_pq<M>, name_pq<M>_fixed<L>)."""
     import copy
     import torch
     from boa_synth import ALL, make_workload
@@ -361,22 +416,29 @@ def measure_config(name, args, dev, steps, cpu_seconds, fixed_widths=(), gt_quer
     out_d2 = torch.empty((w.Q, w.k), dtype=torch.float32, device=dev)
     peak, peak_kind = measured_peak_gbs()
     res = {}
-    for fixed_L in (0,) + tuple(fixed_widths):
+    for var in variants:
+        fixed_L, pq = var.get("fixed_L", 0), var.get("pq", "")
         a = copy.copy(args)
-        a.workload, a.scale_n, a.queries, a.schedule, a.fixed_L = name, 0, 0, "", fixed_L
-        a.eps = OPERATING[name]["eps"]
+        a.workload, a.scale_n, a.queries, a.schedule, a.fixed_L, a.pq = name, 0, 0, "", fixed_L, pq
+        a.eps = var.get("eps", OPERATING[name]["eps"])
         a.plus_k, a.expand_w, a.lam, a.table_kb, a.table_tags, a.max_warps = 0, 1, float("inf"), 0, 0, 0
-        widths = schedule_of(a, w)
-        configure(ix, a, widths)
+        widths = var.get("schedule") or schedule_of(a, w)
+        configure(ix, a, widths, d)
         n_steps = steps if not fixed_L else max(3, steps // 2)
         total_ms, step_ms = timed_steps(ix, t, w.k, widths, out_ids, out_d2, n_steps, 3, torch.cuda.synchronize)
         st = {kk: v.cpu().numpy() for kk, v in ix.stats().items()}
         counts = ix.phase_counts()
         ids_np, d2_np = out_ids.cpu().numpy().view(np.uint32), out_d2.cpu().numpy()
         ql = quality(w, d, t, ix, a, widths, ids_np, d2_np, st, gt_queries, cpu_seconds)
-        alg = algorithmic_bytes(w, st, ql["unique_ratio"], a.mode, widths)
+        pq_M = parse_pq(a)[0]
+        n_rr = ix.rerank_counts().cpu().numpy() if pq_M else None
+        alg = algorithmic_bytes(w, st, ql["unique_ratio"], a.mode, widths, pq_M, n_rr)
         ms = total_ms / n_steps
-        res[name if not fixed_L else f"{name}_fixed{fixed_L}"] = {
+        key = name + (f"_pq{pq_M}" if pq_M else "") + (f"_fixed{fixed_L}" if fixed_L else "") + \
+            (f"_{var['tag']}" if var.get("tag") else "")
+        res[key] = {
+            "pq": config_dict(w, widths, a)["pq"],
+            "mean_rows_reranked": float(n_rr.mean()) if pq_M else None,
             "workload": config_dict(w, widths, a)["workload"], "schedule": widths, "eps": a.eps, "mode": a.mode,
             "steps": n_steps, "ms_per_step": ms, "queries_per_s": w.Q / (ms / 1e3),
             "recall_at_10": ql["recall"], "recall_queries": ql["recall_queries"],
@@ -419,7 +481,7 @@ def main():
     d = make_workload(w, seed=args.seed, device=str(dev))
     t = to_device(d, dev)
     ix = BoaIndex(t["vectors"], t["attrs"], d["attr_types"].tolist(), t["graph"])
-    configure(ix, args, widths)
+    configure(ix, args, widths, d)
     Q, k = w.Q, w.k
     out_ids = torch.empty((Q, k), dtype=torch.int32, device=dev)
     out_d2 = torch.empty((Q, k), dtype=torch.float32, device=dev)
@@ -498,12 +560,15 @@ def main():
 
     # ---- roofline of the search kernel (HBM-bound random gather)
     peak, peak_kind = measured_peak_gbs()
-    alg_bytes = algorithmic_bytes(w, st, ql["unique_ratio"], args.mode, widths)
+    pq_M = parse_pq(args)[0]
+    alg_bytes = algorithmic_bytes(w, st, ql["unique_ratio"], args.mode, widths, pq_M,
+                                  ix.rerank_counts().cpu().numpy() if pq_M else None)
     kernel_ms = float(np.mean(step_ms))
     achieved = alg_bytes / (kernel_ms / 1e3) / 1e9
     traffic, traffic_note = None, "no ncu capture on file for this workload and kernel source"
     cap = NCU_DRAM_BYTES_PER_SCORED.get(args.workload)
-    plain = not (args.scale_n or args.table_kb or args.table_tags or args.expand_w != 1 or args.fixed_L)
+    plain = not (args.scale_n or args.table_kb or args.table_tags or args.expand_w != 1 or args.fixed_L
+                 or args.pq)
     if cap and plain and cap[1] == kernel_source_digest() and widths == OPERATING[args.workload]["schedule"]:
         traffic = cap[0] * float(st["n_scored"].sum())
         traffic_note = f"{cap[0]} DRAM bytes per scored record ({cap[2]}) x records scored in this run"
@@ -526,7 +591,7 @@ def main():
             if r >= 0.95:
                 fixed_same = {"L": L, "recall_at_10": r, "ms_per_step": tot / 5, "queries_per_s": Q / (tot / 5 / 1e3)}
                 break
-        configure(ix, args, widths)
+        configure(ix, args, widths, d)
         del gt_ids, gt_d2, gt_nv
 
     line = {
@@ -559,10 +624,10 @@ def main():
     # ---- the other configurations, one GPU only
     if world == 1 and plain and not args.no_per_config and args.workload == "c2":
         per = {}
-        for name in ("c1", "c1b", "c3", "c4", "c5"):
+        for name in ("c1", "c1b", "c2", "c3", "c4", "c5"):
             try:
                 per.update(measure_config(name, args, dev, OPERATING[name]["steps"], 3.0,
-                                          fixed_widths=(500,) if name == "c5" else ()))
+                                          variants=PER_CONFIG_VARIANTS.get(name, ({},))))
             except Exception as e:           # one workload failing must not lose the line
                 per[name] = {"error": f"{type(e).__name__}: {e}"}
         line["per_config"] = per

@@ -56,9 +56,12 @@ def full():
     return C2, d, orc, gpu, g
 
 
-def test_full_size_bench_configuration(full):
+@pytest.mark.parametrize("which", ["operating point", "wide"])
+def test_full_size_bench_configuration(full, which):
+    import bench
     w, d, orc, gpu, g = full
-    widths, eps = [16, 512], 0.03
+    op = bench.OPERATING["c2"] if which == "operating point" else bench.WIDE["c2"]
+    widths, eps = list(op["schedule"]), op["eps"]
     r = gpu_search(gpu, g, w.k, widths, mode="resume", eps=eps)
     assert gpu.device_status() == 0
     Q = w.Q
@@ -88,7 +91,7 @@ def test_full_size_bench_configuration(full):
     srt = np.sort(np.where(found, ids, np.arange(w.k, dtype=np.uint32)[None, :] + 0xF0000000), axis=1)
     assert (srt[:, :-1] != srt[:, 1:]).all()
     assert set(np.unique(r["final_L"]).tolist()) <= set(widths)
-    assert r["phase_active"][0] == Q and r["phase_active"][1] == int((r["final_L"] == 512).sum())
+    assert r["phase_active"][0] == Q and r["phase_active"][1] == int((r["final_L"] == widths[-1]).sum())
     # --- recall: harness ground truth vs the oracle's brute force, and the >= 0.95 bar
     gt_ids, gt_d2, gt_nv = filtered_topk(g["vectors"], g["attrs"], d["attr_types"], g["queries"],
                                          g["lo"], g["hi"], w.k)
@@ -150,6 +153,15 @@ def test_full_size_float_workload_c3():
                                          g["lo"], g["hi"], w.k)
     rec = recall_against(r["ids"], r["d2"], gt_d2.cpu().numpy(), gt_nv.cpu().numpy(), w.k)
     assert np.nanmean(rec) >= 0.95
+    # the benchmark's operating point on this workload
+    import bench
+    op = bench.OPERATING["c3"]
+    r2 = gpu_search(gpu, g, w.k, op["schedule"], mode="resume", eps=op["eps"])
+    o2 = orc.search(d["queries"][sample], d["lo"][sample], d["hi"][sample], w.k, op["schedule"], eps=op["eps"],
+                    mode="resume", dist_mode=1)
+    _assert_sample_bit_parity(o2, r2, sample)
+    _check_properties(w, d, r2, op["schedule"], w.Q)
+    assert np.nanmean(recall_against(r2["ids"], r2["d2"], gt_d2.cpu().numpy(), gt_nv.cpu().numpy(), w.k)) >= 0.95
     gpu.close()
 
 
@@ -185,6 +197,15 @@ def test_full_size_scale_workload_c4():
     rec_o = recall_against(o["ids"], o["d2"], gt_d2[sample], gt_nv[sample], w.k)
     assert abs(np.nanmean(rec[sample]) - np.nanmean(rec_o)) <= 0.001
     assert np.nanmean(rec) >= 0.95
+    # the benchmark's operating point on this workload
+    import bench
+    op = bench.OPERATING["c4"]
+    r2 = gpu_search(gpu, g, w.k, op["schedule"], mode="resume", eps=op["eps"])
+    o2 = orc.search(d["queries"][sample], d["lo"][sample], d["hi"][sample], w.k, op["schedule"], eps=op["eps"],
+                    mode="resume", dist_mode=1)
+    _assert_sample_bit_parity(o2, r2, sample)
+    _check_properties(w, d, r2, op["schedule"], w.Q)
+    assert np.nanmean(recall_against(r2["ids"], r2["d2"], gt_d2, gt_nv, w.k)) >= 0.95
     # restart mode and the overlapped schedule on the same index
     sel = torch.from_numpy(sample[:32].astype(np.int64)).to("cuda:0")
     rr = gpu_search(gpu, g, w.k, [32, 128], mode="restart", eps=eps, sel=sel)
