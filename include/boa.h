@@ -49,12 +49,9 @@ enum {
     BOA_PARAM_MODE = 3,     /* 0 = restart every phase from the entry point (Algorithm 1 as
                                printed), 1 = resume: later phases continue from the pool the
                                earlier ones built (the "redundancy avoidance" paragraph)      */
-    BOA_PARAM_PLUS_K = 4,   /* 0 or 1 = BOA; K >= 2 = BOA+: phases overlap ("Pipelining Multiple
-                               Batches").  In resume mode this is one persistent launch whose
-                               warps take narrow work first and escalated queries as soon as
-                               they appear (K itself is not used); in restart mode the first
-                               phase is issued as K sub-batches and pooled wider launches
-                               overlap them on a second stream.  Same results as BOA.         */
+    BOA_PARAM_PLUS_K = 4,   /* 0 or 1 = BOA; K >= 2 = BOA+: the first phase is issued as K
+                               sub-batches and wider phases overlap them ("Pipelining
+                               Multiple Batches")                                            */
     BOA_PARAM_CAP_MULT = 5, /* a phase at width L gives up after CAP_MULT*L + CAP_ADD        */
     BOA_PARAM_CAP_ADD = 6,  /*   expansions; defaults 8 and 64                               */
     BOA_PARAM_TABLE_KB = 7, /* 0 = default (6 or 4, whichever keeps 20 query warps per SM
@@ -79,11 +76,6 @@ enum {
                                multiply-add), ties by id.  Answers are filter-valid either
                                way; a finite lambda lets invalid nodes push valid ones out
                                of the pool.                                                  */
-    BOA_PARAM_IDLE_POLLS = 13, /* BOA+ in resume mode: how often a warp that finds no work looks
-                               again (256 ns apart) before it leaves the persistent launch;
-                               default 65536.  What such warps leave is finished by the
-                               follow-up launches of the same call, so results never depend
-                               on it; 0 makes every idle warp leave at once.                   */
     BOA_PARAM_PQ = 12,      /* 1 = traverse on product-quantised distances (needs
                                boa_index_attach_pq) and rank the filter-valid beam entries by
                                exact distance when a phase has converged: Algorithm 2's PQDist
@@ -240,12 +232,10 @@ int boa_workspace_bytes(const boa_index* index, int64_t Q, int Lmax, size_t* byt
 int boa_last_launch_count(const boa_index* index);
 
 /* Device-side status word of the last search on this index (HOST int, synchronises
-   `stream`).  Bit 0 (value 1): a bounded wait ran out and a query's work was dropped, outputs
-   are incomplete (can only be raised by the persistent BOA+ launch, whose warps wait, with a
-   limit, for a list entry whose slot another warp has already reserved).  Bit 1 (value 2):
-   warps of the persistent BOA+ launch left before all work had appeared and the follow-up
-   launches of the same call finished it; results are complete.  Every other loop in the
-   kernels is bounded by the expansion cap. */
+   `stream`): 0 = fine.  The search kernel has no wait on a flag, barrier or peer and
+   every loop in it is bounded by the expansion cap, so no bit is raised today; the word
+   is where a kernel that has to give up would say so (bit 0 is reserved for "a wait
+   timed out, outputs of the affected launches are incomplete"). */
 int boa_device_status(boa_index* index, int* status, void* stream);
 
 /* cudaError_t of the most recent failing CUDA call made by this library (0 if none). */

@@ -178,7 +178,6 @@ struct boa_index {
     double eps = 0.05, growth = 4.0, tau = 0.0;
     int mode = 0, plus_k = 0, cap_mult = 8, cap_add = 64, table_kb = 0, max_ctas = 0, expand_w = 1, table_tags = 0;
     double lambda = INFINITY;          // weight of the filter penalty; infinity = lexicographic keys
-    int idle_polls = 1 << 16;          // fused BOA+: looks of an idle warp before it leaves (256 ns apart)
     int n_sched = 0;
     int sched[BOA_MAX_PHASES] = {0};
     // scratch
@@ -202,9 +201,7 @@ namespace {
 // layout of boa_index::counters (uint32 words)
 constexpr int kCntCount = 0;                          // [P+1] survivors entering phase p (p>=1)
 constexpr int kCntCount2 = 16;                        // [P+1] the same for the second pool of BOA+ (p>=2)
-constexpr int kCntSnap = 32;                          // [2] frozen end of phase 1's list, per pool of BOA+
-constexpr int kCntFusedTicket = 34;                   // [P+1] entries claimed per class of a fused launch
-constexpr int kCntDone = 44;                          // queries a fused launch has ended
+constexpr int kCntSnap = 32;                          // [pool] frozen end of phase 1's list
 constexpr int kCntStatus = 47;                        // device status bits
 constexpr int kCntTicket = 48;                        // one per launch
 constexpr int kMaxLaunches = 128;
@@ -645,9 +642,6 @@ int boa_set_param(boa_index* ix, int key, double v)
         case BOA_PARAM_EXPAND_W:
             if (v != 1.0 && v != 2.0) return BOA_EINVAL;
             ix->expand_w = (int)v; return BOA_OK;
-        case BOA_PARAM_IDLE_POLLS:
-            if (v < 0.0 || v > 16777216.0 || v != floor(v)) return BOA_EINVAL;
-            ix->idle_polls = (int)v; return BOA_OK;
         case BOA_PARAM_PQ:
             if ((v != 0.0 && v != 1.0) || (v == 1.0 && !ix->pq_codes)) return BOA_EINVAL;
             ix->use_pq = (int)v; return BOA_OK;
@@ -756,55 +750,6 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
         if (rc != BOA_OK) return rc;
         for (int p = 1; p < lp.n_phases; ++p) {
             rc = launch_phase(lp, p, st, nullptr, cnt + p, 0u, 0u, (uint32_t)Q);
-            if (rc != BOA_OK) return rc;
-        }
-    } else if (ix->mode == 1) {
-        // BOA+ in resume mode: one persistent launch in which every phase is a class of work.
-        // Warps take narrow tickets first and survivors of any class as soon as they are
-        // published, so no phase waits for the tail of the one before.  The launches that
-        // follow it on the stream process whatever it left (normally nothing: they find empty
-        // ranges): a warp that finds no work leaves after a bounded number of looks.
-        BOA_CUDA(cudaMemsetAsync(ix->lists, 0xFF, (size_t)lp.n_phases * ix->ws_Q * sizeof(uint32_t), st));
-        boa::SearchParams sp = lp.base;
-        const int Lmax_w = lp.widths[lp.n_phases - 1];
-        sp.fused = 1;
-        sp.n_classes = lp.n_phases;
-        for (int p = 0; p < lp.n_phases; ++p) {
-            sp.cls_L[p] = lp.widths[p];
-            sp.cls_max_expand[p] = ix->cap_mult * lp.widths[p] + ix->cap_add;
-            sp.cls_list[p] = ix->lists + (size_t)p * ix->ws_Q;
-        }
-        sp.cls_count = cnt;
-        sp.cls_ticket = ix->counters + kCntFusedTicket;
-        sp.done_count = ix->counters + kCntDone;
-        sp.idle_polls = ix->idle_polls;
-        sp.L = lp.widths[0];
-        sp.C = Lmax_w;
-        {
-            const TableShape t = choose_table(ix, default_table_kb(ix, lp.kc, sp.C));
-            sp.table_bytes = t.bytes; sp.table_narrow = t.narrow; sp.table_mul3 = t.mul3;
-            sp.id_bits = t.id_bits; sp.low_bits = t.low_bits;
-        }
-        sp.ticket = ix->counters + kCntTicket;
-        const boa::WarpSmem lay = boa::warp_smem_layout(sp.C, sp.table_bytes, ix->D, lp.kc.rs, lp.kc.q_in_smem,
-                                                        ix->use_pq ? ix->pq_M * ix->pq_K : 0);
-        const size_t smem = (size_t)lay.total;
-        if (smem > 48 * 1024)
-            BOA_CUDA(cudaFuncSetAttribute((const void*)lp.kc.fn, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)smem));
-        int per_sm = 0;
-        BOA_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, (const void*)lp.kc.fn,
-                                                               boa::kThreads, smem));
-        if (per_sm < 1) return BOA_EINVAL;
-        if (ix->max_ctas > 0 && per_sm > ix->max_ctas) per_sm = ix->max_ctas;
-        int64_t grid = (int64_t)per_sm * ix->num_sms;
-        if (Q < grid) grid = Q;
-        lp.kc.fn<<<(unsigned)grid, boa::kThreads, smem, st>>>(sp);
-        BOA_CUDA(cudaGetLastError());
-        lp.launches = 1;
-        for (int p = 1; p < lp.n_phases; ++p) {
-            rc = launch_phase(lp, p, st, ix->counters + kCntFusedTicket + p, cnt + p, 0u, 0u,
-                              (uint32_t)(2 * ix->num_sms), 0, false);
             if (rc != BOA_OK) return rc;
         }
     } else {

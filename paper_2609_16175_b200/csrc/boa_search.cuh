@@ -72,16 +72,7 @@ constexpr uint32_t kNoId = 0xFFFFFFFFu;
 constexpr int kThreads = 32;           // one warp per CTA
 constexpr uint64_t kKeyMax = ~0ull;
 
-// Bits of the device status word.  kStatusIncomplete: a bounded wait ran out and a query's
-// work was dropped (outputs incomplete).  kStatusLeftover: warps of a fused launch left before
-// all work had appeared; the follow-up launches of the same call finished it (not an error).
-enum : uint32_t { kStatusIncomplete = 1u, kStatusLeftover = 2u };
-constexpr int kEntryPolls = 1 << 20;           // polls for a list entry whose slot is already reserved
-
-__device__ __forceinline__ uint32_t ld_volatile_u32(const uint32_t* ptr)
-{
-    return *reinterpret_cast<const volatile uint32_t*>(ptr);
-}
+enum : uint32_t { kStatusCopyTimeout = 1u };   // reserved: no wait in the kernel can time out
 
 // Keeps the compiler from moving code across this point.
 #define BOA_SCHED_FENCE() asm volatile("" ::: "memory")
@@ -139,18 +130,6 @@ struct SearchParams {
     double tau_q;             // tau * Q: a phase runs only while |A| > tau*Q
     int fin;                  // 1: keys order by the score d^2 + lambda*phi (finite lambda)
     float lambda;
-    // Fused schedule (BOA+ as one persistent launch): every phase is a class of work the
-    // warps of this launch pull from.  Class 0 is the narrow pass over queries [0, Q); class
-    // c >= 1 reads list cls_list[c], which the epilogues of class c-1 fill.  cls_count[c] =
-    // entries appended to that list so far, cls_ticket[c] = entries claimed so far.
-    int fused;
-    int n_classes;
-    int cls_L[8], cls_max_expand[8];
-    uint32_t* cls_list[8];
-    uint32_t* cls_count;           // [n_classes + 1]
-    uint32_t* cls_ticket;          // [n_classes + 1]; [0] = narrow tickets handed out
-    uint32_t* done_count;          // queries that have ended (confident, or through the last class)
-    int idle_polls;                // a warp without work looks again at most this often, then leaves
     // work list of this launch: positions [begin, end) of in_list (identity when null)
     const uint32_t* in_list;
     const uint32_t* in_begin_ptr;  // device values read at kernel start (null: use constants)
@@ -426,69 +405,11 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
     BOA_T_DECL;
 
     for (;;) {
-        // parameters of the phase this piece of work belongs to
-        int cL = p.L, cMaxExpand = p.max_expand, cls = 0;
-        bool ph_first = p.first_phase != 0, ph_resume = p.resume_in != 0, ph_spill = p.spill_out != 0,
-             ph_last = p.last_phase != 0;
-        uint32_t qi;
-        if (!p.fused) {
-            uint32_t t = 0;
-            if (lane == 0) t = atomicAdd(p.ticket, 1u);
-            t = __shfl_sync(0xffffffffu, t, 0);
-            if (t >= n_work) break;
-            qi = p.in_list ? p.in_list[w_begin + t] : (w_begin + t);
-        } else {
-            // Fused schedule: narrow tickets first, then the widest class that has unclaimed
-            // entries.  A warp that finds nothing looks again a bounded number of times (other
-            // warps may still be producing survivors), then leaves; the follow-up launches of
-            // the same call pick up what is left.
-            uint32_t item = 0;
-            cls = -1;
-            if (lane == 0) {
-                int polls = 0;
-                for (;;) {
-                    if (ld_volatile_u32(p.cls_ticket) < (uint32_t)p.Q) {
-                        const uint32_t t = atomicAdd(p.cls_ticket, 1u);
-                        if (t < (uint32_t)p.Q) { cls = 0; item = t; break; }
-                    }
-                    for (int c = p.n_classes - 1; c >= 1 && cls < 0; --c) {
-                        uint32_t t = ld_volatile_u32(p.cls_ticket + c);
-                        while (t < ld_volatile_u32(p.cls_count + c)) {
-                            const uint32_t old = atomicCAS(p.cls_ticket + c, t, t + 1u);
-                            if (old == t) { cls = c; item = t; break; }
-                            t = old;
-                        }
-                    }
-                    if (cls >= 0) break;
-                    if (ld_volatile_u32(p.done_count) >= (uint32_t)p.Q) break;        // all queries have ended
-                    if (polls++ >= p.idle_polls) { atomicOr(p.status, kStatusLeftover); break; }
-                    __nanosleep(256);
-                }
-                if (cls > 0) {
-                    // the slot is reserved; its writer stores the query index a few instructions later
-                    uint32_t v = kNoId;
-                    for (int spin = 0; spin < kEntryPolls; ++spin) {
-                        v = ld_volatile_u32(p.cls_list[cls] + item);
-                        if (v != kNoId) break;
-                        __nanosleep(64);
-                    }
-                    if (v == kNoId) { atomicOr(p.status, kStatusIncomplete); cls = -2; }
-                    item = v;
-                    __threadfence();          // the writer's spilled pool is visible after its entry
-                }
-            }
-            cls = __shfl_sync(0xffffffffu, cls, 0);
-            item = __shfl_sync(0xffffffffu, item, 0);
-            if (cls == -1) break;
-            if (cls == -2) continue;           // entry never appeared: reported, skipped
-            qi = item;
-            cL = p.cls_L[cls];
-            cMaxExpand = p.cls_max_expand[cls];
-            ph_first = cls == 0;
-            ph_resume = cls > 0;
-            ph_last = cls == p.n_classes - 1;
-            ph_spill = !ph_last;
-        }
+        uint32_t t = 0;
+        if (lane == 0) t = atomicAdd(p.ticket, 1u);
+        t = __shfl_sync(0xffffffffu, t, 0);
+        if (t >= n_work) break;
+        const uint32_t qi = p.in_list ? p.in_list[w_begin + t] : (w_begin + t);
 
         // ---- load the query, its bounds; clear the table of scored ids
         {
@@ -909,13 +830,11 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
         int cur = 0;           // every entry before cur is expanded
         int n_exp = 0, n_sc = 0;
         bool capped = false;
-        if (ph_resume) {
-            // read through L2: in a fused launch the pool was written by another SM of the same
-            // launch, and this SM's L1 may hold an older copy of the line
-            n = __ldcg(p.spill_size + qi);
+        if (p.resume_in) {
+            n = p.spill_size[qi];
             const uint64_t* src = p.spill + (size_t)qi * p.spill_stride;
             for (int i = lane; i < n; i += 32) {
-                const uint64_t e = __ldcg(src + i);
+                const uint64_t e = src[i];
                 pool[i] = e;
                 hash_test_and_set(key_id(fin, e));
             }
@@ -934,17 +853,17 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
 
         // ---- Algorithm 2 main loop
         BOA_T_MARK(0);
-        int pos = first_unexpanded(0, n < cL ? n : cL);
+        int pos = first_unexpanded(0, n < p.L ? n : p.L);
         int pos2 = -1;                 // W == 2: the second node of this iteration, or -1
         uint32_t nb[RS];
         bool have_row = false;         // nb[] already holds the adjacency rows of this iteration
         for (;;) {
             if (pos < 0) break;                                   // converged
-            if (n_exp >= cMaxExpand) { capped = true; break; }
+            if (n_exp >= p.max_expand) { capped = true; break; }
             if (!have_row) {
                 load_row_ids(key_id(fin, pool[pos]), nb, 0);
                 if (W > 1) {
-                    pos2 = (n_exp + 1 < cMaxExpand) ? first_unexpanded(pos + 1, n < cL ? n : cL) : -1;
+                    pos2 = (n_exp + 1 < p.max_expand) ? first_unexpanded(pos + 1, n < p.L ? n : p.L) : -1;
                     load_row_ids(pos2 >= 0 ? key_id(fin, pool[pos2]) : kNoId, nb, RN);
                 }
             }
@@ -965,7 +884,7 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
             int pred_pos = -1;
             uint32_t nbp[RS];
             if (PRED) {
-                pred_pos = first_unexpanded(cur, n < cL ? n : cL);
+                pred_pos = first_unexpanded(cur, n < p.L ? n : p.L);
                 load_row_ids(pred_pos >= 0 ? key_id(fin, pool[pred_pos]) : kNoId, nbp, 0);
             }
             BOA_T_MARK(1);
@@ -1131,7 +1050,7 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
                     for (int s = 0; s < RS; ++s) nb[s] = nbp[s];
                     have_row = pos >= 0;
                 } else {
-                    pos = first_unexpanded(cur, n < cL ? n : cL);
+                    pos = first_unexpanded(cur, n < p.L ? n : p.L);
                 }
                 continue;
             }
@@ -1150,7 +1069,7 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
             // ---- which node is expanded next?  Decide on the pool as it is, translate the
             // position, and start loading that node's adjacency row before the merge.
             {
-                const int lim_old = n < cL ? n : cL;
+                const int lim_old = n < p.L ? n : p.L;
                 const int pos_old = PRED ? pred_pos : first_unexpanded(cur, lim_old);
                 int pos_old_new = -1;
                 if (pos_old >= 0) {
@@ -1161,7 +1080,7 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
                     pos_old_new = pos_old + sh;
                 }
                 const int n_new = (n + kept < p.C) ? n + kept : p.C;
-                const int lim_new = n_new < cL ? n_new : cL;
+                const int lim_new = n_new < p.L ? n_new : p.L;
                 if (W == 1) {
                     int next_pos;
                     const bool new_first = pos_old_new < 0 || rmin < pos_old_new;
@@ -1169,7 +1088,7 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
                     else next_pos = pos_old_new;
                     if (next_pos >= lim_new) next_pos = -1;
                     pos = next_pos;
-                    if (pos >= 0 && n_exp < cMaxExpand) {
+                    if (pos >= 0 && n_exp < p.max_expand) {
                         if (new_first || !PRED) {
                             load_row_ids(key_id(fin, new_first ? first_new : pool[pos_old]), nb, 0);
                         } else {
@@ -1224,10 +1143,10 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
                         if (a0 < b1) { p2 = a0; id2 = a0id; } else { p2 = b1; id2 = b1id; }
                     }
                     if (p1 >= lim_new) p1 = -1;
-                    if (p1 < 0 || p2 >= lim_new || !(n_exp + 1 < cMaxExpand)) p2 = -1;
+                    if (p1 < 0 || p2 >= lim_new || !(n_exp + 1 < p.max_expand)) p2 = -1;
                     pos = p1;
                     pos2 = p2;
-                    if (pos >= 0 && n_exp < cMaxExpand) {
+                    if (pos >= 0 && n_exp < p.max_expand) {
                         load_row_ids(id1, nb, 0);
                         load_row_ids(pos2 >= 0 ? id2 : kNoId, nb, RN);
                         have_row = true;
@@ -1290,7 +1209,7 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
             BOA_T_MARK(9);
         }
         // ---- result: the k nearest filter-valid entries; V = the valid ones among the first L
-        const int lim = n < cL ? n : cL;
+        const int lim = n < p.L ? n : p.L;
         int nv_beam = 0;            // |V|
         float d2k = 0.0f, d2max = 0.0f;     // k-th and last distance of V
         int n_rr = 0;               // PQ: rows fetched for the final ranking
@@ -1401,40 +1320,29 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
             else uncertain = !(d2k >= p.c_eps * d2max);
         }
         if (lane == 0) {
-            p.final_L[qi] = cL;
-            if (ph_first) {
+            p.final_L[qi] = p.L;
+            if (p.first_phase) {
                 p.n_expand[qi] = n_exp;
                 p.n_scored[qi] = n_sc;
                 p.flags[qi] = capped ? 1 : 0;
                 p.n_rerank[qi] = n_rr;
             } else {
-                // atomics: they act in L2, whichever SM ran the earlier phases of this query
-                atomicAdd(p.n_expand + qi, n_exp);
-                atomicAdd(p.n_scored + qi, n_sc);
-                if (capped) atomicOr(p.flags + qi, 1);
-                if (PQ) atomicAdd(p.n_rerank + qi, n_rr);
+                p.n_expand[qi] += n_exp;
+                p.n_scored[qi] += n_sc;
+                if (capped) p.flags[qi] |= 1;
+                if (PQ) p.n_rerank[qi] += n_rr;
             }
         }
-        if (uncertain && !ph_last) {
-            if (ph_spill) {
+        if (uncertain && !p.last_phase) {
+            if (p.spill_out) {
                 uint64_t* dst = p.spill + (size_t)qi * p.spill_stride;
                 for (int i = lane; i < n; i += 32) dst[i] = pool[i];
                 if (lane == 0) p.spill_size[qi] = n;
             }
-            if (p.fused) {
-                // pool first, then the entry that tells a consumer it is there
-                __threadfence();
-                __syncwarp();
-                if (lane == 0) {
-                    const uint32_t slot = atomicAdd(p.cls_count + cls + 1, 1u);
-                    *reinterpret_cast<volatile uint32_t*>(p.cls_list[cls + 1] + slot) = qi;
-                }
-            } else if (lane == 0) {
+            if (lane == 0) {
                 const uint32_t slot = atomicAdd(p.out_count, 1u);
                 p.out_list[slot] = qi;
             }
-        } else if (p.fused && lane == 0) {
-            atomicAdd(p.done_count, 1u);
         }
         __syncwarp();
         BOA_T_MARK(10);

@@ -185,29 +185,6 @@ def test_boa_plus_equals_boa(name, plus_k):
         assert (a["phase_active"] == b["phase_active"]).all()
 
 
-def test_boa_plus_persistent_launch_with_impatient_warps():
-    """BOA+ in resume mode is one persistent launch; warps that find no work leave after a
-    bounded number of looks and the follow-up launches finish what they left.  With the limit
-    at zero every idle warp leaves at once, so a good part of the wider phases runs in the
-    follow-up launches: results must not change, and nothing may be reported as dropped."""
-    for name, widths in (("c2", [16, 64, 256]), ("c4", [32, 128]), ("c3", [16, 32, 64, 200])):
-        w, d, orc, gpu, g = _get(name)
-        o = orc.search(d["queries"], d["lo"], d["hi"], w.k, widths, eps=0.05, mode="resume", dist_mode=1)
-        for polls in (0, 3, 1 << 16):
-            gpu.set_param("idle_polls", polls)
-            r = gpu_search(gpu, g, w.k, widths, mode="resume", eps=0.05, plus_k=4)
-            assert_bit_parity(o, r, f"persistent BOA+ {name} polls={polls}")
-            assert gpu.device_status() & 1 == 0
-            assert gpu.last_launch_count == len(widths)
-        gpu.set_param("idle_polls", 1 << 16)
-        # a batch smaller than the grid, and one query
-        for nq in (1, 37):
-            r = gpu_search(gpu, g, w.k, widths, mode="resume", eps=0.05, plus_k=2, sel=slice(0, nq))
-            o1 = orc.search(d["queries"][:nq], d["lo"][:nq], d["hi"][:nq], w.k, widths, eps=0.05, mode="resume",
-                            dist_mode=1)
-            assert_bit_parity(o1, r, f"persistent BOA+ {name} Q={nq}")
-
-
 def test_fixed_width_500_not_a_power_of_two():
     w, d, orc, gpu, g = _get("c2")
     o = orc.search(d["queries"][:80], d["lo"][:80], d["hi"][:80], w.k, [500], dist_mode=1)
