@@ -14,6 +14,8 @@
  *   orc_beam_*         filter-aware beam search at one beamwidth (Algorithm 2),
  *                      with exact L2 distances instead of PQ look-ups
  *   orc_uncertain      confidence test gamma(D_i) <= eps (Eq. 3)
+ *   orc_cos_*          cosine distance (Definition 1 allows the Euclidean norm or cosine distance;
+ *                      the paper itself uses the Euclidean norm throughout)
  *   orc_pq_*           product-quantised traversal (Algorithm 2's PQDist line; Section "BOA
  *                      Implementation on a GPU System": the per-query distance table, the
  *                      asymmetric PQ distance as a sum of table look-ups, and the final
@@ -72,6 +74,9 @@ typedef struct {
     const int32_t *attr_types; /* [m]                          */
     const uint32_t *graph;    /* [N][R], ORC_SENTINEL = no edge */
     int64_t entry;
+    /* metric: 0 = squared Euclidean distance, 1 = cosine distance */
+    int metric;
+    float *unit;              /* [N][D] rows scaled to unit length (cosine metric, fp32 path) */
     /* product quantisation (optional): D = pq_M * dsub */
     int pq_M, pq_K;
     const float *pq_pivots;   /* [M][K][dsub] centroids of every subspace */
@@ -136,6 +141,91 @@ static float orc_dist2(const orc_index *ix, const float *q, int64_t p, int dist_
 {
     if (dist_mode == 1) return orc_dist2_lanes(ix, q, p);
     return (float)orc_dist2_f64(ix, q, p);
+}
+
+/* ------------------------------------------------------------------ */
+/* cosine distance                                                     */
+/* ------------------------------------------------------------------ */
+/*
+ * Cosine distance, taken as half the squared Euclidean distance of the two vectors scaled to
+ * unit length: 0.5 * |x/|x| - q/|q||^2 = 1 - cos(x, q) for non-zero vectors (a zero vector
+ * scales to zero).  The norm is the square root of the sum of squares in double, elements in
+ * ascending order.
+ *   mode 0: everything in double, rounded once to float.
+ *   mode 1: the unit vectors are first rounded to float (x_i * (1/|x|) in double, then
+ *           rounded), their squared distance is summed in fp32 in the fixed order of
+ *           orc_dist2_lanes, and halved (exact).
+ */
+static double orc_inv_norm(const float *v, int D)
+{
+    double s = 0.0;
+    for (int i = 0; i < D; ++i) s += (double)v[i] * (double)v[i];
+    return s > 0.0 ? 1.0 / sqrt(s) : 0.0;
+}
+
+/* unit-length copy of v, rounded to float */
+void orc_unit_f32(const float *v, int D, float *out)
+{
+    double inv = orc_inv_norm(v, D);
+    for (int i = 0; i < D; ++i) out[i] = (float)((double)v[i] * inv);
+}
+
+/* fixed-order fp32 squared distance of two float vectors (the order of orc_dist2_lanes) */
+static float orc_lanes_f32(const float *x, const float *q, int D)
+{
+    const int nchunks = (D + 3) / 4;
+    float part[8];
+    for (int g = 0; g < 8; ++g) {
+        float acc = 0.0f;
+        for (int c = g; c < nchunks; c += 8)
+            for (int j = 0; j < 4 && c * 4 + j < D; ++j) {
+                float diff = x[c * 4 + j] - q[c * 4 + j];
+                acc = fmaf(diff, diff, acc);
+            }
+        part[g] = acc;
+    }
+    float a04 = part[0] + part[4], a15 = part[1] + part[5];
+    float a26 = part[2] + part[6], a37 = part[3] + part[7];
+    float e = a04 + a26, o = a15 + a37;
+    return e + o;
+}
+
+/* q is the query as given (not normalised) */
+float orc_cos_dist(const orc_index *ix, const float *q, int64_t p, int dist_mode)
+{
+    const float *x = (const float *)ix->vectors + p * ix->D;
+    if (dist_mode == 1) {
+        float *qh = (float *)malloc((size_t)ix->D * sizeof(float));
+        orc_unit_f32(q, ix->D, qh);
+        float d = 0.5f * orc_lanes_f32(ix->unit + p * ix->D, qh, ix->D);
+        free(qh);
+        return d;
+    }
+    double ix_ = orc_inv_norm(x, ix->D), iq = orc_inv_norm(q, ix->D), s = 0.0;
+    for (int i = 0; i < ix->D; ++i) {
+        double d = (double)x[i] * ix_ - (double)q[i] * iq;
+        s += d * d;
+    }
+    return (float)(0.5 * s);
+}
+
+/* Choose the metric (0 = squared Euclidean, 1 = cosine; float vectors only).  Call once, after
+   orc_create: the entry point stays the medoid of the vectors as given. */
+void orc_set_metric(orc_index *ix, int metric)
+{
+    ix->metric = metric;
+    if (metric == 1 && !ix->unit) {
+        ix->unit = (float *)malloc((size_t)ix->N * ix->D * sizeof(float));
+        for (int64_t p = 0; p < ix->N; ++p)
+            orc_unit_f32((const float *)ix->vectors + p * ix->D, ix->D, ix->unit + p * ix->D);
+    }
+}
+
+/* the distance of the index's metric, exact (not product-quantised) */
+static float orc_metric_dist(const orc_index *ix, const float *q, int64_t p, int dist_mode)
+{
+    if (ix->metric == 1) return orc_cos_dist(ix, q, p, dist_mode);
+    return orc_dist2(ix, q, p, dist_mode);
 }
 
 /* number of violated closed range predicates; bounds use the column's own type */
@@ -248,7 +338,7 @@ orc_index *orc_create(const void *vectors, int vec_dtype, int64_t N, int D,
     if (entry < 0) ix->entry = orc_medoid(ix);
     return ix;
 }
-void orc_destroy(orc_index *ix) { free(ix); }
+void orc_destroy(orc_index *ix) { free(ix->unit); free(ix); }
 int64_t orc_entry(const orc_index *ix) { return ix->entry; }
 
 /* ------------------------------------------------------------------ */
@@ -265,7 +355,7 @@ int64_t orc_bruteforce(const orc_index *ix, const float *q, const int32_t *lo, c
     for (int64_t p = 0; p < ix->N; ++p) {
         if (orc_phi(ix, lo, hi, p) != 0) continue;
         nvalid++;
-        double d = orc_dist2_f64(ix, q, p);
+        double d = ix->metric == 1 ? (double)orc_cos_dist(ix, q, p, 0) : orc_dist2_f64(ix, q, p);
         /* ids ascend, so a strict < keeps the lower id ahead on equal distance */
         int pos = have;
         while (pos > 0 && d < out_d2[pos - 1]) pos--;
@@ -343,6 +433,14 @@ void orc_state_use_pq(orc_state *st, int on, const float *q, int dist_mode)
     if (!on) { free(st->pq_table); st->pq_table = NULL; return; }
     if (!st->pq_table)
         st->pq_table = (float *)malloc((size_t)st->ix->pq_M * st->ix->pq_K * sizeof(float));
+    if (st->ix->metric == 1) {
+        /* cosine metric: the codebook lives in the space of unit-length vectors */
+        float *qh = (float *)malloc((size_t)st->ix->D * sizeof(float));
+        orc_unit_f32(q, st->ix->D, qh);
+        orc_pq_table(st->ix, qh, dist_mode, st->pq_table);
+        free(qh);
+        return;
+    }
     orc_pq_table(st->ix, q, dist_mode, st->pq_table);
 }
 
@@ -350,7 +448,7 @@ void orc_state_use_pq(orc_state *st, int on, const float *q, int dist_mode)
 static float orc_search_dist(const orc_state *st, const float *q, int64_t p, int dist_mode)
 {
     if (st->pq_table) return orc_pq_dist(st->ix, st->pq_table, dist_mode, p);
-    return orc_dist2(st->ix, q, p, dist_mode);
+    return orc_metric_dist(st->ix, q, p, dist_mode);
 }
 
 static void orc_mark_seen(orc_state *st, uint32_t id)
@@ -464,6 +562,17 @@ void orc_state_pool(const orc_state *st, uint32_t *ids, float *d2, int32_t *phi,
  * evaluated without square roots as d2_k >= (1-eps)^2 * d2_max, in fp32, the
  * constant rounded once to float.  Returns 1 when the query must escalate.
  */
+/* metric 0: the distances are squared norms, gamma is defined on the norms (constant (1-eps)^2);
+   metric 1: the distances are cosine distances themselves (constant 1-eps) */
+static int orc_gap_uncertain_m(int nv, int k, float d2k, float d2max, double eps, int metric)
+{
+    if (nv <= k) return 1;
+    if (eps < 0.0) return 1;
+    if (eps >= 1.0) return 0;
+    float c = metric == 1 ? (float)(1.0 - eps) : (float)((1.0 - eps) * (1.0 - eps));
+    float rhs = c * d2max;
+    return !(d2k >= rhs);
+}
 static int orc_gap_uncertain(int nv, int k, float d2k, float d2max, double eps)
 {
     if (nv <= k) return 1;
@@ -485,7 +594,7 @@ int orc_uncertain(const orc_state *st, int L, int k, double eps)
         if (nv == k) d2k = st->pool[t].d2;
         d2max = st->pool[t].d2;                           /* entries ascend */
     }
-    return orc_gap_uncertain(nv, k, d2k, d2max, eps);
+    return orc_gap_uncertain_m(nv, k, d2k, d2max, eps, st->ix->metric);
 }
 
 /*
@@ -506,7 +615,7 @@ int orc_beam_rerank(const orc_state *st, int L, int k, const float *q, int dist_
     for (int t = 0; t < lim; ++t) {
         if (st->pool[t].phi != 0) continue;
         uint32_t id = st->pool[t].id;
-        float d = orc_dist2(st->ix, q, id, dist_mode);
+        float d = orc_metric_dist(st->ix, q, id, dist_mode);
         int pos = nv;                                      /* insertion by (d2, id) */
         while (pos > 0 && (d < vd[pos - 1] || (d == vd[pos - 1] && id < vid[pos - 1]))) {
             vd[pos] = vd[pos - 1]; vid[pos] = vid[pos - 1]; pos--;
@@ -618,7 +727,7 @@ void orc_boa_search_wl(const orc_index *ix, const float *queries, int64_t Q,
             if (use_pq) {
                 float d2k, d2max;
                 int nv = orc_beam_rerank(st, L, k, q, dist_mode, out_ids + i * k, out_d2 + i * k, &d2k, &d2max);
-                unc = orc_gap_uncertain(nv, k, d2k, d2max, eps);
+                unc = orc_gap_uncertain_m(nv, k, d2k, d2max, eps, ix->metric);
             } else {
                 orc_beam_result(st, k, out_ids + i * k, out_d2 + i * k);    /* scatter */
                 unc = orc_uncertain(st, L, k, eps);

@@ -55,6 +55,10 @@ def lib():
         L.orc_uncertain.argtypes = [vp, i32, i32, dbl]
         L.orc_boa_search_wl.argtypes = [vp, vp, i64, vp, vp, i32, vp, i32, dbl, dbl, i32, i32,
                                         i32, i32, i32, C.c_float, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.orc_set_metric.argtypes = [vp, i32]
+        L.orc_cos_dist.restype = C.c_float
+        L.orc_cos_dist.argtypes = [vp, vp, i64, i32]
+        L.orc_unit_f32.argtypes = [vp, i32, vp]
         L.orc_pq_attach.argtypes = [vp, vp, vp, i32, i32]
         L.orc_pq_table.argtypes = [vp, vp, i32, vp]
         L.orc_pq_dist.restype = C.c_float
@@ -121,6 +125,16 @@ class OracleIndex:
 
     def medoid(self):
         return int(lib().orc_medoid(self.h))
+
+    # --- metric ----------------------------------------------------------------
+    def set_metric(self, metric: str):
+        """'l2' (default) or 'cosine' (float vectors; call once, right after construction)."""
+        assert metric in ("l2", "cosine") and (metric == "l2" or self.vec_dtype == 0)
+        lib().orc_set_metric(self.h, 1 if metric == "cosine" else 0)
+
+    def cos_dist(self, q, p, dist_mode=0):
+        q = np.ascontiguousarray(q, dtype=np.float32)
+        return np.float32(lib().orc_cos_dist(self.h, _p(q), int(p), int(dist_mode)))
 
     # --- product quantisation ------------------------------------------------
     def attach_pq(self, pivots, codes):
