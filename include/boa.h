@@ -22,6 +22,7 @@ typedef struct boa_index boa_index; /* opaque */
 
 enum { BOA_F32 = 0, BOA_U8 = 1 };            /* element type of the stored vectors      */
 enum { BOA_ATTR_I32 = 0, BOA_ATTR_F32 = 1 }; /* cell type of one attribute column       */
+enum { BOA_METRIC_L2 = 0, BOA_METRIC_COSINE = 1 }; /* distance of the search             */
 
 enum {
     BOA_OK = 0,
@@ -131,6 +132,19 @@ int boa_index_create(boa_index** out, const void* vectors, int vec_dtype, int64_
  */
 int boa_index_attach_pq(boa_index* index, const float* pivots, const uint8_t* codes, int M, int K,
                         void* stream);
+
+/*
+ * Choose the distance (Definition 1 allows the Euclidean norm or cosine distance; the paper
+ * itself uses the Euclidean norm, which is the default here).  BOA_METRIC_COSINE: float
+ * vectors only; the index rescales its copy of the vectors to unit length (in place, once:
+ * going back is BOA_EINVAL), every search rescales a copy of its queries, and out_dists
+ * holds cosine distances 1 - cos(x, q) (a zero vector has distance 0.5 to everything),
+ * computed as half the squared Euclidean distance of the unit vectors.  The confidence test
+ * of Eq. 3 then compares cosine distances.  The entry point stays the one chosen at
+ * creation.  A PQ codebook attached to a cosine index must have been trained on unit-length
+ * vectors.  boa_search_noalloc supports the Euclidean metric only.  Synchronises `stream`.
+ */
+int boa_index_set_metric(boa_index* index, int metric, void* stream);
 
 /* Free the index and everything it owns.  NULL is accepted. */
 int boa_index_destroy(boa_index* index);

@@ -67,6 +67,8 @@ def load_library():
     L.boa_get_phase_counts.argtypes = [vp, C.POINTER(i64), i32, C.POINTER(i32), vp]
     L.boa_workspace_bytes.restype = i32
     L.boa_workspace_bytes.argtypes = [vp, i64, i32, C.POINTER(C.c_size_t)]
+    L.boa_index_set_metric.restype = i32
+    L.boa_index_set_metric.argtypes = [vp, i32, vp]
     L.boa_index_attach_pq.restype = i32
     L.boa_index_attach_pq.argtypes = [vp, vp, vp, i32, i32, vp]
     L.boa_get_rerank_counts.restype = i32
@@ -144,6 +146,11 @@ class BoaIndex:
     @property
     def entry(self) -> int:
         return int(self._lib.boa_index_entry(self._h))
+
+    def set_metric(self, metric: str, stream: Optional[torch.cuda.Stream] = None):
+        """boa_index_set_metric: 'l2' (default) or 'cosine' (float vectors, one way)."""
+        _check(self._lib.boa_index_set_metric(self._h, {"l2": 0, "cosine": 1}[metric], _stream_ptr(stream)),
+               "boa_index_set_metric")
 
     def attach_pq(self, pivots: torch.Tensor, codes: torch.Tensor,
                   stream: Optional[torch.cuda.Stream] = None):

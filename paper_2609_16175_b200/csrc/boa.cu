@@ -154,6 +154,29 @@ __global__ void fill_outputs_kernel(uint32_t* ids, float* d2, int64_t n, int32_t
     }
 }
 
+// Cosine metric: scale rows to unit length.  One thread per row: the sum of squares runs in
+// double over the elements in ascending order, the row is multiplied by 1/sqrt(sum) in double
+// and rounded to float (a zero row stays zero).  dst may be src.
+__global__ void unit_rows_kernel(const float* src, int64_t src_stride, float* dst, int64_t dst_stride,
+                                 int64_t n, int D)
+{
+    for (int64_t r = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; r < n; r += (int64_t)gridDim.x * blockDim.x) {
+        const float* x = src + r * src_stride;
+        float* y = dst + r * dst_stride;
+        double s = 0.0;
+        for (int i = 0; i < D; ++i) s += (double)x[i] * (double)x[i];
+        const double inv = s > 0.0 ? 1.0 / sqrt(s) : 0.0;
+        for (int i = 0; i < D; ++i) y[i] = (float)((double)x[i] * inv);
+    }
+}
+
+// out[i] *= 0.5 (cosine distance = half the squared distance of the unit vectors); +inf stays
+__global__ void halve_kernel(float* out, int64_t n)
+{
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        out[i] *= 0.5f;
+}
+
 // dst[0] = src[0]: freezes a survivor count at a point of a stream's order.
 __global__ void copy_word_kernel(uint32_t* dst, const uint32_t* src) { *dst = *src; }
 
@@ -170,6 +193,9 @@ struct boa_index {
     uint8_t* rec = nullptr;
     uint32_t* graph = nullptr;
     int device = 0, num_sms = 0;
+    int metric = BOA_METRIC_L2;
+    float* qunit = nullptr;            // [ws_qunit][D] unit-length copies of a batch's queries (cosine)
+    int64_t ws_qunit = 0;
     // product quantisation (optional)
     uint8_t* pq_codes = nullptr;       // [N][pq_M]
     float* pq_pivots = nullptr;        // [pq_M][pq_K][D / pq_M]
@@ -591,7 +617,7 @@ int boa_index_destroy(boa_index* ix)
     if (!ix) return BOA_OK;
     cudaFree(ix->rec); cudaFree(ix->attr_cells); cudaFree(ix->graph); cudaFree(ix->lists); cudaFree(ix->counters);
     cudaFree(ix->stats); cudaFree(ix->spill); cudaFree(ix->spill_size);
-    cudaFree(ix->pq_codes); cudaFree(ix->pq_pivots);
+    cudaFree(ix->pq_codes); cudaFree(ix->pq_pivots); cudaFree(ix->qunit);
     if (ix->side) cudaStreamDestroy(ix->side);
     if (ix->ev_fork) cudaEventDestroy(ix->ev_fork);
     if (ix->ev_join) cudaEventDestroy(ix->ev_join);
@@ -689,6 +715,19 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
 
     int rc = ensure_workspace(ix, Q, Lmax);
     if (rc != BOA_OK) return rc;
+    if (ix->metric == BOA_METRIC_COSINE) {
+        // the kernels work on unit-length vectors: the index's rows already are, the queries
+        // of this batch are copied
+        if (Q > ix->ws_qunit) {
+            cudaFree(ix->qunit);
+            ix->qunit = nullptr; ix->ws_qunit = 0;
+            BOA_CUDA(cudaMalloc(&ix->qunit, (size_t)Q * ix->D * sizeof(float)));
+            ix->ws_qunit = Q;
+        }
+        unit_rows_kernel<<<(unsigned)((Q + 127) / 128), 128, 0, st>>>(queries, ix->D, ix->qunit, ix->D, Q, ix->D);
+        BOA_CUDA(cudaGetLastError());
+        queries = ix->qunit;
+    }
 
     LaunchPlan lp;
     lp.ix = ix;
@@ -713,7 +752,12 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
     b.lambda = b.fin ? (float)ix->lambda : 0.0f;
     if (ix->eps < 0.0) b.eps_mode = -1;
     else if (ix->eps >= 1.0) b.eps_mode = 1;
-    else { b.eps_mode = 0; b.c_eps = (float)((1.0 - ix->eps) * (1.0 - ix->eps)); }
+    else {
+        // Eq. 3 on norms with squared distances as keys: (1-eps)^2; on cosine distances: 1-eps
+        b.eps_mode = 0;
+        b.c_eps = ix->metric == BOA_METRIC_COSINE ? (float)(1.0 - ix->eps)
+                                                  : (float)((1.0 - ix->eps) * (1.0 - ix->eps));
+    }
     b.final_L = ix->stats; b.n_expand = ix->stats + ix->ws_Q; b.n_scored = ix->stats + 2 * ix->ws_Q;
     b.flags = ix->stats + 3 * ix->ws_Q;
     b.n_rerank = ix->stats + 4 * ix->ws_Q;
@@ -791,6 +835,11 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
             BOA_CUDA(cudaStreamWaitEvent(st, ix->ev_join, 0));
         }
     }
+    if (ix->metric == BOA_METRIC_COSINE) {
+        halve_kernel<<<ix->num_sms * 2, 256, 0, st>>>(out_dists, Q * k);
+        BOA_CUDA(cudaGetLastError());
+        extra_launches += 2;
+    }
     ix->last_launches = lp.launches + extra_launches;
     return BOA_OK;
 }
@@ -826,6 +875,21 @@ int boa_index_attach_pq(boa_index* ix, const float* pivots, const uint8_t* codes
     BOA_CUDA(cudaMemcpyAsync(ix->pq_pivots, pivots, pb, cudaMemcpyDeviceToDevice, st));
     BOA_CUDA(cudaStreamSynchronize(st));
     ix->pq_M = M; ix->pq_K = K;
+    return BOA_OK;
+}
+
+int boa_index_set_metric(boa_index* ix, int metric, void* stream)
+{
+    if (!ix || (metric != BOA_METRIC_L2 && metric != BOA_METRIC_COSINE)) return BOA_EINVAL;
+    if (metric == ix->metric) return BOA_OK;
+    // the rows are rescaled in place, once: there is no way back to the Euclidean metric
+    if (ix->metric != BOA_METRIC_L2 || ix->vec_dtype != BOA_F32 || !on_device(ix->device)) return BOA_EINVAL;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    float* rows = reinterpret_cast<float*>(ix->rec);
+    unit_rows_kernel<<<ix->num_sms * 8, 128, 0, st>>>(rows, ix->rec_stride / 4, rows, ix->rec_stride / 4, ix->N, ix->D);
+    BOA_CUDA(cudaGetLastError());
+    BOA_CUDA(cudaStreamSynchronize(st));
+    ix->metric = BOA_METRIC_COSINE;
     return BOA_OK;
 }
 
@@ -867,6 +931,7 @@ int boa_search_noalloc(boa_index* ix, const float* queries, int64_t Q, const voi
     if (!ix) return BOA_EINVAL;
     if (Q > kNoAllocMaxQ || Lmax > kNoAllocMaxWidth) return BOA_ETOOBIG;
     if (!on_device(ix->device)) return BOA_EINVAL;
+    if (ix->metric != BOA_METRIC_L2) return BOA_EINVAL;       // the unit-length query copies need scratch of Q*D floats
     unsigned char* base = nullptr;
     const int rc0 = noalloc_scratch(&base);
     if (rc0 != BOA_OK) return rc0;
