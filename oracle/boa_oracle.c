@@ -9,7 +9,11 @@
  * What each function follows:
  *   orc_phi            filter distance: number of the query's closed range
  *                      predicates a point violates (Background, "Graph
- *                      construction", last paragraph; Eq. 2 gives g = [phi == 0])
+ *                      construction", last paragraph; Eq. 2 gives g = [phi == 0]);
+ *                      a column can also hold membership masks (the Conclusion's
+ *                      equality / subset filters)
+ *   orc_range_penalty  the numeric range distance the same paragraph mentions as the
+ *                      alternative to counting (extension: the paper counts)
  *   orc_bruteforce     exact range-filtered k-NN (Definition 1, Definition 2, Eq. 1)
  *   orc_beam_*         filter-aware beam search at one beamwidth (Algorithm 2),
  *                      with exact L2 distances instead of PQ look-ups
@@ -65,6 +69,7 @@
 #define ORC_U8 1
 #define ORC_ATTR_I32 0
 #define ORC_ATTR_F32 1
+#define ORC_ATTR_SET 2          /* cell = 32-bit membership mask of the point */
 
 typedef struct {
     int64_t N;
@@ -240,11 +245,51 @@ int orc_phi(const orc_index *ix, const int32_t *lo, const int32_t *hi, int64_t p
             memcpy(&l, &lo[j], 4);
             memcpy(&h, &hi[j], 4);
             if (!(a >= l && a <= h)) v++;      /* NaN violates */
+        } else if (ix->attr_types[j] == ORC_ATTR_SET) {
+            /* membership predicate: lo = the wanted tags; hi == 0: the point must carry at
+               least one of them, hi != 0: all of them */
+            uint32_t have = (uint32_t)cell & (uint32_t)lo[j];
+            if (hi[j] == 0 ? have == 0u : have != (uint32_t)lo[j]) v++;
         } else {
             if (cell < lo[j] || cell > hi[j]) v++;
         }
     }
     return v;
+}
+
+/*
+ * Distance-to-range penalty, the numeric alternative to the violation count: for every
+ * violated predicate the distance from the cell to the nearer end of its range, times the
+ * caller's scale for that attribute, added over the attributes in ascending order in fp32.
+ * Integer cells: the distance is taken in double (exact) and rounded once to float; float
+ * cells: one fp32 subtraction, a NaN cell counts as infinitely far; a violated membership
+ * predicate costs its scale.  Zero exactly when the point is filter-valid.
+ */
+float orc_range_penalty(const orc_index *ix, const int32_t *lo, const int32_t *hi, int64_t p,
+                        const float *scales)
+{
+    float pen = 0.0f;
+    for (int j = 0; j < ix->m; ++j) {
+        int32_t cell = ix->attrs[p * ix->m + j];
+        float e = 0.0f;
+        if (ix->attr_types[j] == ORC_ATTR_F32) {
+            float a, l, h;
+            memcpy(&a, &cell, 4);
+            memcpy(&l, &lo[j], 4);
+            memcpy(&h, &hi[j], 4);
+            if (a < l) e = l - a;
+            else if (a > h) e = a - h;
+            else if (!(a >= l && a <= h)) e = INFINITY;
+        } else if (ix->attr_types[j] == ORC_ATTR_SET) {
+            uint32_t have = (uint32_t)cell & (uint32_t)lo[j];
+            if (hi[j] == 0 ? have == 0u : have != (uint32_t)lo[j]) e = 1.0f;
+        } else {
+            if (cell < lo[j]) e = (float)((double)lo[j] - (double)cell);
+            else if (cell > hi[j]) e = (float)((double)cell - (double)hi[j]);
+        }
+        pen = pen + e * scales[j];
+    }
+    return pen;
 }
 
 /* ------------------------------------------------------------------ */
@@ -375,6 +420,7 @@ typedef struct {
     int phi;
     float d2;
     float score;         /* d2 + lambda*phi (finite lambda only) */
+    float pen;           /* distance-to-range penalty (when it replaces phi in the score) */
     uint32_t id;
     int expanded;
 } orc_entry_t;
@@ -391,6 +437,7 @@ typedef struct {
     int64_t n_expand, n_scored;
     int hit_cap;
     float *pq_table;     /* [M][K] of the current query when the search runs on PQ distances, else NULL */
+    const float *pen_scales; /* [m] when the score uses the distance-to-range penalty, else NULL */
 } orc_state;
 
 /* The order the search works by.  The paper's score is dist + lambda*phi with one lambda
@@ -420,6 +467,9 @@ orc_state *orc_state_new(const orc_index *ix, int C)
 }
 /* set before orc_beam_init; lambda >= 0, INFINITY for the lexicographic order */
 void orc_state_set_lambda(orc_state *st, float lambda) { st->lambda = lambda; }
+/* score = d2 + lambda * (distance-to-range penalty with these per-attribute scales) instead of
+   d2 + lambda * (violation count); needs a finite lambda.  NULL switches back. */
+void orc_state_set_penalty(orc_state *st, const float *scales) { st->pen_scales = scales; }
 void orc_state_free(orc_state *st)
 {
     free(st->pool); free(st->seen); free(st->touched); free(st->pq_table); free(st);
@@ -464,7 +514,8 @@ static void orc_mark_seen(orc_state *st, uint32_t id)
 static void orc_pool_insert(orc_state *st, orc_entry_t e)
 {
     int pos = st->size;
-    e.score = isinf(st->lambda) ? e.d2 : fmaf(st->lambda, (float)e.phi, e.d2);
+    e.score = isinf(st->lambda) ? e.d2
+              : fmaf(st->lambda, st->pen_scales ? e.pen : (float)e.phi, e.d2);
     while (pos > 0 && orc_less(st, &e, &st->pool[pos - 1])) { st->pool[pos] = st->pool[pos - 1]; pos--; }
     st->pool[pos] = e;
     st->size++;
@@ -480,6 +531,7 @@ void orc_beam_init(orc_state *st, int C, const float *q, const int32_t *lo, cons
     orc_entry_t e;
     e.id = (uint32_t)ix->entry; e.expanded = 0;
     e.phi = orc_phi(ix, lo, hi, ix->entry);
+    e.pen = st->pen_scales ? orc_range_penalty(ix, lo, hi, ix->entry, st->pen_scales) : 0.0f;
     e.d2 = orc_search_dist(st, q, ix->entry, dist_mode);
     orc_mark_seen(st, e.id);
     orc_pool_insert(st, e);
@@ -526,6 +578,7 @@ void orc_beam_run_w(orc_state *st, int L, const float *q, const int32_t *lo, con
                 orc_entry_t e;
                 e.id = n; e.expanded = 0;
                 e.phi = orc_phi(ix, lo, hi, n);
+                e.pen = st->pen_scales ? orc_range_penalty(ix, lo, hi, n, st->pen_scales) : 0.0f;
                 e.d2 = orc_search_dist(st, q, n, dist_mode);
                 orc_pool_insert(st, e);
             }
@@ -688,7 +741,7 @@ void orc_boa_search_wl(const orc_index *ix, const float *queries, int64_t Q,
                       const int32_t *lo, const int32_t *hi, int k,
                       const int32_t *widths, int n_widths, double eps, double tau,
                       int mode, int dist_mode, int cap_mult, int cap_add, int W, float lambda,
-                      int use_pq,
+                      int use_pq, const float *pen_scales,
                       uint32_t *out_ids, float *out_d2,
                       int32_t *final_L, int32_t *n_expand, int32_t *n_scored, int32_t *flags,
                       int64_t *phase_active)
@@ -697,6 +750,7 @@ void orc_boa_search_wl(const orc_index *ix, const float *queries, int64_t Q,
     for (int p = 0; p < n_widths; ++p) if (widths[p] > Cmax) Cmax = widths[p];
     orc_state *st = orc_state_new(ix, Cmax);
     orc_state_set_lambda(st, lambda);
+    orc_state_set_penalty(st, pen_scales);
     for (int p = 0; p < n_widths; ++p) phase_active[p] = 0;
 
     uint8_t *active = (uint8_t *)malloc((size_t)Q + 1);             /* the set A */

@@ -54,7 +54,10 @@ def lib():
         L.orc_uncertain.restype = i32
         L.orc_uncertain.argtypes = [vp, i32, i32, dbl]
         L.orc_boa_search_wl.argtypes = [vp, vp, i64, vp, vp, i32, vp, i32, dbl, dbl, i32, i32,
-                                        i32, i32, i32, C.c_float, i32, vp, vp, vp, vp, vp, vp, vp]
+                                        i32, i32, i32, C.c_float, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.orc_range_penalty.restype = C.c_float
+        L.orc_range_penalty.argtypes = [vp, vp, vp, i64, vp]
+        L.orc_state_set_penalty.argtypes = [vp, vp]
         L.orc_set_metric.argtypes = [vp, i32]
         L.orc_cos_dist.restype = C.c_float
         L.orc_cos_dist.argtypes = [vp, vp, i64, i32]
@@ -123,6 +126,12 @@ class OracleIndex:
         hi = np.ascontiguousarray(hi, dtype=np.int32)
         return int(lib().orc_phi(self.h, _p(lo), _p(hi), int(p)))
 
+    def range_penalty(self, lo, hi, p, scales):
+        lo = np.ascontiguousarray(lo, dtype=np.int32)
+        hi = np.ascontiguousarray(hi, dtype=np.int32)
+        scales = np.ascontiguousarray(scales, dtype=np.float32)
+        return np.float32(lib().orc_range_penalty(self.h, _p(lo), _p(hi), int(p), _p(scales)))
+
     def medoid(self):
         return int(lib().orc_medoid(self.h))
 
@@ -172,14 +181,15 @@ class OracleIndex:
 
     # --- one beam search, step-wise ------------------------------------------
     def beam(self, q, lo, hi, L, C=None, dist_mode=0, max_expand=1 << 40, expand_w=1,
-             lam=float("inf"), pq=False):
+             lam=float("inf"), pq=False, penalty_scales=None):
         return OracleBeam(self, q, lo, hi, L, C if C is not None else L, dist_mode, max_expand,
-                          expand_w, lam, pq)
+                          expand_w, lam, pq, penalty_scales)
 
     # --- the multi-phase batch driver ----------------------------------------
     def search(self, queries, lo, hi, k, widths, eps=0.05, tau=0.0, mode="restart",
-               dist_mode=0, cap=DEFAULT_CAP, expand_w=1, lam=float("inf"), pq=False):
+               dist_mode=0, cap=DEFAULT_CAP, expand_w=1, lam=float("inf"), pq=False, penalty_scales=None):
         queries = np.ascontiguousarray(queries, dtype=np.float32)
+        ps = None if penalty_scales is None else np.ascontiguousarray(penalty_scales, dtype=np.float32)
         lo = np.ascontiguousarray(lo, dtype=np.int32)
         hi = np.ascontiguousarray(hi, dtype=np.int32)
         Q = queries.shape[0]
@@ -194,7 +204,7 @@ class OracleIndex:
         lib().orc_boa_search_wl(self.h, _p(queries), Q, _p(lo), _p(hi), k, _p(w), len(w),
                                float(eps), float(tau), 1 if mode == "resume" else 0, int(dist_mode),
                                int(cap[0]), int(cap[1]), int(expand_w), float(lam), 1 if pq else 0,
-                               _p(ids), _p(d2), _p(final_L),
+                               None if ps is None else _p(ps), _p(ids), _p(d2), _p(final_L),
                                _p(n_expand), _p(n_scored), _p(flags), _p(phase_active))
         return dict(ids=ids, d2=d2, final_L=final_L, n_expand=n_expand, n_scored=n_scored,
                     flags=flags, phase_active=phase_active)
@@ -204,9 +214,10 @@ class OracleBeam:
     """One query's Algorithm-2 state, for tests that look inside a search."""
 
     def __init__(self, index, q, lo, hi, L, C, dist_mode, max_expand, expand_w=1, lam=float("inf"),
-                 pq=False):
+                 pq=False, penalty_scales=None):
         self.ix = index
         self.pq = bool(pq)
+        self.pen = None if penalty_scales is None else np.ascontiguousarray(penalty_scales, dtype=np.float32)
         self.expand_w = int(expand_w)
         self.q = np.ascontiguousarray(q, dtype=np.float32)
         self.lo = np.ascontiguousarray(lo, dtype=np.int32)
@@ -214,6 +225,8 @@ class OracleBeam:
         self.dist_mode = dist_mode
         self.st = lib().orc_state_new(index.h, int(C))
         lib().orc_state_set_lambda(self.st, float(lam))
+        if self.pen is not None:
+            lib().orc_state_set_penalty(self.st, _p(self.pen))
         if self.pq:
             lib().orc_state_use_pq(self.st, 1, _p(self.q), dist_mode)
         lib().orc_beam_init(self.st, int(C), _p(self.q), _p(self.lo), _p(self.hi), dist_mode)
