@@ -21,7 +21,8 @@ extern "C" {
 typedef struct boa_index boa_index; /* opaque */
 
 enum { BOA_F32 = 0, BOA_U8 = 1 };            /* element type of the stored vectors      */
-enum { BOA_ATTR_I32 = 0, BOA_ATTR_F32 = 1 }; /* cell type of one attribute column       */
+enum { BOA_ATTR_I32 = 0, BOA_ATTR_F32 = 1,   /* cell type of one attribute column       */
+       BOA_ATTR_SET32 = 2 };                 /* 32-bit membership mask (see boa_search)  */
 enum { BOA_METRIC_L2 = 0, BOA_METRIC_COSINE = 1 }; /* distance of the search             */
 
 enum {
@@ -160,7 +161,11 @@ int64_t boa_index_entry(const boa_index* index);
  *
  *   queries   [Q][D] float
  *   lo, hi    [Q][m] closed bounds, cell types as the index's columns; lo > hi is legal
- *             (empty valid set); an unconstrained attribute gets the type's full range
+ *             (empty valid set); an unconstrained attribute gets the type's full range; an
+ *             equality predicate is lo == hi.  For a BOA_ATTR_SET32 column (the equality /
+ *             subset filters the paper's Conclusion mentions: the cell is the set of tags
+ *             the point carries) lo is the set of wanted tags and hi the mode: 0 = the
+ *             point must carry at least one of them, non-zero = all of them
  *   out_ids   [Q][k]  ids of the filter-valid nearest points found, ascending by
  *             (squared distance, id), duplicate-free; BOA_NO_ID fills unused slots
  *   out_dists [Q][k]  squared L2 distances in fp32; +inf in unused slots
@@ -209,6 +214,20 @@ int boa_search(boa_index* index, const float* queries, int64_t Q, const void* lo
 int boa_search_noalloc(boa_index* index, const float* queries, int64_t Q, const void* lo,
                        const void* hi, int k, int L0, int Lmax, uint32_t* out_ids, float* out_dists,
                        void* stream);
+
+/*
+ * Replace the violation count in the finite-lambda score by the numeric distance to the
+ * range (the range filter distance the paper's graph-construction paragraph names; the
+ * paper's own system counts violated predicates, which stays the default): score =
+ * d^2 + lambda * sum_j scales[j] * dist_j, where dist_j is how far attribute j lies outside
+ * its range (0 inside; integer cells exact, float cells one subtraction, NaN infinitely
+ * far, a violated membership predicate 1), added over j in ascending order in fp32.
+ * Validity of an answer is still decided by the predicates alone.
+ *   scales  HOST array [m], every entry finite and > 0; NULL goes back to the count
+ * Needs a finite BOA_PARAM_LAMBDA at search time (else boa_search returns BOA_EINVAL);
+ * not combined with PQ traversal or expansion width 2.  Synchronises `stream`.
+ */
+int boa_set_range_penalty(boa_index* index, const float* scales, void* stream);
 
 /* Set one parameter (keys above).  BOA_EINVAL for an unknown key or a value out of range. */
 int boa_set_param(boa_index* index, int key, double value);

@@ -67,6 +67,8 @@ def load_library():
     L.boa_get_phase_counts.argtypes = [vp, C.POINTER(i64), i32, C.POINTER(i32), vp]
     L.boa_workspace_bytes.restype = i32
     L.boa_workspace_bytes.argtypes = [vp, i64, i32, C.POINTER(C.c_size_t)]
+    L.boa_set_range_penalty.restype = i32
+    L.boa_set_range_penalty.argtypes = [vp, C.POINTER(C.c_float), vp]
     L.boa_index_set_metric.restype = i32
     L.boa_index_set_metric.argtypes = [vp, i32, vp]
     L.boa_index_attach_pq.restype = i32
@@ -146,6 +148,11 @@ class BoaIndex:
     @property
     def entry(self) -> int:
         return int(self._lib.boa_index_entry(self._h))
+
+    def set_range_penalty(self, scales: Optional[Sequence[float]], stream: Optional[torch.cuda.Stream] = None):
+        """boa_set_range_penalty: per-attribute scales (None: back to the violation count)."""
+        arr = None if scales is None else (C.c_float * self.m)(*[float(x) for x in scales])
+        _check(self._lib.boa_set_range_penalty(self._h, arr, _stream_ptr(stream)), "boa_set_range_penalty")
 
     def set_metric(self, metric: str, stream: Optional[torch.cuda.Stream] = None):
         """boa_index_set_metric: 'l2' (default) or 'cosine' (float vectors, one way)."""

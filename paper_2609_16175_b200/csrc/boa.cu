@@ -189,6 +189,8 @@ struct boa_index {
     int rec_stride = 0, nchunks = 0;
     uint32_t* attr_cells = nullptr;    // [N][m] attribute cells
     uint32_t attr_float_mask = 0;
+    uint32_t attr_set_mask = 0;        // columns holding membership masks
+    float* pen_scales = nullptr;       // [8] device copy of the range-penalty scales, or null (count)
     int64_t entry = 0;
     uint8_t* rec = nullptr;
     uint32_t* graph = nullptr;
@@ -284,21 +286,22 @@ struct KernelChoice {
     bool q_in_smem;     // the generic-length kernels keep the query in shared memory
 };
 
-template <int VT, int CPL, int W, bool PQ>
+template <int VT, int CPL, int W, bool PQ, bool EXT>
 KernelChoice pick_rn(int R, bool exact)
 {
     if (R <= 32) {
-        if (exact) return {boa::boa_search_kernel<VT, 1, W, CPL, (CPL > 0), PQ>, W, CPL == 0};
-        return {boa::boa_search_kernel<VT, 1, W, CPL, false, PQ>, W, CPL == 0};
+        if (exact) return {boa::boa_search_kernel<VT, 1, W, CPL, (CPL > 0), PQ, EXT>, W, CPL == 0};
+        return {boa::boa_search_kernel<VT, 1, W, CPL, false, PQ, EXT>, W, CPL == 0};
     }
-    if (exact) return {boa::boa_search_kernel<VT, 2, W, CPL, (CPL > 0), PQ>, 2 * W, CPL == 0};
-    return {boa::boa_search_kernel<VT, 2, W, CPL, false, PQ>, 2 * W, CPL == 0};
+    if (exact) return {boa::boa_search_kernel<VT, 2, W, CPL, (CPL > 0), PQ, EXT>, 2 * W, CPL == 0};
+    return {boa::boa_search_kernel<VT, 2, W, CPL, false, PQ, EXT>, 2 * W, CPL == 0};
 }
 template <int VT, int CPL>
-KernelChoice pick_rs(int R, bool exact, int expand_w, bool pq)
+KernelChoice pick_rs(int R, bool exact, int expand_w, bool pq, bool ext)
 {
-    if (pq) return pick_rn<VT, CPL, 1, true>(R, exact);
-    return expand_w == 2 ? pick_rn<VT, CPL, 2, false>(R, exact) : pick_rn<VT, CPL, 1, false>(R, exact);
+    if (pq) return pick_rn<VT, CPL, 1, true, false>(R, exact);
+    if (ext) return pick_rn<VT, CPL, 1, false, true>(R, exact);
+    return expand_w == 2 ? pick_rn<VT, CPL, 2, false, false>(R, exact) : pick_rn<VT, CPL, 1, false, false>(R, exact);
 }
 
 KernelChoice pick_kernel(const boa_index* ix)
@@ -306,19 +309,20 @@ KernelChoice pick_kernel(const boa_index* ix)
     const int cpl = (ix->nchunks + 7) / 8;      // 16-byte chunks per lane of an 8-lane group
     const bool exact = ix->nchunks == 8 * cpl;
     const bool pq = ix->use_pq != 0;
+    const bool ext = ix->attr_set_mask != 0 || ix->pen_scales != nullptr;
     if (ix->vec_dtype == BOA_F32) {
         switch (cpl) {
-            case 1: return pick_rs<0, 1>(ix->R, exact, ix->expand_w, pq);
-            case 2: return pick_rs<0, 2>(ix->R, exact, ix->expand_w, pq);
-            case 3: return pick_rs<0, 3>(ix->R, exact, ix->expand_w, pq);
-            case 4: return pick_rs<0, 4>(ix->R, exact, ix->expand_w, pq);
-            default: return pick_rs<0, 0>(ix->R, false, ix->expand_w, pq);
+            case 1: return pick_rs<0, 1>(ix->R, exact, ix->expand_w, pq, ext);
+            case 2: return pick_rs<0, 2>(ix->R, exact, ix->expand_w, pq, ext);
+            case 3: return pick_rs<0, 3>(ix->R, exact, ix->expand_w, pq, ext);
+            case 4: return pick_rs<0, 4>(ix->R, exact, ix->expand_w, pq, ext);
+            default: return pick_rs<0, 0>(ix->R, false, ix->expand_w, pq, ext);
         }
     }
     switch (cpl) {
-        case 1: return pick_rs<1, 1>(ix->R, exact, ix->expand_w, pq);
-        case 2: return pick_rs<1, 2>(ix->R, exact, ix->expand_w, pq);
-        default: return pick_rs<1, 0>(ix->R, false, ix->expand_w, pq);
+        case 1: return pick_rs<1, 1>(ix->R, exact, ix->expand_w, pq, ext);
+        case 2: return pick_rs<1, 2>(ix->R, exact, ix->expand_w, pq, ext);
+        default: return pick_rs<1, 0>(ix->R, false, ix->expand_w, pq, ext);
     }
 }
 
@@ -516,7 +520,8 @@ int boa_index_create(boa_index** out, const void* vectors, int vec_dtype, int64_
     if (!aligned16(vectors) || !aligned16(attrs) || !aligned16(graph)) return BOA_EINVAL;
     if (entry >= N || entry < -1) return BOA_EINVAL;
     for (int j = 0; j < m; ++j)
-        if (attr_types[j] != BOA_ATTR_I32 && attr_types[j] != BOA_ATTR_F32) return BOA_EINVAL;
+        if (attr_types[j] != BOA_ATTR_I32 && attr_types[j] != BOA_ATTR_F32 && attr_types[j] != BOA_ATTR_SET32)
+            return BOA_EINVAL;
 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     boa_index* ix = new (std::nothrow) boa_index();
@@ -537,6 +542,7 @@ int boa_index_create(boa_index** out, const void* vectors, int vec_dtype, int64_
     ix->rec_stride = (vec_bytes + 31) & ~31;
     for (int j = 0; j < m; ++j)
         if (attr_types[j] == BOA_ATTR_F32) ix->attr_float_mask |= 1u << j;
+        else if (attr_types[j] == BOA_ATTR_SET32) ix->attr_set_mask |= 1u << j;
     BOA_TRY(cudaGetDevice(&ix->device));
     BOA_TRY(cudaDeviceGetAttribute(&ix->num_sms, cudaDevAttrMultiProcessorCount, ix->device));
     BOA_TRY(cudaMalloc(&ix->rec, (size_t)N * ix->rec_stride));
@@ -617,7 +623,7 @@ int boa_index_destroy(boa_index* ix)
     if (!ix) return BOA_OK;
     cudaFree(ix->rec); cudaFree(ix->attr_cells); cudaFree(ix->graph); cudaFree(ix->lists); cudaFree(ix->counters);
     cudaFree(ix->stats); cudaFree(ix->spill); cudaFree(ix->spill_size);
-    cudaFree(ix->pq_codes); cudaFree(ix->pq_pivots); cudaFree(ix->qunit);
+    cudaFree(ix->pq_codes); cudaFree(ix->pq_pivots); cudaFree(ix->qunit); cudaFree(ix->pen_scales);
     if (ix->side) cudaStreamDestroy(ix->side);
     if (ix->ev_fork) cudaEventDestroy(ix->ev_fork);
     if (ix->ev_join) cudaEventDestroy(ix->ev_join);
@@ -705,6 +711,11 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
     if (k < 1 || k > L0 || L0 > Lmax || Lmax > BOA_MAX_WIDTH) return BOA_EINVAL;
     if (ix->n_sched > 0 && (L0 != ix->sched[0] || Lmax != ix->sched[ix->n_sched - 1])) return BOA_EINVAL;
     if (ix->use_pq && (k > boa::kPqMaxK || ix->expand_w != 1)) return BOA_EINVAL;
+    // membership columns and the range penalty have kernels for one node per iteration and
+    // exact distances; the penalty is a term of the finite-lambda score
+    const bool ext = ix->attr_set_mask != 0 || ix->pen_scales != nullptr;
+    if (ext && (ix->use_pq || ix->expand_w != 1)) return BOA_EINVAL;
+    if (ix->pen_scales && isinf(ix->lambda)) return BOA_EINVAL;
     if (Q == 0) { ix->last_Q = 0; ix->last_phases = 0; ix->last_launches = 0; return BOA_OK; }
     if (!queries || !lo || !hi || !out_ids || !out_dists) return BOA_EINVAL;
     if (!on_device(ix->device)) return BOA_EINVAL;
@@ -743,6 +754,7 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
     b.timers = reinterpret_cast<unsigned long long*>(ix->counters + kCntWords);
 #endif
     b.attr_float_mask = ix->attr_float_mask; b.entry = (uint32_t)ix->entry;
+    b.attr_set_mask = ix->attr_set_mask; b.pen_scales = ix->pen_scales;
     b.queries = queries;
     b.lo = reinterpret_cast<const int32_t*>(lo);
     b.hi = reinterpret_cast<const int32_t*>(hi);
@@ -875,6 +887,26 @@ int boa_index_attach_pq(boa_index* ix, const float* pivots, const uint8_t* codes
     BOA_CUDA(cudaMemcpyAsync(ix->pq_pivots, pivots, pb, cudaMemcpyDeviceToDevice, st));
     BOA_CUDA(cudaStreamSynchronize(st));
     ix->pq_M = M; ix->pq_K = K;
+    return BOA_OK;
+}
+
+int boa_set_range_penalty(boa_index* ix, const float* scales, void* stream)
+{
+    if (!ix || !on_device(ix->device)) return BOA_EINVAL;
+    if (!scales) {
+        cudaFree(ix->pen_scales);
+        ix->pen_scales = nullptr;
+        return BOA_OK;
+    }
+    float h[BOA_MAX_ATTRS] = {0};
+    for (int j = 0; j < ix->m; ++j) {
+        if (!(scales[j] > 0.0f) || isinf(scales[j])) return BOA_EINVAL;
+        h[j] = scales[j];
+    }
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (!ix->pen_scales) BOA_CUDA(cudaMalloc(&ix->pen_scales, sizeof(h)));
+    BOA_CUDA(cudaMemcpyAsync(ix->pen_scales, h, sizeof(h), cudaMemcpyHostToDevice, st));
+    BOA_CUDA(cudaStreamSynchronize(st));
     return BOA_OK;
 }
 

@@ -99,6 +99,9 @@ struct SearchParams {
     int rec_stride;           // bytes, multiple of 32
     int nchunks;              // 16-byte chunks of one vector
     uint32_t attr_float_mask; // bit j set: column j is float
+    uint32_t attr_set_mask;   // bit j set: column j holds membership masks (EXT kernels)
+    const float* pen_scales;  // [8] per-attribute scale of the distance-to-range penalty, or null:
+                              // the score's filter term is then the violation count (EXT kernels)
     uint32_t entry;
     // product quantisation (PQ kernels only): D = pq_M * pq_dsub
     const uint8_t* pq_codes;  // [N][pq_M] centroid index per subspace, rows of pq_M bytes (multiple of 16)
@@ -366,11 +369,14 @@ __host__ __device__ inline WarpSmem warp_smem_layout(int C, int table_bytes, int
 // subvector-to-centroid distances in shared memory, one look-up per subspace and candidate,
 // a lane per candidate); when a phase has converged the filter-valid beam entries are ranked
 // by exact distance with the same row-scoring code the exact search uses.
-template <int VT, int RN, int W, int CPL, bool EXACT, bool PQ = false>
+// EXT: membership-mask columns and the distance-to-range penalty (kept out of the default
+// kernels, whose register allocation has no room to spare).
+template <int VT, int RN, int W, int CPL, bool EXACT, bool PQ = false, bool EXT = false>
 __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_kernel(const SearchParams p)
 {
     static_assert(W == 1 || W == 2, "expansion width 1 or 2");
     static_assert(!PQ || W == 1, "PQ traversal expands one node per iteration");
+    static_assert(!EXT || (W == 1 && !PQ), "extended predicates: one node per iteration, exact distances");
     constexpr int RS = RN * W;                      // adjacency slots per lane and iteration
     extern __shared__ __align__(128) uint8_t smem_raw[];
     const int lane = threadIdx.x;
@@ -427,6 +433,9 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
             my_hi = p.hi[(size_t)qi * p.m + g];
         }
         const bool my_float = (p.attr_float_mask >> g) & 1u;
+        const bool my_set = EXT && ((p.attr_set_mask >> g) & 1u);
+        const bool pen_on = EXT && p.pen_scales != nullptr;
+        const float my_scale = (pen_on && g < p.m) ? __ldg(p.pen_scales + g) : 0.0f;
         __syncwarp();
         float4 qreg[NQ];           // this lane's slices of the query (CPL > 0)
         if (CPL > 0) {
@@ -514,23 +523,53 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
             v += __shfl_xor_sync(0xffffffffu, v, 2);
             v += __shfl_xor_sync(0xffffffffu, v, 1);
             bool v0, v1;
+            float e0 = 0.0f, e1 = 0.0f;      // EXT: this lane's attribute's distance to its range
             if (my_float) {
                 const float l = __int_as_float(my_lo), h = __int_as_float(my_hi);
-                v0 = !(__uint_as_float(av0) >= l && __uint_as_float(av0) <= h);
-                v1 = !(__uint_as_float(av1) >= l && __uint_as_float(av1) <= h);
+                const float c0 = __uint_as_float(av0), c1 = __uint_as_float(av1);
+                v0 = !(c0 >= l && c0 <= h);
+                v1 = !(c1 >= l && c1 <= h);
+                if (EXT) {
+                    e0 = c0 < l ? l - c0 : (c0 > h ? c0 - h : (v0 ? __int_as_float(0x7f800000) : 0.0f));
+                    e1 = c1 < l ? l - c1 : (c1 > h ? c1 - h : (v1 ? __int_as_float(0x7f800000) : 0.0f));
+                }
+            } else if (my_set) {
+                // membership: lo = the wanted tags; hi == 0: at least one of them, else all of them
+                const uint32_t h0 = av0 & (uint32_t)my_lo, h1 = av1 & (uint32_t)my_lo;
+                v0 = my_hi == 0 ? h0 == 0u : h0 != (uint32_t)my_lo;
+                v1 = my_hi == 0 ? h1 == 0u : h1 != (uint32_t)my_lo;
+                e0 = v0 ? 1.0f : 0.0f;
+                e1 = v1 ? 1.0f : 0.0f;
             } else {
                 v0 = (int32_t)av0 < my_lo || (int32_t)av0 > my_hi;
                 v1 = (int32_t)av1 < my_lo || (int32_t)av1 > my_hi;
+                if (EXT) {
+                    // exact in double, rounded once
+                    const int32_t c0 = (int32_t)av0, c1 = (int32_t)av1;
+                    e0 = c0 < my_lo ? (float)((double)my_lo - (double)c0) : (c0 > my_hi ? (float)((double)c0 - (double)my_hi) : 0.0f);
+                    e1 = c1 < my_lo ? (float)((double)my_lo - (double)c1) : (c1 > my_hi ? (float)((double)c1 - (double)my_hi) : 0.0f);
+                }
             }
             const unsigned bal0 = __ballot_sync(0xffffffffu, v0 && act0 && g < p.m);
             const unsigned bal1 = __ballot_sync(0xffffffffu, v1 && act1 && g < p.m);
             const unsigned bal = hi4 ? bal1 : bal0;
             const int jj = hi4 ? j1 : j0;
+            float pen = 0.0f;
+            if (pen_on) {
+                // the attributes' scaled distances, added in ascending attribute order
+                const float s0 = __fmul_rn(e0, my_scale), s1 = __fmul_rn(e1, my_scale);
+                float p0 = 0.0f, p1 = 0.0f;
+                for (int a = 0; a < p.m; ++a) {
+                    p0 = __fadd_rn(p0, __shfl_sync(0xffffffffu, s0, (lane & ~7) + a));
+                    p1 = __fadd_rn(p1, __shfl_sync(0xffffffffu, s1, (lane & ~7) + a));
+                }
+                pen = hi4 ? p1 : p0;
+            }
             if ((g & 3) == 0 && jj < cnt)
             {
                 const uint32_t phi = __popc((bal >> (8 * gi)) & 0xFFu);
                 // finite lambda: one fused multiply-add gives the score the pool orders by
-                if (fin) nk[jj] = pack_key(true, phi, __fmaf_rn(p.lambda, (float)phi, v), hi4 ? id1 : id0);
+                if (fin) nk[jj] = pack_key(true, phi, __fmaf_rn(p.lambda, pen_on ? pen : (float)phi, v), hi4 ? id1 : id0);
                 else nk[jj] = pack_key(false, phi, v, hi4 ? id1 : id0);
             }
         };

@@ -30,7 +30,7 @@ def make_pair(d, entry=-1):
 
 
 def gpu_search(gpu, g, k, widths, mode="restart", eps=0.05, tau=0.0, plus_k=0, cap=(8, 64),
-               sel=None, expand_w=1, lam=float("inf"), pq=False):
+               sel=None, expand_w=1, lam=float("inf"), pq=False, penalty_scales=None):
     gpu.set_param("mode", 1 if mode == "resume" else 0)
     gpu.set_param("eps", eps)
     gpu.set_param("tau", tau)
@@ -40,6 +40,7 @@ def gpu_search(gpu, g, k, widths, mode="restart", eps=0.05, tau=0.0, plus_k=0, c
     gpu.set_param("expand_w", expand_w)
     gpu.set_param("lam", lam)
     gpu.set_param("pq", 1 if pq else 0)
+    gpu.set_range_penalty(penalty_scales)
     gpu.set_schedule(list(widths))
     q, lo, hi = g["queries"], g["lo"], g["hi"]
     if sel is not None:
