@@ -18,6 +18,9 @@
  *   orc_beam_*         filter-aware beam search at one beamwidth (Algorithm 2),
  *                      with exact L2 distances instead of PQ look-ups
  *   orc_uncertain      confidence test gamma(D_i) <= eps (Eq. 3)
+ *   orc_prune, orc_build_graph   construction of the proximity graph (Background, "Graph
+ *                      construction": Vamana insertion with alpha-dominance pruning, one
+ *                      pruning run per attribute threshold)
  *   orc_cos_*          cosine distance (Definition 1 allows the Euclidean norm or cosine distance;
  *                      the paper itself uses the Euclidean norm throughout)
  *   orc_pq_*           product-quantised traversal (Algorithm 2's PQDist line; Section "BOA
@@ -801,4 +804,203 @@ void orc_boa_search_wl(const orc_index *ix, const float *queries, int64_t Q,
     free(saved);
     free(active);
     orc_state_free(st);
+}
+
+/* ------------------------------------------------------------------ */
+/* graph construction (Background, "Graph construction")               */
+/* ------------------------------------------------------------------ */
+/*
+ * A Vamana-style build with the threshold pruning the paper adopts: points are inserted in
+ * batches; a beam search over the graph built so far collects candidates for each new point;
+ * a pruning step keeps at most R out-neighbours by the alpha-dominance rule, run once per
+ * attribute threshold with a degree budget of R/|T| each; reverse edges are added, pruning
+ * again where a row overflows.  The paper gives the outline only; what is fixed here:
+ *   - batches are [start, start + size) in index order, size = min(B, points inserted so
+ *     far) (1, 1, 2, 4, ...); every point of a batch searches the graph as it stood before
+ *     the batch; `passes` > 1 repeats the sweep with batches of B over the finished graph
+ *   - candidates of p: the Lb best nodes of an unfiltered beam search at width Lb from the
+ *     entry point (Algorithm 2 with every point valid), plus p's current out-neighbours
+ *   - distances are squared L2 in the fixed-order fp32 of orc_dist2_lanes; candidates are
+ *     ordered by (d2, id); c2 is dominated by a selected c when alpha^2 * d2(c, c2) <=
+ *     d2(p, c2) (alpha^2 rounded once to float, one fp32 multiply)
+ *   - attribute distance of two points = the largest absolute difference of their
+ *     positions (pos[N][m], e.g. rank / N per attribute); threshold pass i takes only
+ *     candidates whose attribute distance is <= thresholds[i], forgets the dominance marks
+ *     of the pass before, and may select R*(i+1)/T - R*i/T more neighbours
+ *   - after a batch every selected edge p -> n asks for n -> p: the requesters of n, in
+ *     ascending id order, at most cap_in of them, those not yet in n's row; if they fit
+ *     they are appended in that order, else n's row is pruned over row + requesters
+ */
+typedef struct {
+    uint32_t id;
+    float d2;
+} orc_cand_t;
+
+static int orc_cand_cmp(const void *a, const void *b)
+{
+    const orc_cand_t *x = (const orc_cand_t *)a, *y = (const orc_cand_t *)b;
+    if (x->d2 != y->d2) return x->d2 < y->d2 ? -1 : 1;
+    return x->id < y->id ? -1 : (x->id > y->id ? 1 : 0);
+}
+
+/* squared distance between two points of the index, fixed-order fp32 */
+static float orc_point_dist2(const orc_index *ix, int64_t a, int64_t b)
+{
+    const int per = (ix->vec_dtype == ORC_U8) ? 16 : 4;
+    const int nchunks = (ix->D + per - 1) / per;
+    float part[8];
+    for (int g = 0; g < 8; ++g) {
+        float acc = 0.0f;
+        for (int c = g; c < nchunks; c += 8)
+            for (int j = 0; j < per && c * per + j < ix->D; ++j) {
+                float diff = orc_elem(ix, a, c * per + j) - orc_elem(ix, b, c * per + j);
+                acc = fmaf(diff, diff, acc);
+            }
+        part[g] = acc;
+    }
+    float a04 = part[0] + part[4], a15 = part[1] + part[5];
+    float a26 = part[2] + part[6], a37 = part[3] + part[7];
+    float e = a04 + a26, o = a15 + a37;
+    return e + o;
+}
+
+static float orc_attr_dist(const float *pos, int m, int64_t a, int64_t b)
+{
+    float d = 0.0f;
+    for (int j = 0; j < m; ++j) {
+        float x = fabsf(pos[a * m + j] - pos[b * m + j]);
+        if (x > d) d = x;
+    }
+    return d;
+}
+
+/* The pruning step.  ids[0..n): candidate ids (any order, repeats and p itself allowed).
+   Writes the selected neighbours, in selection order, to row[0..R), padded with the
+   sentinel.  Returns how many were selected. */
+int orc_prune(const orc_index *ix, const float *pos, int m_pos, int64_t p, const uint32_t *ids, int n,
+              int R, float alpha, const float *thresholds, int T, uint32_t *row)
+{
+    orc_cand_t *c = (orc_cand_t *)malloc((size_t)(n + 1) * sizeof(orc_cand_t));
+    int nc = 0;
+    for (int i = 0; i < n; ++i) {
+        if (ids[i] == ORC_SENTINEL || (int64_t)ids[i] == p) continue;
+        c[nc].id = ids[i];
+        c[nc].d2 = orc_point_dist2(ix, p, ids[i]);
+        nc++;
+    }
+    qsort(c, (size_t)nc, sizeof(orc_cand_t), orc_cand_cmp);
+    int u = 0;                                               /* drop repeats */
+    for (int i = 0; i < nc; ++i)
+        if (u == 0 || c[i].id != c[u - 1].id) c[u++] = c[i];
+    nc = u;
+    uint8_t *sel = (uint8_t *)calloc((size_t)nc + 1, 1), *occ = (uint8_t *)malloc((size_t)nc + 1);
+    const float alpha2 = alpha * alpha;
+    int total = 0;
+    for (int ti = 0; ti < T; ++ti) {
+        int budget = R * (ti + 1) / T - R * ti / T, taken = 0;
+        memset(occ, 0, (size_t)nc + 1);
+        for (int i = 0; i < nc && taken < budget; ++i) {
+            if (sel[i] || occ[i]) continue;
+            if (orc_attr_dist(pos, m_pos, p, c[i].id) > thresholds[ti]) continue;
+            sel[i] = 1; taken++;
+            row[total++] = c[i].id;
+            for (int j = i + 1; j < nc; ++j) {
+                if (sel[j]) continue;
+                float dcc = orc_point_dist2(ix, c[i].id, c[j].id);
+                if (alpha2 * dcc <= c[j].d2) occ[j] = 1;
+            }
+        }
+    }
+    for (int i = total; i < R; ++i) row[i] = ORC_SENTINEL;
+    free(c); free(sel); free(occ);
+    return total;
+}
+
+/* graph: [N][R] output (the index's own graph pointer must be this array: the searches of a
+   batch read it).  Returns the number of batches. */
+int64_t orc_build_graph(orc_index *ix, const float *pos, int m_pos, uint32_t *graph, int R, int Lb,
+                        float alpha, const float *thresholds, int T, int B, int passes, int cap_in)
+{
+    const int64_t N = ix->N;
+    for (int64_t i = 0; i < N * R; ++i) graph[i] = ORC_SENTINEL;
+    ix->graph = graph; ix->R = R;
+    orc_state *st = orc_state_new(ix, Lb);
+    int32_t *full_lo = (int32_t *)malloc((size_t)ix->m * 4), *full_hi = (int32_t *)malloc((size_t)ix->m * 4);
+    for (int j = 0; j < ix->m; ++j) {
+        if (ix->attr_types[j] == ORC_ATTR_F32) { float a = -INFINITY, b = INFINITY; memcpy(&full_lo[j], &a, 4); memcpy(&full_hi[j], &b, 4); }
+        else if (ix->attr_types[j] == ORC_ATTR_SET) { full_lo[j] = 0; full_hi[j] = 1; }
+        else { full_lo[j] = INT32_MIN; full_hi[j] = INT32_MAX; }
+    }
+    float *q = (float *)malloc((size_t)ix->D * sizeof(float));
+    uint32_t *cand = (uint32_t *)malloc((size_t)B * (Lb + R) * sizeof(uint32_t));
+    int *ncand = (int *)malloc((size_t)B * sizeof(int));
+    uint32_t *req = (uint32_t *)malloc((size_t)B * R * 2 * sizeof(uint32_t));
+    uint32_t *tmp = (uint32_t *)malloc((size_t)(R + cap_in + 1) * sizeof(uint32_t));
+    int64_t batches = 0, inserted = 0;
+    for (int pass = 0; pass < passes; ++pass) {
+        int64_t start = 0;
+        while (start < N) {
+            int64_t bsz = pass == 0 ? (inserted < 1 ? 1 : (inserted < B ? inserted : B)) : B;
+            if (start + bsz > N) bsz = N - start;
+            /* (a) candidates from the graph as it stands */
+            for (int64_t b = 0; b < bsz; ++b) {
+                int64_t p = start + b;
+                for (int i = 0; i < ix->D; ++i) q[i] = orc_elem(ix, p, i);
+                orc_beam_init(st, Lb, q, full_lo, full_hi, 1);
+                orc_beam_run_w(st, Lb, q, full_lo, full_hi, 1, (int64_t)8 * Lb + 64, 1);
+                int n = 0;
+                for (int t = 0; t < st->size && t < Lb; ++t) cand[b * (Lb + R) + n++] = st->pool[t].id;
+                ncand[b] = n;
+            }
+            /* (b) prune every batch point over candidates + its current row */
+            for (int64_t b = 0; b < bsz; ++b) {
+                int64_t p = start + b;
+                int n = ncand[b];
+                for (int j = 0; j < R; ++j) cand[b * (Lb + R) + n++] = graph[p * R + j];
+                orc_prune(ix, pos, m_pos, p, cand + b * (Lb + R), n, R, alpha, thresholds, T, graph + p * R);
+            }
+            /* (c) reverse edges, per target in ascending (target, requester) order */
+            int64_t nreq = 0;
+            for (int64_t b = 0; b < bsz; ++b)
+                for (int j = 0; j < R; ++j) {
+                    uint32_t n = graph[(start + b) * R + j];
+                    if (n != ORC_SENTINEL) { req[2 * nreq] = n; req[2 * nreq + 1] = (uint32_t)(start + b); nreq++; }
+                }
+            /* sort the pairs by (target, requester) */
+            uint64_t *keys = (uint64_t *)malloc((size_t)(nreq + 1) * sizeof(uint64_t));
+            for (int64_t i = 0; i < nreq; ++i) keys[i] = ((uint64_t)req[2 * i] << 32) | req[2 * i + 1];
+            for (int64_t i = 1; i < nreq; ++i) {                     /* insertion sort: plain, small */
+                uint64_t k = keys[i]; int64_t j = i;
+                while (j > 0 && keys[j - 1] > k) { keys[j] = keys[j - 1]; j--; }
+                keys[j] = k;
+            }
+            for (int64_t i = 0; i < nreq;) {
+                uint32_t tgt = (uint32_t)(keys[i] >> 32);
+                int64_t e = i;
+                while (e < nreq && (uint32_t)(keys[e] >> 32) == tgt) e++;
+                uint32_t *row = graph + (int64_t)tgt * R;
+                int deg = 0, nm = 0;
+                while (deg < R && row[deg] != ORC_SENTINEL) deg++;
+                for (int64_t r = i; r < e && r < i + cap_in; ++r) {
+                    uint32_t rq = (uint32_t)keys[r];
+                    int have = 0;
+                    for (int j = 0; j < deg; ++j) if (row[j] == rq) have = 1;
+                    if (!have) tmp[deg + nm++] = rq;
+                }
+                if (deg + nm <= R) {
+                    for (int j = 0; j < nm; ++j) row[deg + j] = tmp[deg + j];
+                } else {
+                    for (int j = 0; j < deg; ++j) tmp[j] = row[j];
+                    orc_prune(ix, pos, m_pos, tgt, tmp, deg + nm, R, alpha, thresholds, T, row);
+                }
+                i = e;
+            }
+            free(keys);
+            start += bsz; if (pass == 0) inserted += bsz;
+            batches++;
+        }
+    }
+    free(q); free(cand); free(ncand); free(req); free(tmp); free(full_lo); free(full_hi);
+    orc_state_free(st);
+    return batches;
 }

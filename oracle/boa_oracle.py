@@ -55,6 +55,10 @@ def lib():
         L.orc_uncertain.argtypes = [vp, i32, i32, dbl]
         L.orc_boa_search_wl.argtypes = [vp, vp, i64, vp, vp, i32, vp, i32, dbl, dbl, i32, i32,
                                         i32, i32, i32, C.c_float, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.orc_prune.restype = i32
+        L.orc_prune.argtypes = [vp, vp, i32, i64, vp, i32, i32, C.c_float, vp, i32, vp]
+        L.orc_build_graph.restype = i64
+        L.orc_build_graph.argtypes = [vp, vp, i32, vp, i32, i32, C.c_float, vp, i32, i32, i32, i32]
         L.orc_range_penalty.restype = C.c_float
         L.orc_range_penalty.argtypes = [vp, vp, vp, i64, vp]
         L.orc_state_set_penalty.argtypes = [vp, vp]
@@ -125,6 +129,27 @@ class OracleIndex:
         lo = np.ascontiguousarray(lo, dtype=np.int32)
         hi = np.ascontiguousarray(hi, dtype=np.int32)
         return int(lib().orc_phi(self.h, _p(lo), _p(hi), int(p)))
+
+    # --- graph construction -------------------------------------------------------
+    def prune(self, pos, p, ids, R, alpha=1.2, thresholds=(float("inf"),)):
+        pos = np.ascontiguousarray(pos, dtype=np.float32)
+        ids = np.ascontiguousarray(ids, dtype=np.uint32)
+        th = np.ascontiguousarray(thresholds, dtype=np.float32)
+        row = np.empty(R, dtype=np.uint32)
+        n = lib().orc_prune(self.h, _p(pos), pos.shape[1], int(p), _p(ids), len(ids), int(R), float(alpha),
+                            _p(th), len(th), _p(row))
+        return row, n
+
+    def build_graph(self, pos, R, Lb, alpha=1.2, thresholds=(float("inf"),), B=1024, passes=1, cap_in=64):
+        """Builds the graph into a new array, which becomes this index's graph."""
+        pos = np.ascontiguousarray(pos, dtype=np.float32)
+        th = np.ascontiguousarray(thresholds, dtype=np.float32)
+        g = np.empty((self.N, R), dtype=np.uint32)
+        self._build_pos, self._build_th = pos, th
+        lib().orc_build_graph(self.h, _p(pos), pos.shape[1], _p(g), int(R), int(Lb), float(alpha), _p(th),
+                              len(th), int(B), int(passes), int(cap_in))
+        self.graph, self.R = g, R
+        return g
 
     def range_penalty(self, lo, hi, p, scales):
         lo = np.ascontiguousarray(lo, dtype=np.int32)

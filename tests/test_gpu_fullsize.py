@@ -260,3 +260,36 @@ def test_full_size_long_rows_c5():
     rec_f = recall_against(f["ids"], f["d2"], gt_d2, gt_nv, w.k)
     assert np.nanmean(rec_f) > np.nanmean(rec)                           # the wide fixed beam finds more
     gpu.close()
+
+
+def test_more_than_2_pow_25_points():
+    """Node ids of 26 bits: the table of scored ids has to double its size until 16-bit tags
+    identify an id again, and keys carry ids beyond 2^25.  Tiny vectors (4 floats) and a random
+    degree-4 graph keep the 33.5M-point index small; queries are exact copies of high-numbered
+    points, so the answers come from the top of the id range."""
+    N, D, R, Q, k = (1 << 25) + 8, 4, 4, 64, 5
+    rng = np.random.default_rng(3)
+    x = rng.integers(0, 64, size=(N, D)).astype(np.float32)
+    x[N - 40:] = np.array([200, 210, 220, 230], np.float32) + rng.integers(0, 3, size=(40, D))   # a far-off family
+    attrs = rng.integers(0, 100, size=(N, 1)).astype(np.int32)
+    attrs[N - 40:] = 50
+    graph = rng.integers(0, N, size=(N, R)).astype(np.uint32)
+    graph[:, 0] = (np.arange(N, dtype=np.uint32) + np.uint32(1)) % np.uint32(N)      # a ring keeps it connected
+    graph[0, 1] = N - 1                                                               # reach the top of the range at once
+    graph[N - 40:, 1] = np.arange(N - 41, N - 1, dtype=np.uint32)                     # and walk down from there
+    src = N - 1 - rng.integers(0, 32, size=Q)
+    q = x[src].copy()
+    lo = np.full((Q, 1), 0, np.int32)
+    hi = np.full((Q, 1), 70, np.int32)
+    d = dict(vectors=x, attrs=attrs, attr_types=np.zeros(1, np.int32), graph=graph, queries=q, lo=lo, hi=hi)
+    orc, gpu, g = make_pair(d, entry=0)
+    for mode, widths in (("resume", [16, 64, 256]), ("restart", [16, 128])):
+        o = orc.search(q, lo, hi, k, widths, eps=0.1, mode=mode, dist_mode=1)
+        r = gpu_search(gpu, g, k, widths, mode=mode, eps=0.1)
+        assert (o["ids"] == r["ids"]).all() and (o["d2"].view(np.uint32) == r["d2"].view(np.uint32)).all()
+        assert (o["final_L"] == r["final_L"]).all() and (o["n_expand"] == r["n_expand"]).all()
+        assert (r["n_scored"] >= o["n_scored"]).all()
+    found = r["ids"][r["ids"] != SENTINEL]
+    assert found.size and found.max() >= (1 << 25)
+    assert gpu.device_status() == 0
+    gpu.close()
