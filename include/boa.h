@@ -116,6 +116,41 @@ int boa_index_create(boa_index** out, const void* vectors, int vec_dtype, int64_
                      int64_t entry, void* stream);
 
 /*
+ * Build a proximity graph on the GPU (Background section, "Graph construction": Vamana
+ * insertion -- a beam search over the graph built so far collects candidates for each new
+ * point, a pruning step keeps at most R diverse out-neighbours by the alpha-dominance rule --
+ * with the threshold pruning the paper adopts: the pruning runs once per attribute threshold,
+ * each run with a degree budget of R/T and only over candidates whose attribute distance to
+ * the point is within the threshold, so part of every row links attribute-near points).
+ * Not part of the search hot path; its output is the `graph` argument of boa_index_create.
+ *
+ *   vectors     [N][D] as for boa_index_create
+ *   attr_pos    [N][m_pos] float: where the point sits in each attribute (for instance its
+ *               rank divided by N); the attribute distance of two points is the largest
+ *               absolute difference of their positions
+ *   R, Lb       out-degree and the beamwidth of the build's searches (Lb <= 128, Lb + R <= 256)
+ *   alpha       dominance factor >= 1 on distances (applied squared to squared distances)
+ *   thresholds  HOST array [T], T <= 8, +infinity = every candidate; pass i may add
+ *               R*(i+1)/T - R*i/T neighbours
+ *   B           largest batch; batches are [start, start+size) in index order with size =
+ *               min(B, points inserted so far) (1, 1, 2, 4, ...); every point of a batch
+ *               searches the graph as it stood before the batch
+ *   passes      sweeps over all points (the second and later ones in batches of B)
+ *   cap_in      reverse edges: at most this many requesters (lowest ids first) are
+ *               considered per target and batch (<= 64)
+ *   entry       start node of the build's searches, -1 = the medoid as in boa_index_create
+ *   out_graph   [N][R] device; BOA_NO_ID pads
+ *   n_batches   HOST, may be NULL
+ *
+ * Deterministic: the same inputs give the same graph.  Synchronises `stream`; allocates and
+ * frees its own scratch (a search index over the vectors among it).
+ * Errors: BOA_EINVAL (nulls, sizes out of range), BOA_ENOMEM, BOA_ECUDA.
+ */
+int boa_graph_build(const void* vectors, int vec_dtype, int64_t N, int D, const float* attr_pos, int m_pos,
+                    int R, int Lb, float alpha, const float* thresholds, int T, int B, int passes,
+                    int cap_in, int64_t entry, uint32_t* out_graph, int64_t* n_batches, void* stream);
+
+/*
  * Give the index a product-quantisation codebook (Section "BOA Implementation on a GPU
  * System": PQ codes and quantisation pivots live in GPU memory; a query's distance table
  * holds the distance from each of its subvectors to every centroid of that subspace, and a

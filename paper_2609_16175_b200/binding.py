@@ -79,6 +79,9 @@ def load_library():
     L.boa_last_launch_count.argtypes = [vp]
     L.boa_device_status.restype = i32
     L.boa_device_status.argtypes = [vp, C.POINTER(i32), vp]
+    L.boa_graph_build.restype = i32
+    L.boa_graph_build.argtypes = [vp, i32, i64, i32, vp, i32, i32, i32, C.c_float, C.POINTER(C.c_float), i32, i32,
+                                  i32, i32, i64, vp, C.POINTER(i64), vp]
     L.boa_last_cuda_error.restype = i32
     L.boa_strerror.restype = C.c_char_p
     L.boa_strerror.argtypes = [i32]
@@ -100,6 +103,26 @@ def _dev(t: torch.Tensor, name: str) -> torch.Tensor:
     if not t.is_cuda:
         raise ValueError(f"{name} must be a CUDA tensor")
     return t.contiguous()
+
+
+def build_graph(vectors: torch.Tensor, attr_pos: torch.Tensor, R: int, Lb: int, alpha: float = 1.2,
+                thresholds: Sequence[float] = (float("inf"),), B: int = 1024, passes: int = 1, cap_in: int = 64,
+                entry: int = -1, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """boa_graph_build: returns the [N][R] graph (int32 storage of node ids) on the vectors' device."""
+    lib = load_library()
+    vectors = _dev(vectors, "vectors")
+    attr_pos = _dev(attr_pos, "attr_pos")
+    if attr_pos.dtype != torch.float32 or attr_pos.dim() != 2:
+        raise ValueError("attr_pos must be float32 [N][m]")
+    dt = F32 if vectors.dtype == torch.float32 else U8
+    N, D = vectors.shape
+    out = torch.empty((N, R), dtype=torch.int32, device=vectors.device)
+    th = (C.c_float * len(thresholds))(*[float(t) for t in thresholds])
+    nb = C.c_int64(0)
+    _check(lib.boa_graph_build(vectors.data_ptr(), dt, N, D, attr_pos.data_ptr(), attr_pos.shape[1], R, Lb,
+                               float(alpha), th, len(thresholds), B, passes, cap_in, int(entry), out.data_ptr(),
+                               C.byref(nb), _stream_ptr(stream)), "boa_graph_build")
+    return out
 
 
 class BoaIndex:

@@ -7,8 +7,8 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libboa.so")
-SOURCES = ["boa.cu"]
-DEPS = ["boa.cu", "boa_search.cuh", os.path.join("..", "..", "include", "boa.h")]
+SOURCES = ["boa.cu", "boa_build.cu"]
+DEPS = ["boa.cu", "boa_build.cu", "boa_search.cuh", os.path.join("..", "..", "include", "boa.h")]
 
 
 def nvcc_command(extra=()):

@@ -633,6 +633,10 @@ int boa_index_destroy(boa_index* ix)
 
 int64_t boa_index_entry(const boa_index* ix) { return ix ? ix->entry : -1; }
 
+// For the graph builder in this library (not declared in the public header): the index's own
+// copy of the graph, which the builder fills in while it searches it.
+uint32_t* boa_internal_graph(boa_index* ix) { return ix ? ix->graph : nullptr; }
+
 int boa_set_param(boa_index* ix, int key, double v)
 {
     if (!ix || v != v) return BOA_EINVAL;
