@@ -121,14 +121,15 @@ int boa_index_create(boa_index** out, const void* vectors, int vec_dtype, int64_
  * point, a pruning step keeps at most R diverse out-neighbours by the alpha-dominance rule --
  * with the threshold pruning the paper adopts: the pruning runs once per attribute threshold,
  * each run with a degree budget of R/T and only over candidates whose attribute distance to
- * the point is within the threshold, so part of every row links attribute-near points).
+ * the point is within the threshold, so part of every row links attribute-near points.
+ * Candidates come from one filter-aware search per threshold, filtered to that window).
  * Not part of the search hot path; its output is the `graph` argument of boa_index_create.
  *
  *   vectors     [N][D] as for boa_index_create
  *   attr_pos    [N][m_pos] float: where the point sits in each attribute (for instance its
  *               rank divided by N); the attribute distance of two points is the largest
  *               absolute difference of their positions
- *   R, Lb       out-degree and the beamwidth of the build's searches (Lb <= 128, Lb + R <= 256)
+ *   R, Lb       out-degree and the beamwidth of the build's searches (Lb <= 128, T*Lb + R <= 256)
  *   alpha       dominance factor >= 1 on distances (applied squared to squared distances)
  *   thresholds  HOST array [T], T <= 8, +infinity = every candidate; pass i may add
  *               R*(i+1)/T - R*i/T neighbours

@@ -818,8 +818,10 @@ void orc_boa_search_wl(const orc_index *ix, const float *queries, int64_t Q,
  *   - batches are [start, start + size) in index order, size = min(B, points inserted so
  *     far) (1, 1, 2, 4, ...); every point of a batch searches the graph as it stood before
  *     the batch; `passes` > 1 repeats the sweep with batches of B over the finished graph
- *   - candidates of p: the Lb best nodes of an unfiltered beam search at width Lb from the
- *     entry point (Algorithm 2 with every point valid), plus p's current out-neighbours
+ *   - candidates of p: for every threshold t one filter-aware beam search (Algorithm 2) at
+ *     width Lb from the entry point whose predicate is "attribute position within t of p's in
+ *     every attribute" (bounds pos - t and pos + t, one fp32 operation each; t = +infinity is the
+ *     unfiltered search): its filter-valid results, at most Lb; plus p's current out-neighbours
  *   - distances are squared L2 in the fixed-order fp32 of orc_dist2_lanes; candidates are
  *     ordered by (d2, id); c2 is dominated by a selected c when alpha^2 * d2(c, c2) <=
  *     d2(p, c2) (alpha^2 rounded once to float, one fp32 multiply)
@@ -924,15 +926,19 @@ int64_t orc_build_graph(orc_index *ix, const float *pos, int m_pos, uint32_t *gr
     const int64_t N = ix->N;
     for (int64_t i = 0; i < N * R; ++i) graph[i] = ORC_SENTINEL;
     ix->graph = graph; ix->R = R;
-    orc_state *st = orc_state_new(ix, Lb);
-    int32_t *full_lo = (int32_t *)malloc((size_t)ix->m * 4), *full_hi = (int32_t *)malloc((size_t)ix->m * 4);
-    for (int j = 0; j < ix->m; ++j) {
-        if (ix->attr_types[j] == ORC_ATTR_F32) { float a = -INFINITY, b = INFINITY; memcpy(&full_lo[j], &a, 4); memcpy(&full_hi[j], &b, 4); }
-        else if (ix->attr_types[j] == ORC_ATTR_SET) { full_lo[j] = 0; full_hi[j] = 1; }
-        else { full_lo[j] = INT32_MIN; full_hi[j] = INT32_MAX; }
-    }
+    /* the build's searches see the attribute positions as float attribute columns */
+    orc_index six = *ix;
+    int32_t *ftypes = (int32_t *)malloc((size_t)m_pos * sizeof(int32_t));
+    for (int j = 0; j < m_pos; ++j) ftypes[j] = ORC_ATTR_F32;
+    six.attrs = (const int32_t *)pos; six.attr_types = ftypes; six.m = m_pos;
+    six.metric = 0; six.unit = NULL; six.pq_M = 0;
+    orc_state *st = orc_state_new(&six, Lb);
+    int32_t *full_lo = (int32_t *)malloc((size_t)m_pos * 4), *full_hi = (int32_t *)malloc((size_t)m_pos * 4);
     float *q = (float *)malloc((size_t)ix->D * sizeof(float));
-    uint32_t *cand = (uint32_t *)malloc((size_t)B * (Lb + R) * sizeof(uint32_t));
+    const int CW = T * Lb + R;                                 /* candidate slots per point */
+    uint32_t *cand = (uint32_t *)malloc((size_t)B * CW * sizeof(uint32_t));
+    uint32_t *res_ids = (uint32_t *)malloc((size_t)Lb * sizeof(uint32_t));
+    float *res_d2 = (float *)malloc((size_t)Lb * sizeof(float));
     int *ncand = (int *)malloc((size_t)B * sizeof(int));
     uint32_t *req = (uint32_t *)malloc((size_t)B * R * 2 * sizeof(uint32_t));
     uint32_t *tmp = (uint32_t *)malloc((size_t)(R + cap_in + 1) * sizeof(uint32_t));
@@ -946,18 +952,25 @@ int64_t orc_build_graph(orc_index *ix, const float *pos, int m_pos, uint32_t *gr
             for (int64_t b = 0; b < bsz; ++b) {
                 int64_t p = start + b;
                 for (int i = 0; i < ix->D; ++i) q[i] = orc_elem(ix, p, i);
-                orc_beam_init(st, Lb, q, full_lo, full_hi, 1);
-                orc_beam_run_w(st, Lb, q, full_lo, full_hi, 1, (int64_t)8 * Lb + 64, 1);
                 int n = 0;
-                for (int t = 0; t < st->size && t < Lb; ++t) cand[b * (Lb + R) + n++] = st->pool[t].id;
+                for (int ti = 0; ti < T; ++ti) {
+                    for (int j = 0; j < m_pos; ++j) {
+                        float l = pos[p * m_pos + j] - thresholds[ti], h = pos[p * m_pos + j] + thresholds[ti];
+                        memcpy(&full_lo[j], &l, 4); memcpy(&full_hi[j], &h, 4);
+                    }
+                    orc_beam_init(st, Lb, q, full_lo, full_hi, 1);
+                    orc_beam_run_w(st, Lb, q, full_lo, full_hi, 1, (int64_t)8 * Lb + 64, 1);
+                    int got = orc_beam_result(st, Lb, res_ids, res_d2);
+                    for (int t = 0; t < got; ++t) cand[b * CW + n++] = res_ids[t];
+                }
                 ncand[b] = n;
             }
             /* (b) prune every batch point over candidates + its current row */
             for (int64_t b = 0; b < bsz; ++b) {
                 int64_t p = start + b;
                 int n = ncand[b];
-                for (int j = 0; j < R; ++j) cand[b * (Lb + R) + n++] = graph[p * R + j];
-                orc_prune(ix, pos, m_pos, p, cand + b * (Lb + R), n, R, alpha, thresholds, T, graph + p * R);
+                for (int j = 0; j < R; ++j) cand[b * CW + n++] = graph[p * R + j];
+                orc_prune(ix, pos, m_pos, p, cand + b * CW, n, R, alpha, thresholds, T, graph + p * R);
             }
             /* (c) reverse edges, per target in ascending (target, requester) order */
             int64_t nreq = 0;
@@ -1001,6 +1014,7 @@ int64_t orc_build_graph(orc_index *ix, const float *pos, int m_pos, uint32_t *gr
         }
     }
     free(q); free(cand); free(ncand); free(req); free(tmp); free(full_lo); free(full_hi);
+    free(res_ids); free(res_d2); free(ftypes);
     orc_state_free(st);
     return batches;
 }

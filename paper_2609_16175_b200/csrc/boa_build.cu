@@ -2,8 +2,9 @@
 // per attribute threshold (the paper's Background section, "Graph construction").  Not part of
 // the search hot path; it produces the graph boa_index_create takes.  sm_100a only.
 //
-// Per batch of new points: (a) the library's own beam search over the graph built so far
-// collects candidates for every point of the batch, (b) one warp per point prunes candidates +
+// Per batch of new points: (a) the library's own filter-aware beam search over the graph built
+// so far collects candidates for every point of the batch, once per attribute threshold with
+// the predicate "attribute position within the threshold of the point's own", (b) one warp per point prunes candidates +
 // current row down to R neighbours, (c) every selected edge p -> n asks for n -> p: the
 // requests are sorted by (target, requester) and one warp per target appends them or, when the
 // row overflows, prunes row + requesters.  Everything that decides the result is fixed
@@ -172,8 +173,8 @@ __device__ void prune_point(const BuildParams& bp, int64_t p, const uint32_t* ca
     __syncwarp();
 }
 
-// (b) one warp per batch point: candidates of the search + the point's current row
-__global__ void prune_batch_kernel(BuildParams bp, int64_t start, int bsz, const uint32_t* cand_ids, int Lb)
+// (b) one warp per batch point: candidates of the T searches + the point's current row
+__global__ void prune_batch_kernel(BuildParams bp, int64_t start, int bsz, const uint32_t* cand_ids, int Lb, int B)
 {
     __shared__ unsigned long long keys[kMaxCand];
     __shared__ uint32_t cand[kMaxCand];
@@ -182,10 +183,22 @@ __global__ void prune_batch_kernel(BuildParams bp, int64_t start, int bsz, const
     for (int b = blockIdx.x; b < bsz; b += gridDim.x) {
         const int64_t p = start + b;
         uint32_t* row = bp.graph + (size_t)p * bp.R;
-        for (int i = lane; i < Lb; i += 32) cand[i] = cand_ids[(size_t)b * Lb + i];
-        for (int i = lane; i < bp.R; i += 32) cand[Lb + i] = row[i];
+        for (int ti = 0; ti < bp.T; ++ti)
+            for (int i = lane; i < Lb; i += 32) cand[ti * Lb + i] = cand_ids[((size_t)ti * B + b) * Lb + i];
+        for (int i = lane; i < bp.R; i += 32) cand[bp.T * Lb + i] = row[i];
         __syncwarp();
-        prune_point(bp, p, cand, Lb + bp.R, keys, flags, row, lane);
+        prune_point(bp, p, cand, bp.T * Lb + bp.R, keys, flags, row, lane);
+    }
+}
+
+// bounds of the build's searches: lo = pos - t, hi = pos + t per attribute (one fp32 operation each)
+__global__ void window_bounds_kernel(const float* pos, int m, int64_t start, int bsz, float t, float* lo, float* hi)
+{
+    const int64_t n = (int64_t)bsz * m;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const float v = pos[start * m + i];
+        lo[i] = __fsub_rn(v, t);
+        hi[i] = __fadd_rn(v, t);
     }
 }
 
@@ -281,12 +294,13 @@ extern "C" int boa_graph_build(const void* vectors, int vec_dtype, int64_t N, in
     if (N < 1 || R < 1 || R > BOA_MAX_DEGREE || Lb < 1 || Lb > 128 || T < 1 || T > 8 || m_pos < 1 || m_pos > BOA_MAX_ATTRS)
         return BOA_EINVAL;
     if (B < 1 || B > (1 << 20) || passes < 1 || passes > 4 || cap_in < 1 || cap_in > 64 || !(alpha >= 1.0f)) return BOA_EINVAL;
-    if (Lb + R > kMaxCand || R + cap_in > kMaxCand) return BOA_EINVAL;
+    if (T * Lb + R > kMaxCand || R + cap_in > kMaxCand) return BOA_EINVAL;
     if (vec_dtype != BOA_F32 && vec_dtype != BOA_U8) return BOA_EINVAL;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     int rc = BOA_OK;
     boa_index* ix = nullptr;
-    int32_t *zeros = nullptr, *lo0 = nullptr;
+    float *wlo = nullptr, *whi = nullptr;
+    int types[BOA_MAX_ATTRS];
     uint32_t *empty = nullptr, *cand_ids = nullptr, *heads = nullptr, *n_heads = nullptr;
     float *cand_d = nullptr, *qf = nullptr;
     unsigned long long *req = nullptr, *req_sorted = nullptr;
@@ -294,22 +308,20 @@ extern "C" int boa_graph_build(const void* vectors, int vec_dtype, int64_t N, in
     size_t cub_bytes = 0;
     int64_t batches = 0, inserted = 0;
     int sms = 0, dev = 0;
-    const int types[1] = {BOA_ATTR_I32};
     BuildParams bp;
+    for (int j = 0; j < BOA_MAX_ATTRS; ++j) types[j] = BOA_ATTR_F32;
 
     BUILD_CUDA(cudaGetDevice(&dev));
     BUILD_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    BUILD_CUDA(cudaMalloc(&zeros, (size_t)N * sizeof(int32_t)));
-    BUILD_CUDA(cudaMemsetAsync(zeros, 0, (size_t)N * sizeof(int32_t), st));
     BUILD_CUDA(cudaMalloc(&empty, (size_t)N * R * sizeof(uint32_t)));
     fill_u32_kernel<<<sms * 8, 256, 0, st>>>(empty, N * (int64_t)R, kNone);
     BUILD_CUDA(cudaGetLastError());
-    // every point is valid for the searches of the build: one attribute, always 0, range [0, 0]
-    rc = boa_index_create(&ix, vectors, vec_dtype, N, D, zeros, types, 1, empty, R, entry, st);
+    // the build's searches see the attribute positions as float attribute columns
+    rc = boa_index_create(&ix, vectors, vec_dtype, N, D, attr_pos, types, m_pos, empty, R, entry, st);
     if (rc != BOA_OK) goto done;
-    BUILD_CUDA(cudaMalloc(&lo0, (size_t)B * sizeof(int32_t)));
-    BUILD_CUDA(cudaMemsetAsync(lo0, 0, (size_t)B * sizeof(int32_t), st));
-    BUILD_CUDA(cudaMalloc(&cand_ids, (size_t)B * Lb * sizeof(uint32_t)));
+    BUILD_CUDA(cudaMalloc(&wlo, (size_t)B * m_pos * sizeof(float)));
+    BUILD_CUDA(cudaMalloc(&whi, (size_t)B * m_pos * sizeof(float)));
+    BUILD_CUDA(cudaMalloc(&cand_ids, (size_t)T * B * Lb * sizeof(uint32_t)));
     BUILD_CUDA(cudaMalloc(&cand_d, (size_t)B * Lb * sizeof(float)));
     BUILD_CUDA(cudaMalloc(&req, (size_t)B * R * sizeof(unsigned long long)));
     BUILD_CUDA(cudaMalloc(&req_sorted, (size_t)B * R * sizeof(unsigned long long)));
@@ -336,7 +348,8 @@ extern "C" int boa_graph_build(const void* vectors, int vec_dtype, int64_t N, in
         while (start < N) {
             int64_t bsz = pass == 0 ? (inserted < 1 ? 1 : (inserted < B ? inserted : B)) : B;
             if (start + bsz > N) bsz = N - start;
-            // (a) candidates: the beam of an unfiltered search at width Lb over the graph so far
+            // (a) candidates: per threshold, the filter-valid results of a search at width Lb over the
+            // graph so far whose ranges are the point's own attribute positions +- the threshold
             const float* q = reinterpret_cast<const float*>(vectors) + (size_t)start * D;
             if (vec_dtype == BOA_U8) {
                 bytes_to_float_kernel<<<sms * 4, 256, 0, st>>>(reinterpret_cast<const uint8_t*>(vectors) + (size_t)start * D,
@@ -344,10 +357,14 @@ extern "C" int boa_graph_build(const void* vectors, int vec_dtype, int64_t N, in
                 BUILD_CUDA(cudaGetLastError());
                 q = qf;
             }
-            rc = boa_search(ix, q, bsz, lo0, lo0, Lb, Lb, Lb, cand_ids, cand_d, st);
-            if (rc != BOA_OK) goto done;
+            for (int ti = 0; ti < T; ++ti) {
+                window_bounds_kernel<<<sms, 256, 0, st>>>(attr_pos, m_pos, start, (int)bsz, thresholds[ti], wlo, whi);
+                BUILD_CUDA(cudaGetLastError());
+                rc = boa_search(ix, q, bsz, wlo, whi, Lb, Lb, Lb, cand_ids + (size_t)ti * B * Lb, cand_d, st);
+                if (rc != BOA_OK) goto done;
+            }
             // (b) prune every point of the batch
-            prune_batch_kernel<<<(unsigned)(bsz < sms * 16 ? bsz : sms * 16), 32, 0, st>>>(bp, start, (int)bsz, cand_ids, Lb);
+            prune_batch_kernel<<<(unsigned)(bsz < sms * 16 ? bsz : sms * 16), 32, 0, st>>>(bp, start, (int)bsz, cand_ids, Lb, B);
             BUILD_CUDA(cudaGetLastError());
             // (c) reverse edges
             {
@@ -373,7 +390,7 @@ extern "C" int boa_graph_build(const void* vectors, int vec_dtype, int64_t N, in
 done:
     if (rc != BOA_OK) cudaStreamSynchronize(st);
     if (ix) boa_index_destroy(ix);
-    cudaFree(zeros); cudaFree(empty); cudaFree(lo0); cudaFree(cand_ids); cudaFree(cand_d); cudaFree(req);
+    cudaFree(wlo); cudaFree(whi); cudaFree(empty); cudaFree(cand_ids); cudaFree(cand_d); cudaFree(req);
     cudaFree(req_sorted); cudaFree(heads); cudaFree(n_heads); cudaFree(qf); cudaFree(cub_tmp);
     return rc;
 }
