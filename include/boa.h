@@ -127,11 +127,13 @@ int boa_index_create(boa_index** out, const void* vectors, int vec_dtype, int64_
  *
  *   vectors     [N][D] as for boa_index_create
  *   attr_pos    [N][m_pos] float: where the point sits in each attribute (for instance its
- *               rank divided by N); the attribute distance of two points is the largest
+ *               rank divided by N); the distance of two points in attribute j is the
  *               absolute difference of their positions
  *   R, Lb       out-degree and the beamwidth of the build's searches (Lb <= 128, T*Lb + R <= 256)
  *   alpha       dominance factor >= 1 on distances (applied squared to squared distances)
- *   thresholds  HOST array [T], T <= 8, +infinity = every candidate; pass i may add
+ *   thresholds  HOST array [T][m_pos], T <= 8: pass i admits the candidates whose distance in
+ *               every attribute j is <= thresholds[i][j] (+infinity leaves the attribute
+ *               free; a row of +infinity is the plain Vamana pass) and may add
  *               R*(i+1)/T - R*i/T neighbours
  *   B           largest batch; batches are [start, start+size) in index order with size =
  *               min(B, points inserted so far) (1, 1, 2, 4, ...); every point of a batch

@@ -818,17 +818,21 @@ void orc_boa_search_wl(const orc_index *ix, const float *queries, int64_t Q,
  *   - batches are [start, start + size) in index order, size = min(B, points inserted so
  *     far) (1, 1, 2, 4, ...); every point of a batch searches the graph as it stood before
  *     the batch; `passes` > 1 repeats the sweep with batches of B over the finished graph
+ *   - a threshold is a vector t[0..m) over the attributes (thresholds[T][m]); t[j] = +infinity
+ *     leaves attribute j free
  *   - candidates of p: for every threshold t one filter-aware beam search (Algorithm 2) at
- *     width Lb from the entry point whose predicate is "attribute position within t of p's in
- *     every attribute" (bounds pos - t and pos + t, one fp32 operation each; t = +infinity is the
- *     unfiltered search): its filter-valid results, at most Lb; plus p's current out-neighbours
+ *     width Lb from the entry point whose predicate is "attribute position j within t[j] of
+ *     p's, for every j" (bounds pos - t[j] and pos + t[j], one fp32 operation each; all
+ *     +infinity is the unfiltered search): its filter-valid results, at most Lb; plus p's
+ *     current out-neighbours
  *   - distances are squared L2 in the fixed-order fp32 of orc_dist2_lanes; candidates are
  *     ordered by (d2, id); c2 is dominated by a selected c when alpha^2 * d2(c, c2) <=
  *     d2(p, c2) (alpha^2 rounded once to float, one fp32 multiply)
- *   - attribute distance of two points = the largest absolute difference of their
+ *   - attribute distance of two points in attribute j = the absolute difference of their
  *     positions (pos[N][m], e.g. rank / N per attribute); threshold pass i takes only
- *     candidates whose attribute distance is <= thresholds[i], forgets the dominance marks
- *     of the pass before, and may select R*(i+1)/T - R*i/T more neighbours
+ *     candidates whose capped distance max(dist_j - thresholds[i][j], 0) is zero in every
+ *     attribute, forgets the dominance marks of the pass before, and may select
+ *     R*(i+1)/T - R*i/T more neighbours
  *   - after a batch every selected edge p -> n asks for n -> p: the requesters of n, in
  *     ascending id order, at most cap_in of them, those not yet in n's row; if they fit
  *     they are appended in that order, else n's row is pruned over row + requesters
@@ -866,14 +870,14 @@ static float orc_point_dist2(const orc_index *ix, int64_t a, int64_t b)
     return e + o;
 }
 
-static float orc_attr_dist(const float *pos, int m, int64_t a, int64_t b)
+/* 1 when b is within threshold vector t of a in every attribute */
+static int orc_attr_within(const float *pos, int m, int64_t a, int64_t b, const float *t)
 {
-    float d = 0.0f;
     for (int j = 0; j < m; ++j) {
         float x = fabsf(pos[a * m + j] - pos[b * m + j]);
-        if (x > d) d = x;
+        if (x > t[j]) return 0;
     }
-    return d;
+    return 1;
 }
 
 /* The pruning step.  ids[0..n): candidate ids (any order, repeats and p itself allowed).
@@ -903,7 +907,7 @@ int orc_prune(const orc_index *ix, const float *pos, int m_pos, int64_t p, const
         memset(occ, 0, (size_t)nc + 1);
         for (int i = 0; i < nc && taken < budget; ++i) {
             if (sel[i] || occ[i]) continue;
-            if (orc_attr_dist(pos, m_pos, p, c[i].id) > thresholds[ti]) continue;
+            if (!orc_attr_within(pos, m_pos, p, c[i].id, thresholds + (size_t)ti * m_pos)) continue;
             sel[i] = 1; taken++;
             row[total++] = c[i].id;
             for (int j = i + 1; j < nc; ++j) {
@@ -955,7 +959,8 @@ int64_t orc_build_graph(orc_index *ix, const float *pos, int m_pos, uint32_t *gr
                 int n = 0;
                 for (int ti = 0; ti < T; ++ti) {
                     for (int j = 0; j < m_pos; ++j) {
-                        float l = pos[p * m_pos + j] - thresholds[ti], h = pos[p * m_pos + j] + thresholds[ti];
+                        float tj = thresholds[(size_t)ti * m_pos + j];
+                        float l = pos[p * m_pos + j] - tj, h = pos[p * m_pos + j] + tj;
                         memcpy(&full_lo[j], &l, 4); memcpy(&full_hi[j], &h, 4);
                     }
                     orc_beam_init(st, Lb, q, full_lo, full_hi, 1);

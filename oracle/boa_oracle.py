@@ -131,10 +131,17 @@ class OracleIndex:
         return int(lib().orc_phi(self.h, _p(lo), _p(hi), int(p)))
 
     # --- graph construction -------------------------------------------------------
+    @staticmethod
+    def _threshold_rows(thresholds, m):
+        """[T][m] float32: a scalar threshold applies to every attribute."""
+        rows = [[float(t)] * m if np.isscalar(t) else [float(x) for x in t] for t in thresholds]
+        assert all(len(r) == m for r in rows)
+        return np.ascontiguousarray(rows, dtype=np.float32)
+
     def prune(self, pos, p, ids, R, alpha=1.2, thresholds=(float("inf"),)):
         pos = np.ascontiguousarray(pos, dtype=np.float32)
         ids = np.ascontiguousarray(ids, dtype=np.uint32)
-        th = np.ascontiguousarray(thresholds, dtype=np.float32)
+        th = self._threshold_rows(thresholds, pos.shape[1])
         row = np.empty(R, dtype=np.uint32)
         n = lib().orc_prune(self.h, _p(pos), pos.shape[1], int(p), _p(ids), len(ids), int(R), float(alpha),
                             _p(th), len(th), _p(row))
@@ -143,7 +150,7 @@ class OracleIndex:
     def build_graph(self, pos, R, Lb, alpha=1.2, thresholds=(float("inf"),), B=1024, passes=1, cap_in=64):
         """Builds the graph into a new array, which becomes this index's graph."""
         pos = np.ascontiguousarray(pos, dtype=np.float32)
-        th = np.ascontiguousarray(thresholds, dtype=np.float32)
+        th = self._threshold_rows(thresholds, pos.shape[1])
         g = np.empty((self.N, R), dtype=np.uint32)
         self._build_pos, self._build_th = pos, th
         lib().orc_build_graph(self.h, _p(pos), pos.shape[1], _p(g), int(R), int(Lb), float(alpha), _p(th),

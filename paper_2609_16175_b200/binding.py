@@ -106,9 +106,11 @@ def _dev(t: torch.Tensor, name: str) -> torch.Tensor:
 
 
 def build_graph(vectors: torch.Tensor, attr_pos: torch.Tensor, R: int, Lb: int, alpha: float = 1.2,
-                thresholds: Sequence[float] = (float("inf"),), B: int = 1024, passes: int = 1, cap_in: int = 64,
+                thresholds: Sequence = (float("inf"),), B: int = 1024, passes: int = 1, cap_in: int = 64,
                 entry: int = -1, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
-    """boa_graph_build: returns the [N][R] graph (int32 storage of node ids) on the vectors' device."""
+    """boa_graph_build: returns the [N][R] graph (int32 storage of node ids) on the vectors' device.
+    Every entry of `thresholds` is one number (the same threshold in every attribute) or a
+    sequence of one number per attribute."""
     lib = load_library()
     vectors = _dev(vectors, "vectors")
     attr_pos = _dev(attr_pos, "attr_pos")
@@ -117,7 +119,14 @@ def build_graph(vectors: torch.Tensor, attr_pos: torch.Tensor, R: int, Lb: int, 
     dt = F32 if vectors.dtype == torch.float32 else U8
     N, D = vectors.shape
     out = torch.empty((N, R), dtype=torch.int32, device=vectors.device)
-    th = (C.c_float * len(thresholds))(*[float(t) for t in thresholds])
+    m_pos = attr_pos.shape[1]
+    flat = []
+    for t in thresholds:
+        row = [float(t)] * m_pos if isinstance(t, (int, float)) else [float(x) for x in t]
+        if len(row) != m_pos:
+            raise ValueError("a threshold needs one value per attribute")
+        flat += row
+    th = (C.c_float * len(flat))(*flat)
     nb = C.c_int64(0)
     _check(lib.boa_graph_build(vectors.data_ptr(), dt, N, D, attr_pos.data_ptr(), attr_pos.shape[1], R, Lb,
                                float(alpha), th, len(thresholds), B, passes, cap_in, int(entry), out.data_ptr(),

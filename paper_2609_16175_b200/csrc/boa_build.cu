@@ -42,7 +42,7 @@ struct BuildParams {
     uint32_t* graph;          // [N][R] the graph being built (the search index's own copy)
     int R, T;
     float alpha2;
-    float thr[8];
+    float thr[8][BOA_MAX_ATTRS];   // [T][m_pos] per-attribute thresholds
 };
 
 // Squared L2 distance of two rows by one 8-lane group (g = lane & 7), in the fixed fp32 order of
@@ -81,14 +81,12 @@ __device__ __forceinline__ float group_dist2(const uint8_t* a, const uint8_t* b,
     return acc;
 }
 
-__device__ __forceinline__ float attr_dist(const float* pos, int m, int64_t a, int64_t b)
+// b within the threshold vector t of a in every attribute
+__device__ __forceinline__ bool attr_within(const float* pos, int m, int64_t a, int64_t b, const float* t)
 {
-    float d = 0.0f;
-    for (int j = 0; j < m; ++j) {
-        const float x = fabsf(pos[a * m + j] - pos[b * m + j]);
-        d = x > d ? x : d;
-    }
-    return d;
+    bool ok = true;
+    for (int j = 0; j < m; ++j) ok = ok && !(fabsf(pos[a * m + j] - pos[b * m + j]) > t[j]);
+    return ok;
 }
 
 // Warp-wide bitonic sort of n <= kMaxCand 64-bit keys in shared memory (ascending); slots
@@ -152,7 +150,7 @@ __device__ void prune_point(const BuildParams& bp, int64_t p, const uint32_t* ca
         for (int i = 0; i < nc && taken < budget; ++i) {
             if (flags[i]) continue;                                       // selected or dominated (warp-uniform)
             const uint32_t ci = (uint32_t)keys[i];
-            if (attr_dist(bp.pos, bp.m_pos, p, ci) > bp.thr[ti]) continue;
+            if (!attr_within(bp.pos, bp.m_pos, p, ci, bp.thr[ti])) continue;
             if (lane == 0) { flags[i] = 1; row[total] = ci; }
             total++; taken++;
             const uint8_t* xc = bp.vec + (size_t)ci * bp.row_bytes;
@@ -191,12 +189,16 @@ __global__ void prune_batch_kernel(BuildParams bp, int64_t start, int bsz, const
     }
 }
 
-// bounds of the build's searches: lo = pos - t, hi = pos + t per attribute (one fp32 operation each)
-__global__ void window_bounds_kernel(const float* pos, int m, int64_t start, int bsz, float t, float* lo, float* hi)
+// bounds of the build's searches: lo = pos - t[j], hi = pos + t[j] per attribute j (one fp32 operation each)
+struct ThresholdRow { float t[BOA_MAX_ATTRS]; };
+__global__ void window_bounds_kernel(const float* pos, int m, int64_t start, int bsz, ThresholdRow tr, float* lo, float* hi)
 {
     const int64_t n = (int64_t)bsz * m;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
         const float v = pos[start * m + i];
+        float t = tr.t[0];
+#pragma unroll
+        for (int j = 1; j < BOA_MAX_ATTRS; ++j) t = (int)(i % m) == j ? tr.t[j] : t;
         lo[i] = __fsub_rn(v, t);
         hi[i] = __fadd_rn(v, t);
     }
@@ -341,7 +343,8 @@ extern "C" int boa_graph_build(const void* vectors, int vec_dtype, int64_t N, in
     bp.R = R;
     bp.T = T;
     bp.alpha2 = alpha * alpha;
-    for (int i = 0; i < 8; ++i) bp.thr[i] = i < T ? thresholds[i] : INFINITY;
+    for (int i = 0; i < 8; ++i)
+        for (int j = 0; j < BOA_MAX_ATTRS; ++j) bp.thr[i][j] = i < T && j < m_pos ? thresholds[(size_t)i * m_pos + j] : INFINITY;
 
     for (int pass = 0; pass < passes; ++pass) {
         int64_t start = 0;
@@ -358,7 +361,9 @@ extern "C" int boa_graph_build(const void* vectors, int vec_dtype, int64_t N, in
                 q = qf;
             }
             for (int ti = 0; ti < T; ++ti) {
-                window_bounds_kernel<<<sms, 256, 0, st>>>(attr_pos, m_pos, start, (int)bsz, thresholds[ti], wlo, whi);
+                ThresholdRow tr;
+                for (int j = 0; j < BOA_MAX_ATTRS; ++j) tr.t[j] = bp.thr[ti][j];
+                window_bounds_kernel<<<sms, 256, 0, st>>>(attr_pos, m_pos, start, (int)bsz, tr, wlo, whi);
                 BUILD_CUDA(cudaGetLastError());
                 rc = boa_search(ix, q, bsz, wlo, whi, Lb, Lb, Lb, cand_ids + (size_t)ti * B * Lb, cand_d, st);
                 if (rc != BOA_OK) goto done;

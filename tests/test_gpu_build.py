@@ -36,6 +36,8 @@ def _build_both(w, seed, **kw):
     ("c2", C2.scaled(3000, 20, name="c2_b"), dict(R=16, Lb=32, alpha=1.2, B=128, passes=1)),
     ("c2t", C2.scaled(4000, 20, name="c2_bt"), dict(R=24, Lb=48, alpha=1.2, thresholds=(INF, 0.2, 0.05), B=256, passes=2)),
     ("c3", C3.scaled(3000, 20, name="c3_b"), dict(R=16, Lb=32, alpha=1.3, thresholds=(INF, 0.1), B=64, passes=1)),
+    ("c3v", C3.scaled(3000, 20, name="c3_bv"), dict(R=24, Lb=40, alpha=1.2, B=128, passes=2,
+                                                    thresholds=(INF, (0.1, INF, INF), (INF, 0.05, 0.2)))),
     ("c4", C4.scaled(3000, 20, name="c4_b"), dict(R=32, Lb=40, alpha=1.2, thresholds=(INF, 0.15), B=200, passes=2, cap_in=8)),
 ], ids=lambda c: c[0])
 def test_gpu_builds_the_oracles_graph(case):
@@ -47,35 +49,56 @@ def test_gpu_builds_the_oracles_graph(case):
     assert (gg[real] < w.N).all() and real.sum(1).min() >= 1
 
 
+def test_search_parity_over_the_oracles_built_graph():
+    """The graph the oracle's builder made (equal to the library's, checked first) handed to both
+    searches: the filter-aware search agrees bit for bit over a threshold-pruned graph too."""
+    from paper_2609_16175_b200 import BoaIndex
+    from tests.helpers import assert_bit_parity, gpu_search, to_gpu
+    w = C2.scaled(5000, 60, name="c2_bs")
+    d, pos, _, go, gg = _build_both(w, seed=53, R=24, Lb=48, alpha=1.2, thresholds=(INF, 0.2, 0.05), B=512, passes=1)
+    assert (go == gg).all()
+    d["graph"] = go
+    t = to_gpu(d)
+    gpu = BoaIndex(t["vectors"], t["attrs"], d["attr_types"].tolist(), t["graph"])
+    orc = OracleIndex(d["vectors"], d["attrs"], d["attr_types"], go)
+    o = orc.search(d["queries"], d["lo"], d["hi"], w.k, [16, 64, 256], mode="resume", dist_mode=1)
+    r = gpu_search(gpu, t, w.k, [16, 64, 256], mode="resume")
+    assert_bit_parity(o, r, "search over a built graph")
+    gpu.close()
+
+
 def test_built_graph_serves_the_search():
     """A graph built by the library, handed to boa_index_create: an unfiltered search finds the
-    true neighbours, a filtered one returns valid points, and it agrees with the oracle's
-    search over the same graph."""
+    true neighbours and a filtered one finds more of them than over a graph built without the
+    attribute thresholds (what the threshold passes are for)."""
     from paper_2609_16175_b200 import BoaIndex, build_graph
     from boa_synth.groundtruth import filtered_topk, recall_against
-    from tests.helpers import assert_bit_parity, gpu_search, to_gpu
+    from tests.helpers import to_gpu
     w = C2.scaled(60_000, 400, name="c2_built")
     d = make_workload(w, seed=52, with_graph=False)
     pos = _positions(d["attrs"], d["attr_types"])
     dev = torch.device("cuda:0")
-    g = build_graph(torch.from_numpy(d["vectors"]).to(dev), torch.from_numpy(pos).to(dev), R=32, Lb=64, alpha=1.2,
-                    thresholds=(INF, 0.3, 0.05), B=2048, passes=2)
-    d["graph"] = g.cpu().numpy().view(np.uint32)
+    d["graph"] = np.zeros((w.N, 1), np.uint32)
     t = to_gpu(d)
-    gpu = BoaIndex(t["vectors"], t["attrs"], d["attr_types"].tolist(), t["graph"])
-    orc = OracleIndex(d["vectors"], d["attrs"], d["attr_types"], d["graph"])
-    o = orc.search(d["queries"][:60], d["lo"][:60], d["hi"][:60], w.k, [16, 64, 256], mode="resume", dist_mode=1)
-    r = gpu_search(gpu, t, w.k, [16, 64, 256], mode="resume", sel=slice(0, 60))
-    assert_bit_parity(o, r, "search over a built graph")
     full_lo = torch.full_like(t["lo"], -2 ** 31)
     full_hi = torch.full_like(t["hi"], 2 ** 31 - 1)
-    gpu.set_schedule([64]); gpu.set_param("mode", 0)
-    ids, d2 = gpu.search(t["queries"], full_lo, full_hi, w.k, 64, 64)
-    gt_ids, gt_d2, gt_nv = filtered_topk(t["vectors"], t["attrs"], d["attr_types"], t["queries"], full_lo, full_hi, w.k)
-    rec = recall_against(ids.cpu().numpy().view(np.uint32), d2.cpu().numpy(), gt_d2.cpu().numpy(), gt_nv.cpu().numpy(), w.k)
-    assert np.nanmean(rec) > 0.9
-    ids, d2 = gpu.search(t["queries"], t["lo"], t["hi"], w.k, 64, 64)
-    gt_ids, gt_d2, gt_nv = filtered_topk(t["vectors"], t["attrs"], d["attr_types"], t["queries"], t["lo"], t["hi"], w.k)
-    rec_f = recall_against(ids.cpu().numpy().view(np.uint32), d2.cpu().numpy(), gt_d2.cpu().numpy(), gt_nv.cpu().numpy(), w.k)
-    assert np.nanmean(rec_f) > 0.7
-    gpu.close()
+
+    def recalls(thresholds):
+        g = build_graph(t["vectors"], torch.from_numpy(pos).to(dev), R=32, Lb=64, alpha=1.2, thresholds=thresholds,
+                        B=2048, passes=2)
+        gpu = BoaIndex(t["vectors"], t["attrs"], d["attr_types"].tolist(), g)
+        gpu.set_schedule([64]); gpu.set_param("mode", 0)
+        out = []
+        for lo, hi in ((full_lo, full_hi), (t["lo"], t["hi"])):
+            ids, d2 = gpu.search(t["queries"], lo, hi, w.k, 64, 64)
+            _, gt_d2, gt_nv = filtered_topk(t["vectors"], t["attrs"], d["attr_types"], t["queries"], lo, hi, w.k)
+            rec = recall_against(ids.cpu().numpy().view(np.uint32), d2.cpu().numpy(), gt_d2.cpu().numpy(),
+                                 gt_nv.cpu().numpy(), w.k)
+            out.append(float(np.nanmean(rec)))
+        gpu.close()
+        return out
+
+    plain, plain_f = recalls((INF,))
+    mixed, mixed_f = recalls((INF, 0.3, 0.05))
+    assert plain > 0.95 and mixed > 0.9
+    assert mixed_f > 0.95 and mixed_f > plain_f

@@ -83,6 +83,15 @@ def test_pruning_rule_properties(data):
         assert n2 - n1 <= 8
         for c in row2[n1:n2]:
             assert np.abs(pos[c] - pos[p]).max() <= 0.2
+        # a threshold that binds one attribute only: the second half is near in that attribute and
+        # free in the others, and it is what a one-attribute position table gives
+        if pos.shape[1] >= 2:
+            one = (INF,) * (pos.shape[1] - 1) + (0.1,)
+            row3, n3 = ix.prune(pos, p, ids, R=16, alpha=1.2, thresholds=(INF, one))
+            assert row3[:n1].tolist() == first[:n1].tolist()
+            assert all(abs(pos[c, -1] - pos[p, -1]) <= 0.1 for c in row3[n1:n3])
+            row4, n4 = ix.prune(np.ascontiguousarray(pos[:, -1:]), p, ids, R=16, alpha=1.2, thresholds=(INF, 0.1))
+            assert n3 == n4 and row3.tolist() == row4.tolist()
 
 
 def test_built_graph_structure_and_quality(data):
