@@ -71,6 +71,24 @@ PER_CONFIG_VARIANTS = {
 }
 
 
+# Graphs made by the library's own builder (boa_graph_build) instead of the fixture graph:
+# build parameters (attribute thresholds in rank space, sized to the workload's query
+# windows) and the settings timed over the built graph: the fastest adaptive schedule and
+# the fastest fixed beamwidth with recall@10 >= 0.95 from the sweeps in the design notes.
+# GPU-only figures: the oracle never sees a graph the CUDA builder made.
+INF = float("inf")
+BUILT_GRAPH = {
+    "c2": dict(build=dict(R=32, Lb=64, alpha=1.2, thresholds=(INF, 0.3, 0.05), B=8192, passes=2),
+               runs=(dict(schedule=[16, 32], eps=0.02), dict(schedule=[28], eps=0.05))),
+    "c3": dict(build=dict(R=32, Lb=64, alpha=1.2, thresholds=(INF, 0.2, 0.08), B=8192, passes=2),
+               runs=(dict(schedule=[16, 48], eps=0.02), dict(schedule=[48], eps=0.05))),
+    "c4": dict(build=dict(R=64, Lb=64, alpha=1.2, thresholds=(INF, 0.3, 0.05), B=16384, passes=1),
+               runs=(dict(schedule=[16, 48], eps=0.05), dict(schedule=[24], eps=0.05))),
+    "c5": dict(build=dict(R=32, Lb=64, alpha=1.2, thresholds=(INF, 0.3, 0.12), B=8192, passes=2),
+               runs=(dict(schedule=[16, 128], eps=0.01), dict(schedule=[128], eps=0.05))),
+}
+
+
 def kernel_source_digest() -> str:
     import hashlib
     with open(os.path.join(ROOT, "paper_2609_16175_b200", "csrc", "boa_search.cuh"), "rb") as f:
@@ -89,6 +107,12 @@ def parse_args():
     ap.add_argument("--eps", type=float, default=None, help="default: the workload's operating point")
     ap.add_argument("--mode", default="resume", choices=["restart", "resume"])
     ap.add_argument("--schedule", default="", help="phase widths; default: the workload's operating point")
+    ap.add_argument("--built-graph", default="c2,c3,c5",
+                    help="workloads of per_config also measured over a graph built by boa_graph_build "
+                         "(comma list; c4's 10M-point build takes about a minute)")
+    ap.add_argument("--graph-build-only", action="store_true",
+                    help="time boa_graph_build on the workload (with --scale-n for a small case), search the "
+                         "built graph at BUILT_GRAPH's settings and print that entry alone")
     ap.add_argument("--no-per-config", action="store_true",
                     help="measure the headline workload only (always so with more than one GPU)")
     ap.add_argument("--plus-k", type=int, default=0)
@@ -451,9 +475,76 @@ def measure_config(name, args, dev, steps, cpu_seconds, variants=({},), gt_queri
             "cpu_oracle_queries_per_s": ql["cpu_qps"], "gpu_launches_per_step": ix.last_launch_count,
             "device_status": ix.device_status(), "fixture_build_s": round(t_build, 1)}
     ix.close()
-    del t, d, ix, out_ids, out_d2
+    del ix, out_ids, out_d2
+    torch.cuda.empty_cache()
+    if name in BUILT_GRAPH and name in [x for x in args.built_graph.split(",") if x]:
+        try:
+            res[name + "_built_graph"] = measure_built_graph(name, args, dev, w, d, t, max(3, steps // 2), gt_queries)
+        except Exception as e:
+            res[name + "_built_graph"] = {"error": f"{type(e).__name__}: {e}"}
+    del t, d
     torch.cuda.empty_cache()
     return res
+
+
+def attribute_positions(attrs, types):
+    """rank / N of every point in every attribute column (stable order): the builder's attr_pos."""
+    import torch
+    n, m = attrs.shape
+    pos = torch.empty((n, m), dtype=torch.float32, device=attrs.device)
+    for j in range(m):
+        col = attrs[:, j].view(torch.float32) if int(types[j]) == 1 else attrs[:, j]
+        order = torch.argsort(col, stable=True)
+        pos[order, j] = torch.arange(n, dtype=torch.float32, device=attrs.device) / n
+    return pos
+
+
+def measure_built_graph(name, args, dev, w, d, t, steps, gt_queries=10_000):
+    """per_config[name + "_built_graph"]: the graph built on the GPU by boa_graph_build from the
+    workload's vectors and attributes, then the search over it at the settings of
+    BUILT_GRAPH[name].  No oracle run here."""
+    import copy
+    import torch
+    from boa_synth.groundtruth import filtered_topk, recall_against
+    from paper_2609_16175_b200 import BoaIndex, build_graph
+    spec = BUILT_GRAPH[name]
+    pos = attribute_positions(t["attrs"], d["attr_types"])
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    g = build_graph(t["vectors"], pos, **spec["build"])
+    torch.cuda.synchronize()
+    build_s = time.perf_counter() - t0
+    del pos
+    ix = BoaIndex(t["vectors"], t["attrs"], d["attr_types"].tolist(), g)
+    out_ids = torch.empty((w.Q, w.k), dtype=torch.int32, device=dev)
+    out_d2 = torch.empty((w.Q, w.k), dtype=torch.float32, device=dev)
+    n_gt = min(gt_queries, w.Q)
+    _, gt_d2, gt_nv = filtered_topk(t["vectors"], t["attrs"], d["attr_types"], t["queries"][:n_gt],
+                                    t["lo"][:n_gt], t["hi"][:n_gt], w.k)
+    gt_d2, gt_nv = gt_d2.cpu().numpy(), gt_nv.cpu().numpy()
+    runs = []
+    for run in spec["runs"]:
+        a = copy.copy(args)
+        a.workload, a.pq, a.eps = name, "", run["eps"]
+        a.plus_k, a.expand_w, a.lam, a.table_kb, a.table_tags, a.max_warps = 0, 1, float("inf"), 0, 0, 0
+        widths = run["schedule"]
+        configure(ix, a, widths)
+        total_ms, _ = timed_steps(ix, t, w.k, widths, out_ids, out_d2, steps, 3, torch.cuda.synchronize)
+        st = {kk: v.cpu().numpy() for kk, v in ix.stats().items()}
+        rec = recall_against(out_ids.cpu().numpy().view(np.uint32)[:n_gt], out_d2.cpu().numpy()[:n_gt], gt_d2, gt_nv, w.k)
+        ms = total_ms / steps
+        runs.append({"schedule": widths, "eps": a.eps, "mode": a.mode, "steps": steps, "ms_per_step": ms,
+                     "queries_per_s": w.Q / (ms / 1e3), "recall_at_10": float(np.nanmean(rec)), "recall_queries": n_gt,
+                     "avg_beamwidth": float(st["final_L"].mean()), "mean_expansions": float(st["n_expand"].mean()),
+                     "mean_scored": float(st["n_scored"].mean()), "gpu_launches_per_step": ix.last_launch_count,
+                     "device_status": ix.device_status()})
+    degree = float((g != -1).sum(1).float().mean().item())
+    ix.close()
+    del g, out_ids, out_d2
+    build = dict(spec["build"])
+    build["thresholds"] = [str(x) for x in build["thresholds"]]
+    return {"graph": "boa_graph_build", "build": build, "build_s": round(build_s, 2), "mean_degree": degree,
+            "points_per_s": w.N / build_s, "runs": runs}
 
 
 def main():
@@ -478,6 +569,14 @@ def main():
 
     w = get_workload(args)
     widths = schedule_of(args, w)
+    if args.graph_build_only:
+        d = make_workload(w, seed=args.seed, device=str(dev), with_graph=False)
+        d["graph"] = np.zeros((w.N, 1), np.uint32)
+        t = to_device(d, dev)
+        entry = measure_built_graph(args.workload, args, dev, w, d, t, max(3, args.steps // 2))
+        print(json.dumps({"metric": "graph_build_points_per_s", "value": entry["points_per_s"], "unit": "points/s",
+                          "n_gpus": 1, "config": config_dict(w, widths, args), "built_graph": entry}))
+        return
     d = make_workload(w, seed=args.seed, device=str(dev))
     t = to_device(d, dev)
     ix = BoaIndex(t["vectors"], t["attrs"], d["attr_types"].tolist(), t["graph"])
