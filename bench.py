@@ -85,7 +85,7 @@ BUILT_GRAPH = {
     "c4": dict(build=dict(R=64, Lb=64, alpha=1.2, thresholds=(INF, 0.3, 0.05), B=16384, passes=1),
                runs=(dict(schedule=[16, 48], eps=0.05), dict(schedule=[24], eps=0.05))),
     "c5": dict(build=dict(R=32, Lb=64, alpha=1.2, thresholds=(INF, 0.3, 0.12), B=8192, passes=2),
-               runs=(dict(schedule=[16, 128], eps=0.01), dict(schedule=[128], eps=0.05))),
+               runs=(dict(schedule=[16, 128], eps=0.005), dict(schedule=[96], eps=0.05))),
 }
 
 

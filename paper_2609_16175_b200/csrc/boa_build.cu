@@ -108,25 +108,25 @@ __device__ void sort_keys_smem(unsigned long long* keys, int cap, int lane)
 }
 
 // The pruning step for point p over the ids in cand[0..n) (repeats, kNone and p itself allowed).
-// Shared memory of the warp: keys[kMaxCand], flags[kMaxCand].  Writes row[0..R).
+// Shared memory of the warp: keys[kMaxCand], flags[kMaxCand], live[kMaxCand].  Writes row[0..R).
+// Work is kept to what decides the result: repeats are dropped before any distance is
+// computed, and a threshold pass walks a compacted list of the candidates that are still
+// unselected, inside its threshold and not yet dominated.
 __device__ void prune_point(const BuildParams& bp, int64_t p, const uint32_t* cand, int n, unsigned long long* keys,
-                            uint8_t* flags, uint32_t* row, int lane)
+                            uint8_t* flags, uint16_t* live, uint32_t* row, int lane)
 {
     const int g = lane & 7, gi = lane >> 3;
+    const unsigned lt = (1u << lane) - 1u;
     const uint8_t* xp = bp.vec + (size_t)p * bp.row_bytes;
     int cap = 32;
     while (cap < n) cap <<= 1;
-    // distance of every candidate to p: four candidates per step, one 8-lane group each
-    for (int i0 = 0; i0 < cap; i0 += 4) {
-        const int i = i0 + gi;
+    // distinct candidate ids: sort the ids, keep the first of every run
+    for (int i = lane; i < cap; i += 32) {
         const uint32_t id = i < n ? cand[i] : kNone;
-        const bool ok = id != kNone && (int64_t)id != p;
-        const float d = group_dist2(xp, bp.vec + (size_t)(ok ? id : 0) * bp.row_bytes, bp.row_bytes, bp.vec_u8 != 0, g, ok);
-        if (g == 0 && i < cap) keys[i] = ok ? (((unsigned long long)__float_as_uint(d) << 32) | id) : ~0ull;
+        keys[i] = (id != kNone && (int64_t)id != p) ? (unsigned long long)id : ~0ull;
     }
     __syncwarp();
     sort_keys_smem(keys, cap, lane);
-    // drop repeats (equal ids have equal distances, so they are neighbours now); count what is left
     int nc = 0;
     for (int i0 = 0; i0 < cap; i0 += 32) {
         const int i = i0 + lane;
@@ -134,38 +134,74 @@ __device__ void prune_point(const BuildParams& bp, int64_t p, const uint32_t* ca
         const bool keep = k != ~0ull && (i == 0 || keys[i - 1] != k);
         const unsigned bal = __ballot_sync(0xffffffffu, keep);
         __syncwarp();
-        if (keep) keys[nc + __popc(bal & ((1u << lane) - 1u))] = k;
+        if (keep) keys[nc + __popc(bal & lt)] = k;
         nc += __popc(bal);
         __syncwarp();
     }
-    // flags: bit 0 selected, bit 1 dominated in the current threshold pass
-    for (int i = lane; i < nc; i += 32) flags[i] = 0;
+    cap = 32;
+    while (cap < nc) cap <<= 1;
+    // distance of every candidate to p (four candidates per step, one 8-lane group each), then
+    // the order of the pruning: ascending (distance, id)
+    for (int i0 = 0; i0 < cap; i0 += 4) {
+        const int i = i0 + gi;
+        const bool ok = i < nc;
+        const uint32_t id = ok ? (uint32_t)keys[i] : 0u;
+        const float d = group_dist2(xp, bp.vec + (size_t)id * bp.row_bytes, bp.row_bytes, bp.vec_u8 != 0, g, ok);
+        __syncwarp();
+        if (g == 0) keys[i] = ok ? (((unsigned long long)__float_as_uint(d) << 32) | id) : ~0ull;
+    }
+    __syncwarp();
+    sort_keys_smem(keys, cap, lane);
+    for (int i = lane; i < nc; i += 32) flags[i] = 0;                      // 1 = selected
     __syncwarp();
     int total = 0;
-    for (int ti = 0; ti < bp.T; ++ti) {
+    for (int ti = 0; ti < bp.T && total < bp.R; ++ti) {
         const int budget = bp.R * (ti + 1) / bp.T - bp.R * ti / bp.T;
         int taken = 0;
-        for (int i = lane; i < nc; i += 32) flags[i] &= 1;
+        // the pass's list: unselected candidates within its threshold, in pruning order
+        int nl = 0;
+        for (int i0 = 0; i0 < nc; i0 += 32) {
+            const int i = i0 + lane;
+            const bool in = i < nc && !flags[i] && attr_within(bp.pos, bp.m_pos, p, (uint32_t)keys[i], bp.thr[ti]);
+            const unsigned bal = __ballot_sync(0xffffffffu, in);
+            if (in) live[nl + __popc(bal & lt)] = (uint16_t)i;
+            nl += __popc(bal);
+        }
         __syncwarp();
-        for (int i = 0; i < nc && taken < budget; ++i) {
-            if (flags[i]) continue;                                       // selected or dominated (warp-uniform)
+        while (nl > 0 && taken < budget) {
+            // the head of the list is the nearest candidate nothing selected in this pass dominates
+            const int i = live[0];
             const uint32_t ci = (uint32_t)keys[i];
-            if (!attr_within(bp.pos, bp.m_pos, p, ci, bp.thr[ti])) continue;
+            __syncwarp();
             if (lane == 0) { flags[i] = 1; row[total] = ci; }
             total++; taken++;
+            if (taken == budget) break;
             const uint8_t* xc = bp.vec + (size_t)ci * bp.row_bytes;
-            for (int j0 = i + 1; j0 < nc; j0 += 4) {
-                const int j = j0 + gi;
-                const bool ok = j < nc && !(flags[j] & 1);
-                const uint32_t cj = ok ? (uint32_t)keys[j] : 0u;
-                const float dcc = group_dist2(xc, bp.vec + (size_t)cj * bp.row_bytes, bp.row_bytes, bp.vec_u8 != 0, g, ok);
-                if (ok && g == 0) {
-                    const float dpj = __uint_as_float((uint32_t)(keys[j] >> 32));
-                    if (__fmul_rn(bp.alpha2, dcc) <= dpj) flags[j] |= 2;
+            // drop what the new neighbour dominates: 32 list entries per round, four distances per step
+            int nn = 0;
+            for (int j0 = 1; j0 < nl; j0 += 32) {
+                bool dom_mine = false;
+                for (int sub = 0; sub < 8 && j0 + 4 * sub < nl; ++sub) {
+                    const int jj = j0 + 4 * sub + gi;
+                    const bool ok = jj < nl;
+                    const unsigned long long kj = keys[ok ? live[jj] : 0];
+                    const float dcc = group_dist2(xc, bp.vec + (size_t)(ok ? (uint32_t)kj : 0u) * bp.row_bytes, bp.row_bytes,
+                                                  bp.vec_u8 != 0, g, ok);
+                    const bool dom = ok && __fmul_rn(bp.alpha2, dcc) <= __uint_as_float((uint32_t)(kj >> 32));
+                    const unsigned bal = __ballot_sync(0xffffffffu, dom);       // bit 8*gi: entry j0 + 4*sub + gi
+                    if ((lane >> 2) == sub) dom_mine = (bal >> (8 * (lane & 3))) & 1u;
                 }
+                const bool keep = j0 + lane < nl && !dom_mine;
+                const uint16_t mine = live[j0 + lane < nl ? j0 + lane : 0];
+                const unsigned bal = __ballot_sync(0xffffffffu, keep);
+                __syncwarp();
+                if (keep) live[nn + __popc(bal & lt)] = mine;
+                nn += __popc(bal);
+                __syncwarp();
             }
-            __syncwarp();
+            nl = nn;
         }
+        __syncwarp();
     }
     for (int i = total + lane; i < bp.R; i += 32) row[i] = kNone;
     __syncwarp();
@@ -177,6 +213,7 @@ __global__ void prune_batch_kernel(BuildParams bp, int64_t start, int bsz, const
     __shared__ unsigned long long keys[kMaxCand];
     __shared__ uint32_t cand[kMaxCand];
     __shared__ uint8_t flags[kMaxCand];
+    __shared__ uint16_t live[kMaxCand];
     const int lane = threadIdx.x;
     for (int b = blockIdx.x; b < bsz; b += gridDim.x) {
         const int64_t p = start + b;
@@ -185,7 +222,7 @@ __global__ void prune_batch_kernel(BuildParams bp, int64_t start, int bsz, const
             for (int i = lane; i < Lb; i += 32) cand[ti * Lb + i] = cand_ids[((size_t)ti * B + b) * Lb + i];
         for (int i = lane; i < bp.R; i += 32) cand[bp.T * Lb + i] = row[i];
         __syncwarp();
-        prune_point(bp, p, cand, bp.T * Lb + bp.R, keys, flags, row, lane);
+        prune_point(bp, p, cand, bp.T * Lb + bp.R, keys, flags, live, row, lane);
     }
 }
 
@@ -233,6 +270,7 @@ __global__ void reverse_edges_kernel(BuildParams bp, const unsigned long long* r
     __shared__ unsigned long long keys[kMaxCand];
     __shared__ uint32_t cand[kMaxCand];
     __shared__ uint8_t flags[kMaxCand];
+    __shared__ uint16_t live[kMaxCand];
     const int lane = threadIdx.x;
     const uint32_t nh = *n_heads;
     for (uint32_t h = blockIdx.x; h < nh; h += gridDim.x) {
@@ -265,7 +303,7 @@ __global__ void reverse_edges_kernel(BuildParams bp, const unsigned long long* r
         if (deg + nm <= bp.R) {
             for (int j = lane; j < nm; j += 32) row[deg + j] = cand[deg + j];
         } else {
-            prune_point(bp, tgt, cand, deg + nm, keys, flags, row, lane);
+            prune_point(bp, tgt, cand, deg + nm, keys, flags, live, row, lane);
         }
         __syncwarp();
     }
