@@ -55,3 +55,26 @@ def test_create_rejects_bad_shapes_before_any_cuda_call(lib):
     assert create(vec=C.c_void_p(4100)) == -1  # misaligned
     assert create(t=(C.c_int * 2)(0, 5)) == -1
     assert lib.boa_index_create(None, fake, 0, 100, 16, fake, types, 2, fake, 8, -1, None) == -1
+
+
+def test_graph_build_rejects_bad_arguments_before_any_cuda_call(lib):
+    lib.boa_graph_build.restype = C.c_int
+    lib.boa_graph_build.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                                    C.c_float, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_void_p,
+                                    C.c_void_p, C.c_void_p]
+    fake = C.c_void_p(4096)
+    th = (C.c_float * 6)(float("inf"), float("inf"), 0.3, 0.3, 0.05, 0.05)
+    def build(vec=fake, dt=0, N=1000, D=16, pos=fake, m=2, R=16, Lb=32, alpha=1.2, t=th, T=3, B=256, passes=1,
+              cap_in=16, out=fake):
+        return lib.boa_graph_build(vec, dt, N, D, pos, m, R, Lb, alpha, t, T, B, passes, cap_in, -1, out, None, None)
+    assert build(vec=None) == -1 and build(pos=None) == -1 and build(t=None) == -1 and build(out=None) == -1
+    assert build(N=0) == -1
+    assert build(R=0) == -1 and build(R=65) == -1
+    assert build(Lb=0) == -1 and build(Lb=129) == -1
+    assert build(T=0) == -1 and build(T=9) == -1
+    assert build(m=0) == -1 and build(m=9) == -1
+    assert build(B=0) == -1 and build(passes=0) == -1 and build(passes=5) == -1
+    assert build(cap_in=0) == -1 and build(cap_in=65) == -1
+    assert build(alpha=0.9) == -1
+    assert build(Lb=96, T=3, R=32) == -1       # T*Lb + R beyond the candidate buffer
+    assert build(dt=7) == -1
