@@ -53,7 +53,10 @@ enum {
                                earlier ones built (the "redundancy avoidance" paragraph)      */
     BOA_PARAM_PLUS_K = 4,   /* 0 or 1 = BOA; K >= 2 = BOA+: the first phase is issued as K
                                sub-batches and wider phases overlap them ("Pipelining
-                               Multiple Batches")                                            */
+                               Multiple Batches").  The sub-batches run one after another:
+                               each should hold several times the queries the GPU searches
+                               at once (one per resident warp, about 3,000), or K only adds
+                               launches that leave the GPU partly empty                     */
     BOA_PARAM_CAP_MULT = 5, /* a phase at width L gives up after CAP_MULT*L + CAP_ADD        */
     BOA_PARAM_CAP_ADD = 6,  /*   expansions; defaults 8 and 64                               */
     BOA_PARAM_TABLE_KB = 7, /* 0 = default (6 or 4, whichever keeps 20 query warps per SM
