@@ -102,3 +102,26 @@ def test_built_graph_serves_the_search():
     mixed, mixed_f = recalls((INF, 0.3, 0.05))
     assert plain > 0.95 and mixed > 0.9
     assert mixed_f > 0.95 and mixed_f > plain_f
+
+
+@pytest.mark.parametrize("n", [1, 2, 5, 40])
+def test_tiny_and_degenerate_inputs(n):
+    """Fewer points than the degree or the beamwidth, and repeated vectors (distance 0 to each
+    other): the same graph as the oracle's, no self loops, no repeats in a row."""
+    from paper_2609_16175_b200 import build_graph
+    rng = np.random.default_rng(n)
+    D = 16
+    x = rng.standard_normal((n, D)).astype(np.float32)
+    if n >= 5:
+        x[n // 2:] = x[: n - n // 2]                      # every vector of the second half repeats one of the first
+    attrs = rng.integers(0, 100, size=(n, 2)).astype(np.int32)
+    types = np.zeros(2, np.int32)
+    pos = _positions(attrs, types)
+    kw = dict(R=8, Lb=16, alpha=1.2, thresholds=(INF, 0.3), B=4, passes=2)
+    orc = OracleIndex(x, attrs, types, np.zeros((n, 1), np.uint32))
+    go = orc.build_graph(pos, **kw)
+    gg = build_graph(torch.from_numpy(x).to("cuda:0"), torch.from_numpy(pos).to("cuda:0"), **kw).cpu().numpy().view(np.uint32)
+    assert (go == gg).all(), (go, gg)
+    for r in range(n):
+        row = gg[r][gg[r] != SENTINEL]
+        assert r not in row and len(set(row.tolist())) == len(row) and (row < n).all()
