@@ -85,7 +85,8 @@ BUILT_GRAPH = {
     "c4": dict(build=dict(R=64, Lb=64, alpha=1.2, thresholds=(INF, 0.3, 0.05), B=16384, passes=1),
                runs=(dict(schedule=[16, 48], eps=0.05), dict(schedule=[24], eps=0.05))),
     "c5": dict(build=dict(R=32, Lb=64, alpha=1.2, thresholds=(INF, 0.3, 0.12), B=8192, passes=2),
-               runs=(dict(schedule=[16, 128], eps=0.005), dict(schedule=[96], eps=0.05))),
+               runs=(dict(schedule=[16, 128], eps=0.005), dict(schedule=[96], eps=0.05),
+                     dict(schedule=[256], eps=0.05, pq="48,64"))),
 }
 
 
@@ -525,15 +526,17 @@ def measure_built_graph(name, args, dev, w, d, t, steps, gt_queries=10_000):
     runs = []
     for run in spec["runs"]:
         a = copy.copy(args)
-        a.workload, a.pq, a.eps = name, "", run["eps"]
+        a.workload, a.pq, a.eps = name, run.get("pq", ""), run["eps"]
         a.plus_k, a.expand_w, a.lam, a.table_kb, a.table_tags, a.max_warps = 0, 1, float("inf"), 0, 0, 0
         widths = run["schedule"]
-        configure(ix, a, widths)
+        # the codebook cached beside the workload is reused; "attached" marks belong to another index
+        configure(ix, a, widths, {k: v for k, v in d.items() if not (isinstance(k, tuple) and k[0] == "attached")}
+                  if a.pq else None)
         total_ms, _ = timed_steps(ix, t, w.k, widths, out_ids, out_d2, steps, 3, torch.cuda.synchronize)
         st = {kk: v.cpu().numpy() for kk, v in ix.stats().items()}
         rec = recall_against(out_ids.cpu().numpy().view(np.uint32)[:n_gt], out_d2.cpu().numpy()[:n_gt], gt_d2, gt_nv, w.k)
         ms = total_ms / steps
-        runs.append({"schedule": widths, "eps": a.eps, "mode": a.mode, "steps": steps, "ms_per_step": ms,
+        runs.append({"schedule": widths, "eps": a.eps, "mode": a.mode, "pq": a.pq or None, "steps": steps, "ms_per_step": ms,
                      "queries_per_s": w.Q / (ms / 1e3), "recall_at_10": float(np.nanmean(rec)), "recall_queries": n_gt,
                      "avg_beamwidth": float(st["final_L"].mean()), "mean_expansions": float(st["n_expand"].mean()),
                      "mean_scored": float(st["n_scored"].mean()), "gpu_launches_per_step": ix.last_launch_count,
