@@ -61,10 +61,10 @@ WIDE = {"c2": dict(schedule=[16, 512], eps=0.03), "c3": dict(schedule=[16, 512],
 
 
 # What per_config measures beside each workload's operating point: the wide schedule for
-# c2-c4, the configuration's own fixed beamwidth of 500 for c5, and for c5 the same two runs
+# c2-c4, the operating point with two nodes expanded per iteration for c2 (tag w2), the configuration's own fixed beamwidth of 500 for c5, and for c5 the same two runs
 # with PQ traversal (48 subspaces of 20 dimensions, 64 centroids each; exact final ranking).
 PER_CONFIG_VARIANTS = {
-    "c2": (dict(WIDE["c2"], tag="wide"),),
+    "c2": (dict(WIDE["c2"], tag="wide"), dict(expand_w=2, tag="w2")),
     "c3": ({}, dict(WIDE["c3"], tag="wide")),
     "c4": ({}, dict(WIDE["c4"], tag="wide")),
     "c5": ({}, {"fixed_L": 500}, {"pq": "48,64"}, {"pq": "48,64", "fixed_L": 500}),
@@ -446,7 +446,7 @@ def measure_config(name, args, dev, steps, cpu_seconds, variants=({},), gt_queri
         a = copy.copy(args)
         a.workload, a.scale_n, a.queries, a.schedule, a.fixed_L, a.pq = name, 0, 0, "", fixed_L, pq
         a.eps = var.get("eps", OPERATING[name]["eps"])
-        a.plus_k, a.expand_w, a.lam, a.table_kb, a.table_tags, a.max_warps = 0, 1, float("inf"), 0, 0, 0
+        a.plus_k, a.expand_w, a.lam, a.table_kb, a.table_tags, a.max_warps = 0, var.get("expand_w", 1), float("inf"), 0, 0, 0
         widths = var.get("schedule") or schedule_of(a, w)
         configure(ix, a, widths, d)
         n_steps = steps if not fixed_L else max(3, steps // 2)
