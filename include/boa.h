@@ -87,6 +87,10 @@ enum {
                                line and the "Re-rank exact" step of Section "BOA Implementation
                                on a GPU System".  0 (default) = exact distances throughout.
                                With 1, k <= BOA_PQ_MAX_K and BOA_PARAM_EXPAND_W must be 1.     */
+    BOA_PARAM_HOST_IN_PLACE = 13, /* boa_search_host only.  1 (default): buffers in page-locked host
+                               memory that the device can address are read and written in
+                               place by the search kernels; 0: always staged through device
+                               copies.  Results are the same either way.                     */
     BOA_PARAM_EXPAND_W = 9  /* nodes expanded per iteration of Algorithm 2.  1 (default) is
                                the algorithm as printed (one node per iteration, Section
                                "How Filtered Search Works").  2 is an extension: the first
@@ -221,6 +225,28 @@ int64_t boa_index_entry(const boa_index* index);
  */
 int boa_search(boa_index* index, const float* queries, int64_t Q, const void* lo, const void* hi,
                int k, int L0, int Lmax, uint32_t* out_ids, float* out_dists, void* stream);
+
+/*
+ * boa_search with HOST buffers: the end-to-end call of a caller whose queries arrive in host
+ * memory and whose results are read on the host (the problem statement's (q_i, f_i) -> K_f
+ * with the transfers included).  Copies queries, lo and hi to index-owned device staging
+ * buffers on `stream`, runs boa_search there, copies out_ids and out_dists back and
+ * SYNCHRONISES `stream` before it returns, so the outputs are ready to read.  When all five
+ * buffers are page-locked host memory mapped into the device's address space (cudaHostAlloc,
+ * cudaHostRegister) and start on 16 bytes, nothing is staged: the kernels read each query over
+ * the host link when they start on it and write its results straight back
+ * (BOA_PARAM_HOST_IN_PLACE = 0 turns that off).
+ *
+ *   queries, lo, hi, out_ids, out_dists   HOST pointers, shapes and meaning as in boa_search;
+ *       page-locked memory lets the copies run at full speed and asynchronously, pageable
+ *       memory works too.  No alignment requirement.
+ *   everything else as in boa_search (same results, statistics, parameter handling).
+ *
+ * The staging buffers grow (cudaMalloc) the first time a batch is larger than any before.
+ * Errors: as boa_search, plus BOA_ENOMEM for the staging buffers.
+ */
+int boa_search_host(boa_index* index, const float* queries, int64_t Q, const void* lo, const void* hi, int k,
+                    int L0, int Lmax, uint32_t* out_ids, float* out_dists, void* stream);
 
 /*
  * boa_search for callers that must not allocate device memory.  (The paper has no

@@ -16,7 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = None
 
 PARAM = dict(eps=0, growth=1, tau=2, mode=3, plus_k=4, cap_mult=5, cap_add=6, table_kb=7,
-             max_warps_per_sm=8, expand_w=9, table_tags=10, lam=11, pq=12)
+             max_warps_per_sm=8, expand_w=9, table_tags=10, lam=11, pq=12, host_in_place=13)
 F32, U8 = 0, 1
 NO_ID = 0xFFFFFFFF
 
@@ -57,6 +57,8 @@ def load_library():
     L.boa_search.argtypes = [vp, vp, i64, vp, vp, i32, i32, i32, vp, vp, vp]
     L.boa_search_noalloc.restype = i32
     L.boa_search_noalloc.argtypes = [vp, vp, i64, vp, vp, i32, i32, i32, vp, vp, vp]
+    L.boa_search_host.restype = i32
+    L.boa_search_host.argtypes = [vp, vp, i64, vp, vp, i32, i32, i32, vp, vp, vp]
     L.boa_set_param.restype = i32
     L.boa_set_param.argtypes = [vp, i32, C.c_double]
     L.boa_set_schedule.restype = i32
@@ -231,6 +233,29 @@ class BoaIndex:
         _check(self._lib.boa_search(self._h, queries.data_ptr(), Q, lo.data_ptr(), hi.data_ptr(), k,
                                     L0, Lmax, out_ids.data_ptr(), out_dists.data_ptr(),
                                     _stream_ptr(stream)), "boa_search")
+        self._last_Q = Q
+        return out_ids, out_dists
+
+    def search_host(self, queries: torch.Tensor, lo: torch.Tensor, hi: torch.Tensor, k: int, L0: int,
+                    Lmax: int, out_ids: Optional[torch.Tensor] = None,
+                    out_dists: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+        """boa_search_host: HOST tensors in (pinned for full copy speed), HOST tensors out; the
+        library does the transfers and returns when the results are readable."""
+        for name, t in (("queries", queries), ("lo", lo), ("hi", hi)):
+            if t.is_cuda or not t.is_contiguous():
+                raise ValueError(f"{name} must be a contiguous CPU tensor")
+        Q = queries.shape[0]
+        if out_ids is None:
+            out_ids = torch.empty((Q, k), dtype=torch.int32)
+        if out_dists is None:
+            out_dists = torch.empty((Q, k), dtype=torch.float32)
+        for name, t in (("out_ids", out_ids), ("out_dists", out_dists)):
+            if t.is_cuda or not t.is_contiguous():
+                raise ValueError(f"{name} must be a contiguous CPU tensor")
+        with torch.cuda.device(self.device):
+            _check(self._lib.boa_search_host(self._h, queries.data_ptr(), Q, lo.data_ptr(), hi.data_ptr(), k,
+                                             L0, Lmax, out_ids.data_ptr(), out_dists.data_ptr(),
+                                             _stream_ptr(stream)), "boa_search_host")
         self._last_Q = Q
         return out_ids, out_dists
 

@@ -196,6 +196,11 @@ struct boa_index {
     uint32_t* graph = nullptr;
     int device = 0, num_sms = 0;
     int metric = BOA_METRIC_L2;
+    // device staging of boa_search_host: queries [ws_host_Q][D], lo and hi [ws_host_Q][m], outputs [ws_host_Q][ws_host_k]
+    float* hq = nullptr; int32_t* hlo = nullptr; int32_t* hhi = nullptr; uint32_t* hids = nullptr; float* hd2 = nullptr;
+    int64_t ws_host_Q = 0;
+    int ws_host_k = 0;
+    int host_in_place = 1;             // boa_search_host reads mapped page-locked buffers in place
     float* qunit = nullptr;            // [ws_qunit][D] unit-length copies of a batch's queries (cosine)
     int64_t ws_qunit = 0;
     // product quantisation (optional)
@@ -624,6 +629,7 @@ int boa_index_destroy(boa_index* ix)
     cudaFree(ix->rec); cudaFree(ix->attr_cells); cudaFree(ix->graph); cudaFree(ix->lists); cudaFree(ix->counters);
     cudaFree(ix->stats); cudaFree(ix->spill); cudaFree(ix->spill_size);
     cudaFree(ix->pq_codes); cudaFree(ix->pq_pivots); cudaFree(ix->qunit); cudaFree(ix->pen_scales);
+    cudaFree(ix->hq); cudaFree(ix->hlo); cudaFree(ix->hhi); cudaFree(ix->hids); cudaFree(ix->hd2);
     if (ix->side) cudaStreamDestroy(ix->side);
     if (ix->ev_fork) cudaEventDestroy(ix->ev_fork);
     if (ix->ev_join) cudaEventDestroy(ix->ev_join);
@@ -681,6 +687,9 @@ int boa_set_param(boa_index* ix, int key, double v)
         case BOA_PARAM_PQ:
             if ((v != 0.0 && v != 1.0) || (v == 1.0 && !ix->pq_codes)) return BOA_EINVAL;
             ix->use_pq = (int)v; return BOA_OK;
+        case BOA_PARAM_HOST_IN_PLACE:
+            if (v != 0.0 && v != 1.0) return BOA_EINVAL;
+            ix->host_in_place = (int)v; return BOA_OK;
         default: return BOA_EINVAL;
     }
 }
@@ -960,6 +969,67 @@ int boa_get_phase_counts(boa_index* ix, int64_t* active, int n, int* n_phases, v
 }
 
 int boa_last_launch_count(const boa_index* ix) { return ix ? ix->last_launches : 0; }
+
+int boa_search_host(boa_index* ix, const float* queries, int64_t Q, const void* lo, const void* hi, int k,
+                    int L0, int Lmax, uint32_t* out_ids, float* out_dists, void* stream)
+{
+    if (!ix) return BOA_EINVAL;
+    if (Q < 0 || Q > (int64_t)0x7FFFFFFF || k < 1 || k > BOA_MAX_WIDTH) return BOA_EINVAL;
+    if (Q == 0) return boa_search(ix, nullptr, 0, nullptr, nullptr, k, L0, Lmax, nullptr, nullptr, stream);
+    if (!queries || !lo || !hi || !out_ids || !out_dists) return BOA_EINVAL;
+    if (!on_device(ix->device)) return BOA_EINVAL;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    {
+        // Page-locked host memory that is mapped into the device's address space is read and
+        // written in place: the kernels fetch each query over the host link when they start on
+        // it and write its results straight back, so no transfer is serialised before or after
+        // the search.
+        auto mapped = [](const void* p, const void** dp) {
+            cudaPointerAttributes a;
+            if (cudaPointerGetAttributes(&a, p) != cudaSuccess) { cudaGetLastError(); return false; }
+            if (a.type != cudaMemoryTypeHost || !a.devicePointer) return false;
+            *dp = a.devicePointer;
+            return aligned16(*dp);
+        };
+        const void *dq, *dlo, *dhi, *dids, *dd2;
+        if (ix->host_in_place && mapped(queries, &dq) && mapped(lo, &dlo) && mapped(hi, &dhi) && mapped(out_ids, &dids) &&
+            mapped(out_dists, &dd2)) {
+            const int rc = boa_search(ix, static_cast<const float*>(dq), Q, dlo, dhi, k, L0, Lmax,
+                                      static_cast<uint32_t*>(const_cast<void*>(dids)),
+                                      static_cast<float*>(const_cast<void*>(dd2)), stream);
+            const cudaError_t e = cudaStreamSynchronize(st);
+            if (rc != BOA_OK) return rc;
+            BOA_CUDA(e);
+            return BOA_OK;
+        }
+    }
+    if (Q > ix->ws_host_Q || k > ix->ws_host_k) {
+        const int64_t nq = Q > ix->ws_host_Q ? Q : ix->ws_host_Q;
+        const int nk = k > ix->ws_host_k ? k : ix->ws_host_k;
+        BOA_CUDA(cudaStreamSynchronize(st));        // an earlier call's copies may still read the old buffers
+        cudaFree(ix->hq); cudaFree(ix->hlo); cudaFree(ix->hhi); cudaFree(ix->hids); cudaFree(ix->hd2);
+        ix->hq = nullptr; ix->hlo = nullptr; ix->hhi = nullptr; ix->hids = nullptr; ix->hd2 = nullptr;
+        ix->ws_host_Q = 0; ix->ws_host_k = 0;
+        BOA_CUDA(cudaMalloc(&ix->hq, (size_t)nq * ix->D * sizeof(float)));
+        BOA_CUDA(cudaMalloc(&ix->hlo, (size_t)nq * ix->m * sizeof(int32_t)));
+        BOA_CUDA(cudaMalloc(&ix->hhi, (size_t)nq * ix->m * sizeof(int32_t)));
+        BOA_CUDA(cudaMalloc(&ix->hids, (size_t)nq * nk * sizeof(uint32_t)));
+        BOA_CUDA(cudaMalloc(&ix->hd2, (size_t)nq * nk * sizeof(float)));
+        ix->ws_host_Q = nq; ix->ws_host_k = nk;
+    }
+    BOA_CUDA(cudaMemcpyAsync(ix->hq, queries, (size_t)Q * ix->D * sizeof(float), cudaMemcpyHostToDevice, st));
+    BOA_CUDA(cudaMemcpyAsync(ix->hlo, lo, (size_t)Q * ix->m * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    BOA_CUDA(cudaMemcpyAsync(ix->hhi, hi, (size_t)Q * ix->m * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    const int rc = boa_search(ix, ix->hq, Q, ix->hlo, ix->hhi, k, L0, Lmax, ix->hids, ix->hd2, stream);
+    if (rc != BOA_OK) {
+        cudaStreamSynchronize(st);                   // the caller may free its host buffers right after an error
+        return rc;
+    }
+    BOA_CUDA(cudaMemcpyAsync(out_ids, ix->hids, (size_t)Q * k * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+    BOA_CUDA(cudaMemcpyAsync(out_dists, ix->hd2, (size_t)Q * k * sizeof(float), cudaMemcpyDeviceToHost, st));
+    BOA_CUDA(cudaStreamSynchronize(st));
+    return BOA_OK;
+}
 
 int boa_search_noalloc(boa_index* ix, const float* queries, int64_t Q, const void* lo, const void* hi,
                        int k, int L0, int Lmax, uint32_t* out_ids, float* out_dists, void* stream)
