@@ -117,6 +117,9 @@ def parse_args():
     ap.add_argument("--no-per-config", action="store_true",
                     help="measure the headline workload only (always so with more than one GPU)")
     ap.add_argument("--plus-k", type=int, default=0)
+    ap.add_argument("--plus-min-sub", type=int, default=0,
+                    help="BOA+: fewest queries per sub-batch (0 = the library's default, twice the resident "
+                         "query warps; 1 = always K sub-batches)")
     ap.add_argument("--expand-w", type=int, default=1, choices=[1, 2],
                     help="nodes expanded per iteration: 1 = Algorithm 2 as printed, 2 = extension")
     ap.add_argument("--lam", type=float, default=float("inf"),
@@ -378,6 +381,7 @@ def configure(ix, args, widths, d=None):
     ix.set_param("mode", 1 if args.mode == "resume" else 0)
     ix.set_param("eps", args.eps)
     ix.set_param("plus_k", args.plus_k)
+    ix.set_param("plus_min_sub", getattr(args, "plus_min_sub", 0))
     ix.set_param("expand_w", args.expand_w)
     ix.set_param("lam", args.lam)
     ix.set_param("table_kb", args.table_kb)

@@ -53,10 +53,8 @@ enum {
                                earlier ones built (the "redundancy avoidance" paragraph)      */
     BOA_PARAM_PLUS_K = 4,   /* 0 or 1 = BOA; K >= 2 = BOA+: the first phase is issued as K
                                sub-batches and wider phases overlap them ("Pipelining
-                               Multiple Batches").  The sub-batches run one after another:
-                               each should hold several times the queries the GPU searches
-                               at once (one per resident warp, about 3,000), or K only adds
-                               launches that leave the GPU partly empty                     */
+                               Multiple Batches").  The sub-batches run one after another,
+                               so K is capped by BOA_PARAM_PLUS_MIN_SUB                      */
     BOA_PARAM_CAP_MULT = 5, /* a phase at width L gives up after CAP_MULT*L + CAP_ADD        */
     BOA_PARAM_CAP_ADD = 6,  /*   expansions; defaults 8 and 64                               */
     BOA_PARAM_TABLE_KB = 7, /* 0 = default (6 or 4, whichever keeps 20 query warps per SM
@@ -87,6 +85,10 @@ enum {
                                line and the "Re-rank exact" step of Section "BOA Implementation
                                on a GPU System".  0 (default) = exact distances throughout.
                                With 1, k <= BOA_PQ_MAX_K and BOA_PARAM_EXPAND_W must be 1.     */
+    BOA_PARAM_PLUS_MIN_SUB = 14, /* BOA+: the fewest queries a sub-batch may hold; K is lowered
+                               (down to plain BOA) until Q / K reaches it.  0 (default) = twice
+                               the queries the GPU searches at once (2 x 20 x SM count); 1 =
+                               always K sub-batches.                                         */
     BOA_PARAM_HOST_IN_PLACE = 13, /* boa_search_host only.  1 (default): buffers in page-locked host
                                memory that the device can address are read and written in
                                place by the search kernels; 0: always staged through device

@@ -200,6 +200,7 @@ struct boa_index {
     float* hq = nullptr; int32_t* hlo = nullptr; int32_t* hhi = nullptr; uint32_t* hids = nullptr; float* hd2 = nullptr;
     int64_t ws_host_Q = 0;
     int ws_host_k = 0;
+    int64_t plus_min_sub = 0;          // smallest BOA+ sub-batch; 0 = twice the resident query warps
     int host_in_place = 1;             // boa_search_host reads mapped page-locked buffers in place
     float* qunit = nullptr;            // [ws_qunit][D] unit-length copies of a batch's queries (cosine)
     int64_t ws_qunit = 0;
@@ -687,6 +688,9 @@ int boa_set_param(boa_index* ix, int key, double v)
         case BOA_PARAM_PQ:
             if ((v != 0.0 && v != 1.0) || (v == 1.0 && !ix->pq_codes)) return BOA_EINVAL;
             ix->use_pq = (int)v; return BOA_OK;
+        case BOA_PARAM_PLUS_MIN_SUB:
+            if (v < 0.0 || v > 2147483647.0 || v != floor(v)) return BOA_EINVAL;
+            ix->plus_min_sub = (int64_t)v; return BOA_OK;
         case BOA_PARAM_HOST_IN_PLACE:
             if (v != 0.0 && v != 1.0) return BOA_EINVAL;
             ix->host_in_place = (int)v; return BOA_OK;
@@ -810,7 +814,15 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
         return BOA_OK;
     }
 
-    const int K = (ix->plus_k >= 2 && lp.n_phases > 1 && ix->tau == 0.0) ? ix->plus_k : 1;
+    // BOA+ splits the first phase into sub-batches that run one after another: a sub-batch
+    // smaller than about twice the queries the GPU searches at once (one per resident warp)
+    // would leave it partly empty, so K is lowered until the sub-batches are that large
+    int K = (ix->plus_k >= 2 && lp.n_phases > 1 && ix->tau == 0.0) ? ix->plus_k : 1;
+    {
+        const int64_t min_sub = ix->plus_min_sub > 0 ? ix->plus_min_sub : (int64_t)2 * 20 * ix->num_sms;
+        if (K > 1 && Q / min_sub < K) K = (int)(Q / min_sub);
+        if (K < 2) K = 1;
+    }
     uint32_t* cnt = ix->counters + kCntCount;
     uint32_t* snap = ix->counters + kCntSnap;
     if (K == 1) {

@@ -35,6 +35,7 @@ def gpu_search(gpu, g, k, widths, mode="restart", eps=0.05, tau=0.0, plus_k=0, c
     gpu.set_param("eps", eps)
     gpu.set_param("tau", tau)
     gpu.set_param("plus_k", plus_k)
+    gpu.set_param("plus_min_sub", 1)          # tests want K sub-batches whatever the batch size
     gpu.set_param("cap_mult", cap[0])
     gpu.set_param("cap_add", cap[1])
     gpu.set_param("expand_w", expand_w)

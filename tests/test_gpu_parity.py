@@ -185,6 +185,23 @@ def test_boa_plus_equals_boa(name, plus_k):
         assert (a["phase_active"] == b["phase_active"]).all()
 
 
+def test_boa_plus_sub_batches_are_not_made_smaller_than_the_gpu():
+    """With the default smallest sub-batch (twice the resident query warps) a batch of a few
+    hundred queries runs as plain BOA whatever K says; plus_min_sub = 1 gives the K sub-batches."""
+    w, d, orc, gpu, g = _get("c2")
+    widths = default_widths(w.L0, 256)
+    a = gpu_search(gpu, g, w.k, widths, mode="resume", plus_k=0)
+    boa_launches = gpu.last_launch_count
+    b = gpu_search(gpu, g, w.k, widths, mode="resume", plus_k=5)
+    assert gpu.last_launch_count > boa_launches
+    gpu.set_param("plus_min_sub", 0)
+    ids, d2 = gpu.search(g["queries"], g["lo"], g["hi"], w.k, widths[0], widths[-1])
+    assert gpu.last_launch_count == boa_launches
+    assert (ids.cpu().numpy().view(np.uint32) == a["ids"]).all() and (a["ids"] == b["ids"]).all()
+    gpu.set_param("plus_min_sub", 1)
+    gpu.set_param("plus_k", 0)
+
+
 def test_fixed_width_500_not_a_power_of_two():
     w, d, orc, gpu, g = _get("c2")
     o = orc.search(d["queries"][:80], d["lo"][:80], d["hi"][:80], w.k, [500], dist_mode=1)

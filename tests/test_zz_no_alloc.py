@@ -65,6 +65,7 @@ def test_noalloc_equals_boa_search_on_two_calls_in_a_row(mode):
 def _compare(ix, t, sl, k, widths, plus_k=0):
     """boa_search, then boa_search_noalloc, on queries sl: identical bits, no allocation."""
     ix.set_param("plus_k", plus_k)
+    ix.set_param("plus_min_sub", 1)
     ix.set_schedule(widths)
     q, lo, hi = (t[n][sl].contiguous() for n in ("queries", "lo", "hi"))
     ref_ids, ref_d2 = ix.search(q, lo, hi, k, widths[0], widths[-1])
