@@ -421,14 +421,22 @@ def _cache_load(path: str):
 
 
 def _cache_store(path: str, out: Dict[str, np.ndarray]) -> None:
+    """Written under a name of this process's own and renamed into place in one step, so that
+    several ranks building the same workload at once never read each other's half-written files."""
+    tmp = f"{path}.tmp{os.getpid()}"
     try:
-        os.makedirs(path, exist_ok=True)
+        os.makedirs(tmp, exist_ok=True)
         for k in _CACHED:
-            np.save(os.path.join(path, k + ".npy"), out[k])
-        with open(os.path.join(path, "done"), "w") as f:
+            np.save(os.path.join(tmp, k + ".npy"), out[k])
+        with open(os.path.join(tmp, "done"), "w") as f:
             f.write("ok")
+        os.rename(tmp, path)      # fails when another process got there first
     except Exception:
-        pass                      # a full or read-only disk only costs the next build
+        pass                      # a full or read-only disk, or a lost race, only costs a build
+    finally:
+        if os.path.isdir(tmp):
+            import shutil
+            shutil.rmtree(tmp, ignore_errors=True)
 
 
 def make_workload(w: Workload, seed: int = 0, device: str | None = None,
