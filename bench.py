@@ -41,6 +41,7 @@ UNIT = "queries/s"
 NCU_DRAM_BYTES_PER_SCORED = {
     # workload: (bytes per scored record, sha256[:12] of csrc/boa_search.cuh, summary file)
     "c2": (410.8, "633158171c92", "profiles/boa_search_kernel_c2_dram_traffic.md"),
+    "c3": (312.7, "633158171c92", "profiles/boa_search_kernel_c3_dram_traffic.md"),
 }
 
 # Operating point of each workload: explicit phase widths and eps, chosen from the sweeps in
@@ -475,6 +476,9 @@ def measure_config(name, args, dev, steps, cpu_seconds, variants=({},), gt_queri
             "mean_expansions": float(st["n_expand"].mean()), "mean_scored": float(st["n_scored"].mean()),
             "rescored_fraction": 1.0 - ql["unique_ratio"], "capped_fraction": float((st["flags"] & 1).mean()),
             "algorithmic_bytes_per_step": alg, "achieved_gbs": alg / (ms / 1e3) / 1e9,
+            "traffic": (NCU_DRAM_BYTES_PER_SCORED[name][0] * float(st["n_scored"].sum())
+                        if name in NCU_DRAM_BYTES_PER_SCORED and not var
+                        and NCU_DRAM_BYTES_PER_SCORED[name][1] == kernel_source_digest() else None),
             "frac": alg / (ms / 1e3) / 1e9 / peak, "peak_kind": peak_kind,
             "parity_with_oracle_on_sample": ql["parity"], "oracle_sample_queries": ql["cpu_n"],
             "cpu_oracle_queries_per_s": ql["cpu_qps"], "gpu_launches_per_step": ix.last_launch_count,
