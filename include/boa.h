@@ -194,7 +194,25 @@ int boa_index_attach_pq(boa_index* index, const float* pivots, const uint8_t* co
  */
 int boa_index_set_metric(boa_index* index, int metric, void* stream);
 
-/* Free the index and everything it owns.  NULL is accepted. */
+/*
+ * A second handle on the same index data, for searches that run at the same time as the
+ * first handle's (the paper's "Pipelining Multiple Batches" carried to whole batches: while
+ * the last, partly empty wave of one batch's wide phase drains, the narrow phase of the next
+ * batch fills the GPU from another stream).  boa_search keeps its survivor lists, counters,
+ * statistics and carried pools in its handle, so two searches in flight need two handles.
+ * The new handle shares the vectors, attribute cells, graph and PQ codebook of `src` (no
+ * copy), copies src's parameters, schedule and range-penalty scales as they stand, and owns
+ * its own scratch (allocated on its first search), so it costs a few MB.
+ *
+ * Rules: `src` must be fully set up before (boa_index_attach_pq and boa_index_set_metric are
+ * BOA_EINVAL on a shared handle, and calling them on `src` afterwards is not seen by, or
+ * breaks, its shares) and must outlive every handle shared from it; each handle is used by
+ * one search at a time; parameters set on one handle do not reach the other.
+ * Errors: BOA_EINVAL, BOA_ENOMEM, BOA_ECUDA; *out is NULL then.
+ */
+int boa_index_share(boa_index** out, boa_index* src);
+
+/* Free the index and everything it owns (a shared handle: its scratch only).  NULL is accepted. */
 int boa_index_destroy(boa_index* index);
 
 /* The start node the index uses (host value). */

@@ -49,6 +49,8 @@ def load_library():
     L.boa_index_create.restype = i32
     L.boa_index_create.argtypes = [C.POINTER(vp), vp, i32, i64, i32, vp, C.POINTER(i32), i32, vp, i32,
                                    i64, vp]
+    L.boa_index_share.restype = i32
+    L.boa_index_share.argtypes = [C.POINTER(vp), vp]
     L.boa_index_destroy.restype = i32
     L.boa_index_destroy.argtypes = [vp]
     L.boa_index_entry.restype = i64
@@ -167,6 +169,20 @@ class BoaIndex:
                                           int(entry), _stream_ptr(stream)), "boa_index_create")
         self._h = h
         self.device = vectors.device
+
+    def share(self) -> "BoaIndex":
+        """boa_index_share: another handle on the same index data with scratch of its own, for a
+        search that runs at the same time as this handle's (on another stream).  This object must
+        stay open while the shared one is in use."""
+        other = object.__new__(BoaIndex)
+        other._lib = self._lib
+        other.N, other.D, other.m, other.R, other.device = self.N, self.D, self.m, self.R, self.device
+        other._owner = self                       # keeps the data alive
+        h = C.c_void_p()
+        with torch.cuda.device(self.device):
+            _check(self._lib.boa_index_share(C.byref(h), self._h), "boa_index_share")
+        other._h = h
+        return other
 
     def close(self):
         if getattr(self, "_h", None):

@@ -195,6 +195,7 @@ struct boa_index {
     uint8_t* rec = nullptr;
     uint32_t* graph = nullptr;
     int device = 0, num_sms = 0;
+    int shared = 0;                    // made by boa_index_share: rec, attr_cells, graph, pq_* belong to another handle
     int metric = BOA_METRIC_L2;
     // device staging of boa_search_host: queries [ws_host_Q][D], lo and hi [ws_host_Q][m], outputs [ws_host_Q][ws_host_k]
     float* hq = nullptr; int32_t* hlo = nullptr; int32_t* hhi = nullptr; uint32_t* hids = nullptr; float* hd2 = nullptr;
@@ -624,12 +625,50 @@ int boa_index_create(boa_index** out, const void* vectors, int vec_dtype, int64_
     return BOA_OK;
 }
 
+int boa_index_share(boa_index** out, boa_index* src)
+{
+    if (!out || !src) return BOA_EINVAL;
+    if (!on_device(src->device)) return BOA_EINVAL;
+    *out = nullptr;
+    boa_index* ix = new (std::nothrow) boa_index(*src);      // data pointers and parameters as they stand
+    if (!ix) return BOA_ENOMEM;
+    ix->shared = 1;
+    // everything a search writes is this handle's own, allocated on first use
+    ix->hq = nullptr; ix->hlo = nullptr; ix->hhi = nullptr; ix->hids = nullptr; ix->hd2 = nullptr;
+    ix->ws_host_Q = 0; ix->ws_host_k = 0;
+    ix->qunit = nullptr; ix->ws_qunit = 0;
+    ix->ws_Q = 0; ix->ws_spill = 0;
+    ix->lists = nullptr; ix->counters = nullptr; ix->stats = nullptr; ix->spill = nullptr; ix->spill_size = nullptr;
+    ix->side = nullptr; ix->ev_fork = nullptr; ix->ev_join = nullptr;
+    ix->pen_scales = nullptr;
+    ix->last_Q = 0; ix->last_phases = 0; ix->last_launches = 0;
+    cudaError_t e = cudaStreamCreateWithFlags(&ix->side, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ix->ev_fork, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ix->ev_join, cudaEventDisableTiming);
+    if (e == cudaSuccess && src->pen_scales) {
+        e = cudaMalloc(&ix->pen_scales, BOA_MAX_ATTRS * sizeof(float));
+        if (e == cudaSuccess)
+            e = cudaMemcpy(ix->pen_scales, src->pen_scales, BOA_MAX_ATTRS * sizeof(float), cudaMemcpyDeviceToDevice);
+    }
+    if (e != cudaSuccess) {
+        g_last_cuda = (int)e;
+        boa_index_destroy(ix);
+        return e == cudaErrorMemoryAllocation ? BOA_ENOMEM : BOA_ECUDA;
+    }
+    *out = ix;
+    return BOA_OK;
+}
+
 int boa_index_destroy(boa_index* ix)
 {
     if (!ix) return BOA_OK;
-    cudaFree(ix->rec); cudaFree(ix->attr_cells); cudaFree(ix->graph); cudaFree(ix->lists); cudaFree(ix->counters);
+    if (!ix->shared) {
+        cudaFree(ix->rec); cudaFree(ix->attr_cells); cudaFree(ix->graph);
+        cudaFree(ix->pq_codes); cudaFree(ix->pq_pivots);
+    }
+    cudaFree(ix->lists); cudaFree(ix->counters);
     cudaFree(ix->stats); cudaFree(ix->spill); cudaFree(ix->spill_size);
-    cudaFree(ix->pq_codes); cudaFree(ix->pq_pivots); cudaFree(ix->qunit); cudaFree(ix->pen_scales);
+    cudaFree(ix->qunit); cudaFree(ix->pen_scales);
     cudaFree(ix->hq); cudaFree(ix->hlo); cudaFree(ix->hhi); cudaFree(ix->hids); cudaFree(ix->hd2);
     if (ix->side) cudaStreamDestroy(ix->side);
     if (ix->ev_fork) cudaEventDestroy(ix->ev_fork);
@@ -901,7 +940,7 @@ int boa_index_attach_pq(boa_index* ix, const float* pivots, const uint8_t* codes
     if (!ix || !pivots || !codes) return BOA_EINVAL;
     if (M < 16 || M > BOA_PQ_MAX_SUBSPACES || M % 16 != 0 || ix->D % M != 0) return BOA_EINVAL;
     if (K < 1 || K > 256) return BOA_EINVAL;
-    if (!aligned16(pivots) || !aligned16(codes) || !on_device(ix->device)) return BOA_EINVAL;
+    if (!aligned16(pivots) || !aligned16(codes) || !on_device(ix->device) || ix->shared) return BOA_EINVAL;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     cudaFree(ix->pq_codes); cudaFree(ix->pq_pivots);
     ix->pq_codes = nullptr; ix->pq_pivots = nullptr; ix->pq_M = 0; ix->pq_K = 0; ix->use_pq = 0;
@@ -940,7 +979,7 @@ int boa_index_set_metric(boa_index* ix, int metric, void* stream)
     if (!ix || (metric != BOA_METRIC_L2 && metric != BOA_METRIC_COSINE)) return BOA_EINVAL;
     if (metric == ix->metric) return BOA_OK;
     // the rows are rescaled in place, once: there is no way back to the Euclidean metric
-    if (ix->metric != BOA_METRIC_L2 || ix->vec_dtype != BOA_F32 || !on_device(ix->device)) return BOA_EINVAL;
+    if (ix->metric != BOA_METRIC_L2 || ix->vec_dtype != BOA_F32 || !on_device(ix->device) || ix->shared) return BOA_EINVAL;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     float* rows = reinterpret_cast<float*>(ix->rec);
     unit_rows_kernel<<<ix->num_sms * 8, 128, 0, st>>>(rows, ix->rec_stride / 4, rows, ix->rec_stride / 4, ix->N, ix->D);
