@@ -16,7 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB = None
 
 PARAM = dict(eps=0, growth=1, tau=2, mode=3, plus_k=4, cap_mult=5, cap_add=6, table_kb=7,
-             max_warps_per_sm=8, expand_w=9, table_tags=10, lam=11, pq=12, host_in_place=13, plus_min_sub=14)
+             max_warps_per_sm=8, expand_w=9, table_tags=10, lam=11, pq=12, host_in_place=13, plus_min_sub=14, chains=15)
 F32, U8 = 0, 1
 NO_ID = 0xFFFFFFFF
 

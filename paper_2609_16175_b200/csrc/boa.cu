@@ -201,6 +201,8 @@ struct boa_index {
     float* hq = nullptr; int32_t* hlo = nullptr; int32_t* hhi = nullptr; uint32_t* hids = nullptr; float* hd2 = nullptr;
     int64_t ws_host_Q = 0;
     int ws_host_k = 0;
+    int chains = 2;                    // 2: the batch is searched as two halves, each on a stream of its own; 1: as one
+    int last_split = 0;
     int64_t plus_min_sub = 0;          // smallest BOA+ sub-batch; 0 = twice the resident query warps
     int host_in_place = 1;             // boa_search_host reads mapped page-locked buffers in place
     float* qunit = nullptr;            // [ws_qunit][D] unit-length copies of a batch's queries (cosine)
@@ -439,7 +441,7 @@ struct LaunchPlan {
 // pooled escalation of BOA+); phase 1 always reads the one list the first phase wrote.
 int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_ptr,
                  const uint32_t* end_ptr, uint32_t begin, uint32_t end, uint32_t expected_items,
-                 int chain = 0, bool use_active_count = true)
+                 int chain = 0, bool use_active_count = true, bool own_first = false)
 {
     boa_index* ix = lp.ix;
     if (lp.launches >= kMaxLaunches) return BOA_EINVAL;
@@ -460,7 +462,8 @@ int launch_phase(LaunchPlan& lp, int p, cudaStream_t st, const uint32_t* begin_p
     sp.spill_out = (ix->mode == 1 && !sp.last_phase);
     uint32_t* lists_c = ix->lists + (size_t)chain * BOA_MAX_PHASES * ix->ws_Q;
     uint32_t* cnt_c = ix->counters + (chain == 0 ? kCntCount : kCntCount2);
-    sp.in_list = p == 0 ? nullptr : (p == 1 ? ix->lists : lists_c) + (size_t)p * ix->ws_Q;
+    // own_first: the chain's first phase wrote the chain's own phase-1 list (two-chain schedule)
+    sp.in_list = p == 0 ? nullptr : ((p == 1 && !own_first) ? ix->lists : lists_c) + (size_t)p * ix->ws_Q;
     sp.in_begin_ptr = begin_ptr;
     sp.in_end_ptr = end_ptr;
     sp.in_begin = begin;
@@ -727,6 +730,9 @@ int boa_set_param(boa_index* ix, int key, double v)
         case BOA_PARAM_PQ:
             if ((v != 0.0 && v != 1.0) || (v == 1.0 && !ix->pq_codes)) return BOA_EINVAL;
             ix->use_pq = (int)v; return BOA_OK;
+        case BOA_PARAM_CHAINS:
+            if (v != 1.0 && v != 2.0) return BOA_EINVAL;
+            ix->chains = (int)v; return BOA_OK;
         case BOA_PARAM_PLUS_MIN_SUB:
             if (v < 0.0 || v > 2147483647.0 || v != floor(v)) return BOA_EINVAL;
             ix->plus_min_sub = (int64_t)v; return BOA_OK;
@@ -864,7 +870,31 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
     }
     uint32_t* cnt = ix->counters + kCntCount;
     uint32_t* snap = ix->counters + kCntSnap;
-    if (K == 1) {
+    ix->last_split = 0;
+    if (K == 1 && ix->chains == 2 && lp.n_phases > 1 && ix->tau == 0.0 && Q >= 2) {
+        // Two chains: the halves of the batch go through all their phases independently, one on
+        // the caller's stream, one on the side stream, each with its own survivor lists and
+        // counters.  A query's phases depend on each other, different queries' do not: while
+        // the partly empty last wave of one half's phase drains, the other half's launches fill
+        // the GPU.  Every query is searched exactly as in the one-chain schedule.
+        ix->last_split = 1;
+        BOA_CUDA(cudaEventRecord(ix->ev_fork, st));
+        BOA_CUDA(cudaStreamWaitEvent(ix->side, ix->ev_fork, 0));
+        const uint32_t half = (uint32_t)(Q / 2);
+        for (int c = 0; c < 2; ++c) {
+            cudaStream_t cs = c == 0 ? st : ix->side;
+            const uint32_t b0 = c == 0 ? 0u : half, b1 = c == 0 ? half : (uint32_t)Q;
+            uint32_t* cnt_c = ix->counters + (c == 0 ? kCntCount : kCntCount2);
+            rc = launch_phase(lp, 0, cs, nullptr, nullptr, b0, b1, b1 - b0, c, false, true);
+            if (rc != BOA_OK) return rc;
+            for (int p = 1; p < lp.n_phases; ++p) {
+                rc = launch_phase(lp, p, cs, nullptr, cnt_c + p, 0u, 0u, b1 - b0, c, false, true);
+                if (rc != BOA_OK) return rc;
+            }
+        }
+        BOA_CUDA(cudaEventRecord(ix->ev_join, ix->side));
+        BOA_CUDA(cudaStreamWaitEvent(st, ix->ev_join, 0));
+    } else if (K == 1) {
         // BOA: one launch per phase, each over the survivors of the one before
         rc = launch_phase(lp, 0, st, nullptr, nullptr, 0u, (uint32_t)Q, (uint32_t)Q);
         if (rc != BOA_OK) return rc;
@@ -1012,7 +1042,7 @@ int boa_get_phase_counts(boa_index* ix, int64_t* active, int n, int* n_phases, v
     const double tau_q = ix->tau * (double)ix->last_Q;
     bool stopped = false;
     for (int p = 0; p < n && p < ix->last_phases; ++p) {
-        const int64_t a = p == 0 ? ix->last_Q : (int64_t)h[p] + (p >= 2 ? (int64_t)h2[p] : 0);
+        const int64_t a = p == 0 ? ix->last_Q : (int64_t)h[p] + ((p >= 2 || ix->last_split) ? (int64_t)h2[p] : 0);
         if (!((double)a > tau_q)) stopped = true;
         active[p] = stopped ? 0 : a;
     }
@@ -1098,9 +1128,9 @@ int boa_search_noalloc(boa_index* ix, const float* queries, int64_t Q, const voi
     struct Saved {
         uint32_t *lists, *counters; int32_t *stats, *spill_size; uint64_t* spill;
         int64_t ws_Q; int ws_spill;
-        int64_t last_Q; int last_phases, last_launches; int last_widths[BOA_MAX_PHASES];
+        int64_t last_Q; int last_phases, last_launches, last_split; int last_widths[BOA_MAX_PHASES];
     } sv = {ix->lists, ix->counters, ix->stats, ix->spill_size, ix->spill, ix->ws_Q, ix->ws_spill,
-            ix->last_Q, ix->last_phases, ix->last_launches, {0}};
+            ix->last_Q, ix->last_phases, ix->last_launches, ix->last_split, {0}};
     memcpy(sv.last_widths, ix->last_widths, sizeof(sv.last_widths));
     ix->counters = reinterpret_cast<uint32_t*>(base + kNaCounters);
     ix->lists = reinterpret_cast<uint32_t*>(base + kNaLists);
@@ -1115,6 +1145,7 @@ int boa_search_noalloc(boa_index* ix, const float* queries, int64_t Q, const voi
     // boa_get_stats / boa_get_phase_counts keep describing the last boa_search: this call's
     // statistics sit in the shared array, which the next call overwrites
     ix->last_Q = sv.last_Q; ix->last_phases = sv.last_phases; ix->last_launches = sv.last_launches;
+    ix->last_split = sv.last_split;
     memcpy(ix->last_widths, sv.last_widths, sizeof(sv.last_widths));
     return rc;
 }

@@ -30,12 +30,13 @@ def make_pair(d, entry=-1):
 
 
 def gpu_search(gpu, g, k, widths, mode="restart", eps=0.05, tau=0.0, plus_k=0, cap=(8, 64),
-               sel=None, expand_w=1, lam=float("inf"), pq=False, penalty_scales=None):
+               sel=None, expand_w=1, lam=float("inf"), pq=False, penalty_scales=None, chains=2):
     gpu.set_param("mode", 1 if mode == "resume" else 0)
     gpu.set_param("eps", eps)
     gpu.set_param("tau", tau)
     gpu.set_param("plus_k", plus_k)
     gpu.set_param("plus_min_sub", 1)          # tests want K sub-batches whatever the batch size
+    gpu.set_param("chains", chains)
     gpu.set_param("cap_mult", cap[0])
     gpu.set_param("cap_add", cap[1])
     gpu.set_param("expand_w", expand_w)

@@ -185,14 +185,44 @@ def test_boa_plus_equals_boa(name, plus_k):
         assert (a["phase_active"] == b["phase_active"]).all()
 
 
+@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c5"])
+def test_two_chains_equal_one(name):
+    """BOA_PARAM_CHAINS = 2: the halves of the batch go through their phases on two streams;
+    ids, distances, statistics and phase counts are those of the one-chain schedule (and of the
+    oracle), for even, odd and tiny batches, with PQ-free exact search in both modes."""
+    w, d, orc, gpu, g = _get(name)
+    widths = default_widths(w.L0, 256)
+    for mode in ("restart", "resume"):
+        a = gpu_search(gpu, g, w.k, widths, mode=mode, chains=1)
+        assert gpu.last_launch_count == len(widths)
+        b = gpu_search(gpu, g, w.k, widths, mode=mode, chains=2)
+        assert gpu.last_launch_count == 2 * len(widths)
+        for key in ("ids", "final_L", "n_expand", "n_scored", "flags", "phase_active"):
+            assert (a[key] == b[key]).all(), key
+        assert (a["d2"].view(np.uint32) == b["d2"].view(np.uint32)).all()
+    o = orc.search(d["queries"][:31], d["lo"][:31], d["hi"][:31], w.k, widths, mode="resume", dist_mode=1)
+    r = gpu_search(gpu, g, w.k, widths, mode="resume", chains=2, sel=slice(0, 31))
+    assert_bit_parity(o, r, f"two chains {name}")
+    for n in (1, 2, 3):
+        a = gpu_search(gpu, g, w.k, widths, mode="resume", chains=1, sel=slice(0, n))
+        b = gpu_search(gpu, g, w.k, widths, mode="resume", chains=2, sel=slice(0, n))
+        assert (a["ids"] == b["ids"]).all() and (a["phase_active"] == b["phase_active"]).all()
+    # a finite lambda, two nodes per iteration and BOA+ (which takes precedence) still work with it set
+    a = gpu_search(gpu, g, w.k, widths, mode="resume", lam=500.0, expand_w=2, chains=1)
+    b = gpu_search(gpu, g, w.k, widths, mode="resume", lam=500.0, expand_w=2, chains=2)
+    c = gpu_search(gpu, g, w.k, widths, mode="resume", lam=500.0, expand_w=2, chains=2, plus_k=3)
+    assert (a["ids"] == b["ids"]).all() and (a["ids"] == c["ids"]).all()
+    assert (a["phase_active"] == b["phase_active"]).all() and (a["phase_active"] == c["phase_active"]).all()
+
+
 def test_boa_plus_sub_batches_are_not_made_smaller_than_the_gpu():
     """With the default smallest sub-batch (twice the resident query warps) a batch of a few
     hundred queries runs as plain BOA whatever K says; plus_min_sub = 1 gives the K sub-batches."""
     w, d, orc, gpu, g = _get("c2")
     widths = default_widths(w.L0, 256)
-    a = gpu_search(gpu, g, w.k, widths, mode="resume", plus_k=0)
+    a = gpu_search(gpu, g, w.k, widths, mode="resume", plus_k=0, chains=1)
     boa_launches = gpu.last_launch_count
-    b = gpu_search(gpu, g, w.k, widths, mode="resume", plus_k=5)
+    b = gpu_search(gpu, g, w.k, widths, mode="resume", plus_k=5, chains=1)
     assert gpu.last_launch_count > boa_launches
     gpu.set_param("plus_min_sub", 0)
     ids, d2 = gpu.search(g["queries"], g["lo"], g["hi"], w.k, widths[0], widths[-1])
