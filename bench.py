@@ -118,9 +118,9 @@ def parse_args():
     ap.add_argument("--no-per-config", action="store_true",
                     help="measure the headline workload only (always so with more than one GPU)")
     ap.add_argument("--plus-k", type=int, default=0)
-    ap.add_argument("--chains", type=int, default=2, choices=[1, 2],
-                    help="2 (the library's default): the halves of a batch go through their phases on two "
-                         "streams; 1: the batch as one (BOA_PARAM_CHAINS)")
+    ap.add_argument("--chains", type=int, default=0, choices=[0, 1, 2],
+                    help="2: the halves of a batch go through their phases on two streams; 1: the batch as one; "
+                         "0 (the library's default): 2 while the widest phase is at most 128 (BOA_PARAM_CHAINS)")
     ap.add_argument("--plus-min-sub", type=int, default=0,
                     help="BOA+: fewest queries per sub-batch (0 = the library's default, twice the resident "
                          "query warps; 1 = always K sub-batches)")
@@ -386,7 +386,7 @@ def configure(ix, args, widths, d=None):
     ix.set_param("eps", args.eps)
     ix.set_param("plus_k", args.plus_k)
     ix.set_param("plus_min_sub", getattr(args, "plus_min_sub", 0))
-    ix.set_param("chains", getattr(args, "chains", 2))
+    ix.set_param("chains", getattr(args, "chains", 0))
     ix.set_param("expand_w", args.expand_w)
     ix.set_param("lam", args.lam)
     ix.set_param("table_kb", args.table_kb)

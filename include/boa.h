@@ -85,16 +85,17 @@ enum {
                                line and the "Re-rank exact" step of Section "BOA Implementation
                                on a GPU System".  0 (default) = exact distances throughout.
                                With 1, k <= BOA_PQ_MAX_K and BOA_PARAM_EXPAND_W must be 1.     */
-    BOA_PARAM_CHAINS = 15,  /* 2 (default): the two halves of the batch go through all their
-                               phases independently, one on the caller's stream and one on a
-                               stream of the index, joined before `stream` goes on: the launches
-                               of one half fill the GPU while the last, partly empty wave of
-                               the other half's phase drains (the observation of "Pipelining
-                               Multiple Batches": phases of different queries do not depend on
-                               each other).  1: the batch goes through its phases as one, the
-                               schedule of Algorithm 1 as printed.  Same results either way.
-                               2 applies when BOA+ is off, tau is 0 and the schedule has more
-                               than one phase.                                               */
+    BOA_PARAM_CHAINS = 15,  /* 2: the two halves of the batch go through all their phases
+                               independently, one on the caller's stream and one on a stream of
+                               the index, joined before `stream` goes on: the launches of one
+                               half fill the GPU while the last, partly empty wave of the other
+                               half's phase drains (the observation of "Pipelining Multiple
+                               Batches": phases of different queries do not depend on each
+                               other).  1: the batch goes through its phases as one, the
+                               schedule of Algorithm 1 as printed.  0 (default): 2 while the
+                               widest phase is at most 128, else 1.  Same results in every
+                               case.  Two chains need BOA+ off, tau = 0 and more than one
+                               phase.                                                        */
     BOA_PARAM_PLUS_MIN_SUB = 14, /* BOA+: the fewest queries a sub-batch may hold; K is lowered
                                (down to plain BOA) until Q / K reaches it.  0 (default) = twice
                                the queries the GPU searches at once (2 x 20 x SM count); 1 =

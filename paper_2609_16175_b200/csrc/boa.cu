@@ -201,7 +201,7 @@ struct boa_index {
     float* hq = nullptr; int32_t* hlo = nullptr; int32_t* hhi = nullptr; uint32_t* hids = nullptr; float* hd2 = nullptr;
     int64_t ws_host_Q = 0;
     int ws_host_k = 0;
-    int chains = 2;                    // 2: the batch is searched as two halves, each on a stream of its own; 1: as one
+    int chains = 0;                    // 2: the batch is searched as two halves, each on a stream of its own; 1: as one; 0: chosen per call
     int last_split = 0;
     int64_t plus_min_sub = 0;          // smallest BOA+ sub-batch; 0 = twice the resident query warps
     int host_in_place = 1;             // boa_search_host reads mapped page-locked buffers in place
@@ -731,7 +731,7 @@ int boa_set_param(boa_index* ix, int key, double v)
             if ((v != 0.0 && v != 1.0) || (v == 1.0 && !ix->pq_codes)) return BOA_EINVAL;
             ix->use_pq = (int)v; return BOA_OK;
         case BOA_PARAM_CHAINS:
-            if (v != 1.0 && v != 2.0) return BOA_EINVAL;
+            if (v != 0.0 && v != 1.0 && v != 2.0) return BOA_EINVAL;
             ix->chains = (int)v; return BOA_OK;
         case BOA_PARAM_PLUS_MIN_SUB:
             if (v < 0.0 || v > 2147483647.0 || v != floor(v)) return BOA_EINVAL;
@@ -871,7 +871,10 @@ int boa_search(boa_index* ix, const float* queries, int64_t Q, const void* lo, c
     uint32_t* cnt = ix->counters + kCntCount;
     uint32_t* snap = ix->counters + kCntSnap;
     ix->last_split = 0;
-    if (K == 1 && ix->chains == 2 && lp.n_phases > 1 && ix->tau == 0.0 && Q >= 2) {
+    // chosen per call: two chains while the widest phase is at most 128 (measured: with wider last
+    // phases one query per warp slot lasts so long that splitting the batch only delays the second half)
+    const int chains = ix->chains != 0 ? ix->chains : (lp.widths[lp.n_phases - 1] <= 128 ? 2 : 1);
+    if (K == 1 && chains == 2 && lp.n_phases > 1 && ix->tau == 0.0 && Q >= 2) {
         // Two chains: the halves of the batch go through all their phases independently, one on
         // the caller's stream, one on the side stream, each with its own survivor lists and
         // counters.  A query's phases depend on each other, different queries' do not: while

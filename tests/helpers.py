@@ -30,7 +30,7 @@ def make_pair(d, entry=-1):
 
 
 def gpu_search(gpu, g, k, widths, mode="restart", eps=0.05, tau=0.0, plus_k=0, cap=(8, 64),
-               sel=None, expand_w=1, lam=float("inf"), pq=False, penalty_scales=None, chains=2):
+               sel=None, expand_w=1, lam=float("inf"), pq=False, penalty_scales=None, chains=0):
     gpu.set_param("mode", 1 if mode == "resume" else 0)
     gpu.set_param("eps", eps)
     gpu.set_param("tau", tau)
