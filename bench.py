@@ -637,6 +637,9 @@ def main():
     if world == 1:
         ix2 = ix.share()
         configure(ix2, args, widths)
+        # with two batches in flight each batch runs as one chain: the other batch already fills the tails
+        ix.set_param("chains", 1)
+        ix2.set_param("chains", 1)
         pair = ((ix, torch.cuda.Stream(), out_ids, out_d2),
                 (ix2, torch.cuda.Stream(), torch.empty_like(out_ids), torch.empty_like(out_d2)))
         def pipelined_steps(n):
@@ -661,8 +664,9 @@ def main():
         pipelined = {"handles": 2, "streams": 2, "steps": args.steps, "ms_per_step": p_ms,
                      "value": Q / (p_ms / 1e3), "unit": UNIT, "same_results": same,
                      "note": "value above is one batch at a time on one stream; this is the same work with "
-                             "the next batch's launches enqueued on a second stream and handle"}
+                             "the next batch's launches enqueued on a second stream and handle (each batch as one chain)"}
         ix2.close()
+        ix.set_param("chains", getattr(args, "chains", 0))
 
     # ---- end to end through the public call: pinned host inputs in, results out, every step
     hq = torch.from_numpy(d["queries"]).pin_memory()
@@ -684,6 +688,8 @@ def main():
     if pipelined is not None:
         ix3 = ix.share()
         configure(ix3, args, widths)
+        ix.set_param("chains", 1)
+        ix3.set_param("chains", 1)
         lanes = ((ix, torch.cuda.Stream(), h_ids, h_d2),
                  (ix3, torch.cuda.Stream(), torch.empty_like(h_ids).pin_memory(), torch.empty_like(h_d2).pin_memory()))
         def lane_steps(lane, n):
@@ -707,6 +713,7 @@ def main():
         pipelined["e2e_note"] = (f"{2 * half} boa_search_host calls from two host threads (wall clock: every call "
                                  "returns with its results readable)")
         ix3.close()
+        ix.set_param("chains", getattr(args, "chains", 0))
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
