@@ -468,6 +468,10 @@ def measure_config(name, args, dev, steps, cpu_seconds, variants=({},), gt_queri
         n_rr = ix.rerank_counts().cpu().numpy() if pq_M else None
         alg = algorithmic_bytes(w, st, ql["unique_ratio"], a.mode, widths, pq_M, n_rr)
         ms = total_ms / n_steps
+        in_flight = None
+        if not var and name in ("c2", "c3", "c4"):
+            a.chains = 0
+            in_flight = two_in_flight(ix, t, w.k, widths, a, n_steps, 4, out_ids, out_d2, ids_np)
         key = name + (f"_pq{pq_M}" if pq_M else "") + (f"_fixed{fixed_L}" if fixed_L else "") + \
             (f"_{var['tag']}" if var.get("tag") else "")
         res[key] = {
@@ -486,6 +490,8 @@ def measure_config(name, args, dev, steps, cpu_seconds, variants=({},), gt_queri
             "frac": alg / (ms / 1e3) / 1e9 / peak, "peak_kind": peak_kind,
             "parity_with_oracle_on_sample": ql["parity"], "oracle_sample_queries": ql["cpu_n"],
             "cpu_oracle_queries_per_s": ql["cpu_qps"], "gpu_launches_per_step": ix.last_launch_count,
+            "two_batches_in_flight": ({"ms_per_step": in_flight["ms_per_step"], "queries_per_s": in_flight["value"],
+                                       "same_results": in_flight["same_results"]} if in_flight else None),
             "device_status": ix.device_status(), "fixture_build_s": round(t_build, 1)}
     ix.close()
     del ix, out_ids, out_d2
@@ -498,6 +504,48 @@ def measure_config(name, args, dev, steps, cpu_seconds, variants=({},), gt_queri
     del t, d
     torch.cuda.empty_cache()
     return res
+
+
+def two_in_flight(ix, t, k, widths, args, steps, warmup, out_ids, out_d2, ids_np):
+    """The same steps with two batches in flight: two handles on the index (boa_index_share),
+    steps alternating between two streams, so that the partly empty last wave of one batch's
+    wide phase overlaps the narrow phase of the next batch.  Each batch runs as one chain: the
+    other batch already fills the tails."""
+    import torch
+    Q = t["queries"].shape[0]
+    ix2 = ix.share()
+    configure(ix2, args, widths)
+    ix.set_param("chains", 1)
+    ix2.set_param("chains", 1)
+    pair = ((ix, torch.cuda.Stream(), out_ids, out_d2),
+            (ix2, torch.cuda.Stream(), torch.empty_like(out_ids), torch.empty_like(out_d2)))
+
+    def run(n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _, s_, _, _ in pair:
+            s_.wait_event(e0)
+        for i in range(n):
+            h_, s_, oi, od = pair[i % 2]
+            h_.search(t["queries"], t["lo"], t["hi"], k, widths[0], widths[-1], oi, od, stream=s_)
+        for _, s_, _, _ in pair:
+            ev = torch.cuda.Event()
+            ev.record(s_)
+            torch.cuda.current_stream().wait_event(ev)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    run(warmup)
+    p_ms = run(steps) / steps
+    same = bool((pair[1][2].cpu().numpy().view(np.uint32) == ids_np).all()
+                and (pair[0][2].cpu().numpy().view(np.uint32) == ids_np).all())
+    ix2.close()
+    ix.set_param("chains", getattr(args, "chains", 0))
+    return {"handles": 2, "streams": 2, "steps": steps, "ms_per_step": p_ms, "value": Q / (p_ms / 1e3),
+            "unit": UNIT, "same_results": same,
+            "note": "value above is one batch at a time on one stream; this is the same work with the next "
+                    "batch's launches enqueued on a second stream and handle (each batch as one chain)"}
 
 
 def attribute_positions(attrs, types):
@@ -635,38 +683,7 @@ def main():
     # wide phase overlaps the narrow phase of the next batch
     pipelined = None
     if world == 1:
-        ix2 = ix.share()
-        configure(ix2, args, widths)
-        # with two batches in flight each batch runs as one chain: the other batch already fills the tails
-        ix.set_param("chains", 1)
-        ix2.set_param("chains", 1)
-        pair = ((ix, torch.cuda.Stream(), out_ids, out_d2),
-                (ix2, torch.cuda.Stream(), torch.empty_like(out_ids), torch.empty_like(out_d2)))
-        def pipelined_steps(n):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            for _, s_, _, _ in pair:
-                s_.wait_event(e0)
-            for i in range(n):
-                h_, s_, oi, od = pair[i % 2]
-                h_.search(t["queries"], t["lo"], t["hi"], k, widths[0], widths[-1], oi, od, stream=s_)
-            for _, s_, _, _ in pair:
-                ev = torch.cuda.Event()
-                ev.record(s_)
-                torch.cuda.current_stream().wait_event(ev)
-            e1.record()
-            torch.cuda.synchronize()
-            return e0.elapsed_time(e1)
-        pipelined_steps(max(4, 2 * args.warmup))
-        p_ms = pipelined_steps(args.steps) / args.steps
-        same = bool((pair[1][2].cpu().numpy().view(np.uint32) == ids_np).all()
-                    and (pair[0][2].cpu().numpy().view(np.uint32) == ids_np).all())
-        pipelined = {"handles": 2, "streams": 2, "steps": args.steps, "ms_per_step": p_ms,
-                     "value": Q / (p_ms / 1e3), "unit": UNIT, "same_results": same,
-                     "note": "value above is one batch at a time on one stream; this is the same work with "
-                             "the next batch's launches enqueued on a second stream and handle (each batch as one chain)"}
-        ix2.close()
-        ix.set_param("chains", getattr(args, "chains", 0))
+        pipelined = two_in_flight(ix, t, k, widths, args, args.steps, max(4, 2 * args.warmup), out_ids, out_d2, ids_np)
 
     # ---- end to end through the public call: pinned host inputs in, results out, every step
     hq = torch.from_numpy(d["queries"]).pin_memory()
