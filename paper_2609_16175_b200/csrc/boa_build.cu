@@ -407,7 +407,7 @@ extern "C" int boa_graph_build(const void* vectors, int vec_dtype, int64_t N, in
                 if (rc != BOA_OK) goto done;
             }
             // (b) prune every point of the batch
-            prune_batch_kernel<<<(unsigned)(bsz < sms * 16 ? bsz : sms * 16), 32, 0, st>>>(bp, start, (int)bsz, cand_ids, Lb, B);
+            prune_batch_kernel<<<(unsigned)(bsz < sms * 32 ? bsz : sms * 32), 32, 0, st>>>(bp, start, (int)bsz, cand_ids, Lb, B);
             BUILD_CUDA(cudaGetLastError());
             // (c) reverse edges
             {
@@ -419,7 +419,7 @@ extern "C" int boa_graph_build(const void* vectors, int vec_dtype, int64_t N, in
                 BUILD_CUDA(cudaMemsetAsync(n_heads, 0, sizeof(uint32_t), st));
                 find_heads_kernel<<<sms * 2, 256, 0, st>>>(req_sorted, nreq, heads, n_heads);
                 BUILD_CUDA(cudaGetLastError());
-                reverse_edges_kernel<<<sms * 16, 32, 0, st>>>(bp, req_sorted, nreq, heads, n_heads, cap_in);
+                reverse_edges_kernel<<<sms * 32, 32, 0, st>>>(bp, req_sorted, nreq, heads, n_heads, cap_in);
                 BUILD_CUDA(cudaGetLastError());
             }
             start += bsz;
