@@ -111,7 +111,7 @@ def parse_args():
     ap.add_argument("--schedule", default="", help="phase widths; default: the workload's operating point")
     ap.add_argument("--built-graph", default="c2,c3,c4,c5",
                     help="workloads of per_config also measured over a graph built by boa_graph_build "
-                         "(comma list; the 10M-point build of c4 takes about 50 s, c5's 960-d one about 40 s)")
+                         "(comma list; the 10M-point build of c4 takes about 40 s, c5's 960-d one about 25 s)")
     ap.add_argument("--graph-build-only", action="store_true",
                     help="time boa_graph_build on the workload (with --scale-n for a small case), search the "
                          "built graph at BUILT_GRAPH's settings and print that entry alone")
