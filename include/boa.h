@@ -58,7 +58,9 @@ enum {
     BOA_PARAM_CAP_MULT = 5, /* a phase at width L gives up after CAP_MULT*L + CAP_ADD        */
     BOA_PARAM_CAP_ADD = 6,  /*   expansions; defaults 8 and 64                               */
     BOA_PARAM_TABLE_KB = 7, /* 0 = default (6 or 4, whichever keeps 20 query warps per SM
-                               within 196 KB of shared memory); else KB of shared memory
+                               within 196 KB of shared memory; 1 with PQ traversal, where the
+                               distance table decides how many warps fit and a node scored
+                               twice costs little); else KB of shared memory
                                per query for the table of recently scored ids: 1, 2, 3, 4,
                                6, 8, 12, 16 or 24 (doubled automatically while an index of
                                more than 2^25 points needs tags wider than 16 bits).  Never
