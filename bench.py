@@ -40,8 +40,8 @@ UNIT = "queries/s"
 # the line reports "traffic": null until the capture is repeated.
 NCU_DRAM_BYTES_PER_SCORED = {
     # workload: (bytes per scored record, sha256[:12] of csrc/boa_search.cuh, summary file)
-    "c2": (410.0, "633158171c92", "profiles/boa_search_kernel_c2_dram_traffic.md"),
-    "c3": (312.7, "633158171c92", "profiles/boa_search_kernel_c3_dram_traffic.md"),
+    "c2": (409.8, "bd70335f918a", "profiles/boa_search_kernel_c2_dram_traffic.md"),
+    "c3": (312.7, "bd70335f918a", "profiles/boa_search_kernel_c3_dram_traffic.md"),
 }
 
 # Operating point of each workload: explicit phase widths and eps, chosen from the sweeps in

@@ -299,11 +299,11 @@ template <int VT, int CPL, int W, bool PQ, bool EXT>
 KernelChoice pick_rn(int R, bool exact)
 {
     if (R <= 32) {
-        if (exact) return {boa::boa_search_kernel<VT, 1, W, CPL, (CPL > 0), PQ, EXT>, W, CPL == 0};
-        return {boa::boa_search_kernel<VT, 1, W, CPL, false, PQ, EXT>, W, CPL == 0};
+        if (exact) return {boa::boa_search_kernel<VT, 1, W, CPL, (CPL > 0), PQ, EXT>, W, CPL == 0 && !PQ};
+        return {boa::boa_search_kernel<VT, 1, W, CPL, false, PQ, EXT>, W, CPL == 0 && !PQ};
     }
-    if (exact) return {boa::boa_search_kernel<VT, 2, W, CPL, (CPL > 0), PQ, EXT>, 2 * W, CPL == 0};
-    return {boa::boa_search_kernel<VT, 2, W, CPL, false, PQ, EXT>, 2 * W, CPL == 0};
+    if (exact) return {boa::boa_search_kernel<VT, 2, W, CPL, (CPL > 0), PQ, EXT>, 2 * W, CPL == 0 && !PQ};
+    return {boa::boa_search_kernel<VT, 2, W, CPL, false, PQ, EXT>, 2 * W, CPL == 0 && !PQ};
 }
 template <int VT, int CPL>
 KernelChoice pick_rs(int R, bool exact, int expand_w, bool pq, bool ext)

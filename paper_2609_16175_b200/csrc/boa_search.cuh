@@ -386,7 +386,7 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
     constexpr int QF4 = (VT == 0) ? 1 : 4;          // float4 slices of the query per chunk
     constexpr int NQ = (CPL > 0) ? CPL * QF4 : 1;
 
-    const WarpSmem lay = warp_smem_layout(p.C, p.table_bytes, p.D, RS, CPL == 0, PQ ? p.pq_M * p.pq_K : 0);
+    const WarpSmem lay = warp_smem_layout(p.C, p.table_bytes, p.D, RS, CPL == 0 && !PQ, PQ ? p.pq_M * p.pq_K : 0);
     float* pq_table = reinterpret_cast<float*>(smem_raw + lay.pq_off);
     uint64_t* topk = reinterpret_cast<uint64_t*>(smem_raw + lay.top_off);
     uint64_t* pool = reinterpret_cast<uint64_t*>(smem_raw + lay.pool_off);
@@ -419,7 +419,10 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
 
         // ---- load the query, its bounds; clear the table of scored ids
         {
-            if (CPL == 0) {
+            // PQ traversal needs the whole query only for the final exact ranking: it is read
+            // from global memory there and its shared-memory copy is left out (the per-query
+            // distance table decides how many warps fit)
+            if (CPL == 0 && !PQ) {
                 const float4* qsrc = reinterpret_cast<const float4*>(p.queries + (size_t)qi * p.D);
                 for (int i = lane; i < p.D / 4; i += 32) qs[i] = qsrc[i];
             }
@@ -437,6 +440,7 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
         const bool pen_on = EXT && p.pen_scales != nullptr;
         const float my_scale = (pen_on && g < p.m) ? __ldg(p.pen_scales + g) : 0.0f;
         __syncwarp();
+        const float4* qglob = reinterpret_cast<const float4*>(p.queries + (size_t)qi * p.D);   // PQ, long rows
         float4 qreg[NQ];           // this lane's slices of the query (CPL > 0)
         if (CPL > 0) {
             const float4* qsrc = reinterpret_cast<const float4*>(p.queries + (size_t)qi * p.D);
@@ -741,18 +745,22 @@ __global__ void __launch_bounds__(kThreads, (PQ ? 8 : BOA_MIN_CTAS)) boa_search_
                             const int c = c0 + 8 * i;
                             if (c < p.nchunks) {
                                 if (VT == 0) {
-                                    const float4 qq = qs[c];
+                                    const float4 qq = PQ ? __ldg(qglob + c) : qs[c];
                                     a0 = sq_acc4u(a0, x0[i], qq);
                                     a1 = sq_acc4u(a1, x1[i], qq);
                                 } else {
-                                    a0 = sq_acc_bytes(a0, x0[i].x, qs[4 * c + 0]);
-                                    a1 = sq_acc_bytes(a1, x1[i].x, qs[4 * c + 0]);
-                                    a0 = sq_acc_bytes(a0, x0[i].y, qs[4 * c + 1]);
-                                    a1 = sq_acc_bytes(a1, x1[i].y, qs[4 * c + 1]);
-                                    a0 = sq_acc_bytes(a0, x0[i].z, qs[4 * c + 2]);
-                                    a1 = sq_acc_bytes(a1, x1[i].z, qs[4 * c + 2]);
-                                    a0 = sq_acc_bytes(a0, x0[i].w, qs[4 * c + 3]);
-                                    a1 = sq_acc_bytes(a1, x1[i].w, qs[4 * c + 3]);
+                                    const float4 q0 = PQ ? __ldg(qglob + 4 * c + 0) : qs[4 * c + 0];
+                                    const float4 q1 = PQ ? __ldg(qglob + 4 * c + 1) : qs[4 * c + 1];
+                                    const float4 q2 = PQ ? __ldg(qglob + 4 * c + 2) : qs[4 * c + 2];
+                                    const float4 q3 = PQ ? __ldg(qglob + 4 * c + 3) : qs[4 * c + 3];
+                                    a0 = sq_acc_bytes(a0, x0[i].x, q0);
+                                    a1 = sq_acc_bytes(a1, x1[i].x, q0);
+                                    a0 = sq_acc_bytes(a0, x0[i].y, q1);
+                                    a1 = sq_acc_bytes(a1, x1[i].y, q1);
+                                    a0 = sq_acc_bytes(a0, x0[i].z, q2);
+                                    a1 = sq_acc_bytes(a1, x1[i].z, q2);
+                                    a0 = sq_acc_bytes(a0, x0[i].w, q3);
+                                    a1 = sq_acc_bytes(a1, x1[i].w, q3);
                                 }
                             }
                         }
