@@ -220,7 +220,8 @@ int boa_index_set_metric(boa_index* index, int metric, void* stream);
  * Rules: `src` must be fully set up before (boa_index_attach_pq and boa_index_set_metric are
  * BOA_EINVAL on a shared handle, and calling them on `src` afterwards is not seen by, or
  * breaks, its shares) and must outlive every handle shared from it; each handle is used by
- * one search at a time; parameters set on one handle do not reach the other.
+ * one search at a time, and `src` is not being searched by another thread while it is shared;
+ * parameters set on one handle do not reach the other.
  * Errors: BOA_EINVAL, BOA_ENOMEM, BOA_ECUDA; *out is NULL then.
  */
 int boa_index_share(boa_index** out, boa_index* src);

@@ -126,7 +126,7 @@ def build_graph(vectors: torch.Tensor, attr_pos: torch.Tensor, R: int, Lb: int, 
     m_pos = attr_pos.shape[1]
     flat = []
     for t in thresholds:
-        row = [float(t)] * m_pos if isinstance(t, (int, float)) else [float(x) for x in t]
+        row = [float(x) for x in t] if hasattr(t, "__len__") else [float(t)] * m_pos
         if len(row) != m_pos:
             raise ValueError("a threshold needs one value per attribute")
         flat += row
