@@ -339,6 +339,11 @@ extern "C" int boa_graph_build(const void* vectors, int vec_dtype, int64_t N, in
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     int rc = BOA_OK;
     boa_index* ix = nullptr;
+    // the searches of one batch (one per threshold) are independent: each runs on a handle and a
+    // stream of its own, so the partly empty last wave of one overlaps the others
+    boa_index* shares[8] = {nullptr};
+    cudaStream_t side[8] = {nullptr};
+    cudaEvent_t ev_fork = nullptr, ev_join[8] = {nullptr};
     float *wlo = nullptr, *whi = nullptr;
     int types[BOA_MAX_ATTRS];
     uint32_t *empty = nullptr, *cand_ids = nullptr, *heads = nullptr, *n_heads = nullptr;
@@ -359,10 +364,17 @@ extern "C" int boa_graph_build(const void* vectors, int vec_dtype, int64_t N, in
     // the build's searches see the attribute positions as float attribute columns
     rc = boa_index_create(&ix, vectors, vec_dtype, N, D, attr_pos, types, m_pos, empty, R, entry, st);
     if (rc != BOA_OK) goto done;
-    BUILD_CUDA(cudaMalloc(&wlo, (size_t)B * m_pos * sizeof(float)));
-    BUILD_CUDA(cudaMalloc(&whi, (size_t)B * m_pos * sizeof(float)));
+    BUILD_CUDA(cudaMalloc(&wlo, (size_t)T * B * m_pos * sizeof(float)));
+    BUILD_CUDA(cudaMalloc(&whi, (size_t)T * B * m_pos * sizeof(float)));
+    BUILD_CUDA(cudaEventCreateWithFlags(&ev_fork, cudaEventDisableTiming));
+    for (int ti = 1; ti < T; ++ti) {
+        rc = boa_index_share(&shares[ti], ix);
+        if (rc != BOA_OK) goto done;
+        BUILD_CUDA(cudaStreamCreateWithFlags(&side[ti], cudaStreamNonBlocking));
+        BUILD_CUDA(cudaEventCreateWithFlags(&ev_join[ti], cudaEventDisableTiming));
+    }
     BUILD_CUDA(cudaMalloc(&cand_ids, (size_t)T * B * Lb * sizeof(uint32_t)));
-    BUILD_CUDA(cudaMalloc(&cand_d, (size_t)B * Lb * sizeof(float)));
+    BUILD_CUDA(cudaMalloc(&cand_d, (size_t)T * B * Lb * sizeof(float)));
     BUILD_CUDA(cudaMalloc(&req, (size_t)B * R * sizeof(unsigned long long)));
     BUILD_CUDA(cudaMalloc(&req_sorted, (size_t)B * R * sizeof(unsigned long long)));
     BUILD_CUDA(cudaMalloc(&heads, (size_t)B * R * sizeof(uint32_t)));
@@ -398,14 +410,23 @@ extern "C" int boa_graph_build(const void* vectors, int vec_dtype, int64_t N, in
                 BUILD_CUDA(cudaGetLastError());
                 q = qf;
             }
+            if (T > 1) BUILD_CUDA(cudaEventRecord(ev_fork, st));
             for (int ti = 0; ti < T; ++ti) {
+                cudaStream_t cs = ti == 0 ? st : side[ti];
+                boa_index* h = ti == 0 ? ix : shares[ti];
+                float* lo_t = wlo + (size_t)ti * B * m_pos;
+                float* hi_t = whi + (size_t)ti * B * m_pos;
+                if (ti > 0) BUILD_CUDA(cudaStreamWaitEvent(cs, ev_fork, 0));
                 ThresholdRow tr;
                 for (int j = 0; j < BOA_MAX_ATTRS; ++j) tr.t[j] = bp.thr[ti][j];
-                window_bounds_kernel<<<sms, 256, 0, st>>>(attr_pos, m_pos, start, (int)bsz, tr, wlo, whi);
+                window_bounds_kernel<<<sms, 256, 0, cs>>>(attr_pos, m_pos, start, (int)bsz, tr, lo_t, hi_t);
                 BUILD_CUDA(cudaGetLastError());
-                rc = boa_search(ix, q, bsz, wlo, whi, Lb, Lb, Lb, cand_ids + (size_t)ti * B * Lb, cand_d, st);
+                rc = boa_search(h, q, bsz, lo_t, hi_t, Lb, Lb, Lb, cand_ids + (size_t)ti * B * Lb,
+                                cand_d + (size_t)ti * B * Lb, cs);
                 if (rc != BOA_OK) goto done;
+                if (ti > 0) BUILD_CUDA(cudaEventRecord(ev_join[ti], cs));
             }
+            for (int ti = 1; ti < T; ++ti) BUILD_CUDA(cudaStreamWaitEvent(st, ev_join[ti], 0));
             // (b) prune every point of the batch
             prune_batch_kernel<<<(unsigned)(bsz < sms * 32 ? bsz : sms * 32), 32, 0, st>>>(bp, start, (int)bsz, cand_ids, Lb, B);
             BUILD_CUDA(cudaGetLastError());
@@ -432,6 +453,12 @@ extern "C" int boa_graph_build(const void* vectors, int vec_dtype, int64_t N, in
     if (n_batches) *n_batches = batches;
 done:
     if (rc != BOA_OK) cudaStreamSynchronize(st);
+    for (int ti = 1; ti < 8; ++ti) {
+        if (side[ti]) { cudaStreamSynchronize(side[ti]); cudaStreamDestroy(side[ti]); }
+        if (ev_join[ti]) cudaEventDestroy(ev_join[ti]);
+        if (shares[ti]) boa_index_destroy(shares[ti]);
+    }
+    if (ev_fork) cudaEventDestroy(ev_fork);
     if (ix) boa_index_destroy(ix);
     cudaFree(wlo); cudaFree(whi); cudaFree(empty); cudaFree(cand_ids); cudaFree(cand_d); cudaFree(req);
     cudaFree(req_sorted); cudaFree(heads); cudaFree(n_heads); cudaFree(qf); cudaFree(cub_tmp);
